@@ -1,0 +1,113 @@
+// accept_and_refresh: greedy acceptance walk, then commit of the accepted path into the
+// persistent per-sequence state of every layer.  Two kernels in stream order:
+//   aar_walk   (one CTA per sequence)        validates every layer, walks the tree, writes
+//                                            accept_len / accept_path / bonus_tok
+//   aar_commit (one CTA per sequence, layer) copies window rows, closed entries, open-block
+//                                            state; bumps L.  Reads the verdict of aar_walk,
+//                                            so all layers of a sequence commit or none does.
+#include "kernels.h"
+
+namespace tsv {
+
+__global__ void __launch_bounds__(32) aar_walk_kernel(const tsv_shape s, const AarLayers ls, const int32_t* __restrict__ parent,
+                                                      const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ draft,
+                                                      const int32_t* __restrict__ target, int32_t* __restrict__ accept_len,
+                                                      int32_t* __restrict__ accept_path, int32_t* __restrict__ bonus,
+                                                      int32_t* __restrict__ status, const int do_walk) {
+  __shared__ TreeMeta tm;
+  if (threadIdx.x != 0) return;
+  const int b = blockIdx.x, D = s.D;
+  int st = 0;
+  for (int l = 0; l < ls.n; ++l) {
+    build_tree_meta(tm, s, ls.l[l].c.L[b], parent + (size_t)b * D, n_nodes[b], ls.l[l].c.csa_cap + b, ls.l[l].c.hca_cap + b);
+    st |= tm.status;
+  }
+  if (st) atomicOr(status + b, st);
+  if (!do_walk) return;
+  st |= status[b];
+  int len = 0, bt = -1;
+  if (!st) {
+    const int32_t* dr = draft + (size_t)b * D;
+    const int32_t* tg = target + (size_t)b * D;
+    int cur = 0;
+    accept_path[(size_t)b * D + len++] = 0;
+    for (;;) {
+      int nxt = -1;
+      const int want = tg[cur];
+      for (int c = cur + 1; c < tm.nn; ++c)
+        if (tm.parent[c] == cur && dr[c] == want) { nxt = c; break; }
+      if (nxt < 0) break;
+      accept_path[(size_t)b * D + len++] = nxt;
+      cur = nxt;
+    }
+    bt = tg[cur];
+  }
+  for (int i = len; i < D; ++i) accept_path[(size_t)b * D + i] = -1;
+  accept_len[b] = len;
+  bonus[b] = bt;
+}
+
+__device__ __forceinline__ void copy_row16(void* dst, const void* src, int bytes, int tid, int nthr) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  for (int i = tid; i < bytes / 16; i += nthr) d4[i] = s4[i];
+}
+
+__global__ void __launch_bounds__(128) aar_commit_kernel(const tsv_shape s, const AarLayers ls, const int32_t* __restrict__ accept_len,
+                                                         const int32_t* __restrict__ accept_path, const int32_t* __restrict__ status) {
+  const int b = blockIdx.x, D = s.D;
+  const AarLayer& ly = ls.l[blockIdx.y];
+  const int al = accept_len[b];
+  if (status[b] != 0 || al <= 0) return;
+  const int L = ly.c.L[b];
+  __syncthreads();                      // every thread holds L before anyone moves it
+  const int es = s.dtype == TSV_BF16 ? 2 : 4;
+  const size_t rowb = (size_t)s.d * es, ikb = (size_t)s.di * es;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  for (int i = 0; i < al; ++i) {
+    const int n = accept_path[(size_t)b * D + i];
+    const int pos = L + i;
+    const size_t nidx = (size_t)b * D + n;
+    copy_row16((char*)ly.c.win_kv + ((size_t)b * s.window + pos % s.window) * rowb, (const char*)ly.node_kv + nidx * rowb, (int)rowb, tid, nt);
+    if (ly.sc.csa_done[nidx]) {
+      const size_t row = (size_t)ly.c.csa_row0[b] + pos / s.m_csa;
+      copy_row16((char*)ly.c.csa_kv + row * rowb, (const char*)ly.sc.new_csa_kv + nidx * rowb, (int)rowb, tid, nt);
+      copy_row16((char*)ly.c.csa_ik + row * ikb, (const char*)ly.sc.new_csa_ik + nidx * ikb, (int)ikb, tid, nt);
+    }
+    if (ly.sc.hca_done[nidx]) {
+      const size_t row = (size_t)ly.c.hca_row0[b] + pos / s.m_hca;
+      copy_row16((char*)ly.c.hca_kv + row * rowb, (const char*)ly.sc.new_hca_kv + nidx * rowb, (int)rowb, tid, nt);
+    }
+  }
+  const size_t last = (size_t)b * D + accept_path[(size_t)b * D + al - 1];
+  copy_row16(ly.c.csa_acc_kv + (size_t)b * s.d, ly.sc.csa_acc_kv + last * s.d, s.d * 4, tid, nt);
+  copy_row16(ly.c.csa_acc_ik + (size_t)b * s.di, ly.sc.csa_acc_ik + last * s.di, s.di * 4, tid, nt);
+  copy_row16(ly.c.hca_acc_kv + (size_t)b * s.d, ly.sc.hca_acc_kv + last * s.d, s.d * 4, tid, nt);
+  if (tid == 0) {
+    ly.c.csa_mx[b] = ly.sc.csa_mx[last]; ly.c.csa_s[b] = ly.sc.csa_s[last];
+    ly.c.hca_mx[b] = ly.sc.hca_mx[last]; ly.c.hca_s[b] = ly.sc.hca_s[last];
+    ly.c.L[b] = L + al;
+  }
+}
+
+int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const int32_t* parent, const int32_t* n_nodes,
+               const int32_t* draft, const int32_t* target, int32_t* accept_len, int32_t* accept_path,
+               int32_t* bonus, int32_t* status, cudaStream_t st) {
+  AarLayers ls;
+  for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
+    ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
+    for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
+    const int last = l0 + ls.n >= n_layers;
+    aar_walk_kernel<<<s.B, 32, 0, st>>>(s, ls, parent, n_nodes, draft, target, accept_len, accept_path, bonus, status, last);
+    count_launch();
+  }
+  for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
+    ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
+    for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
+    aar_commit_kernel<<<dim3(s.B, ls.n), 128, 0, st>>>(s, ls, accept_len, accept_path, status);
+    count_launch();
+  }
+  return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
+}
+
+}  // namespace tsv

@@ -1,0 +1,172 @@
+// C-ABI front end: argument validation on the host, workspace carve-up, kernel dispatch.
+// No allocation, no synchronisation, no state between calls.
+#include <math.h>
+
+#include <atomic>
+
+#include "kernels.h"
+
+namespace tsv {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static bool shape_ok(const tsv_shape* s) {
+  if (!s) return false;
+  if (s->dtype != TSV_FP32 && s->dtype != TSV_BF16) return false;
+  if (s->B < 1 || s->D < 1 || s->D > TSV_MAX_D || s->H < 1 || s->H > 256) return false;
+  if (s->d < 8 || s->d > 1024 || s->d % 8) return false;
+  if (s->di < 8 || s->di > 512 || s->di % 8) return false;
+  if (s->HI < 1 || s->HI > 16) return false;
+  if (s->m_csa < 1 || s->m_hca < 1 || s->topk < 1) return false;
+  if (s->window < s->D) return false;
+  if (s->max_L < s->D || s->max_L > (int64_t)1 << 30) return false;
+  return true;
+}
+
+static tsv_shape resolved(const tsv_shape* s) {
+  tsv_shape r = *s;
+  if (!(r.sm_scale > 0.f)) r.sm_scale = (float)(1.0 / sqrt((double)r.d));
+  return r;
+}
+
+static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
+  const int64_t pref = s.max_L / s.m_csa;
+  p.cand_cap = (int32_t)(pref + s.D);
+  p.need_scores = p.cand_cap > s.topk;
+  const int64_t ksel = p.cand_cap < s.topk ? p.cand_cap : s.topk;
+  p.keys_max = (int32_t)(ksel + s.max_L / s.m_hca + s.D + s.window + s.D);
+  const int hgroups = (s.H + 15) / 16;
+  const int64_t base = (int64_t)s.B * s.D * hgroups;
+  int64_t want = (2 * 148 + base - 1) / base;
+  if (want < 1) want = 1;
+  int64_t ks = (p.keys_max + want - 1) / want;
+  ks = (ks + 31) / 32 * 32;
+  if (ks < 64) ks = 64;
+  p.ks = (int32_t)ks;
+  p.nsplit = (int32_t)((p.keys_max + ks - 1) / ks);
+  size_t off = 0;
+  p.off_selcnt = off; off = up256(off + (size_t)s.B * s.D * sizeof(int32_t));
+  p.off_sel = off;    off = up256(off + (size_t)s.B * s.D * s.topk * sizeof(int32_t));
+  p.off_scores = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.cand_cap * sizeof(float));
+  p.off_po = off;     if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * s.d * sizeof(float));
+  p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
+  p.total = off;
+  return true;
+}
+
+static inline bool al16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+static int check_cache(const tsv_cache* c) {
+  if (!c) return TSV_ERR_NULL;
+  const void* all[] = {c->L, c->csa_kv, c->csa_ik, c->csa_row0, c->csa_cap, c->hca_kv, c->hca_row0, c->hca_cap, c->win_kv,
+                       c->csa_mx, c->csa_s, c->csa_acc_kv, c->csa_acc_ik, c->hca_mx, c->hca_s, c->hca_acc_kv};
+  for (const void* p : all) if (!p) return TSV_ERR_NULL;
+  const void* vec[] = {c->csa_kv, c->csa_ik, c->hca_kv, c->win_kv, c->csa_acc_kv, c->csa_acc_ik, c->hca_acc_kv};
+  for (const void* p : vec) if (!al16(p)) return TSV_ERR_ALIGN;
+  return TSV_OK;
+}
+
+static int check_nodes(const tsv_nodes* n, bool attn) {
+  if (!n) return TSV_ERR_NULL;
+  const void* base[] = {n->kv, n->c_csa, n->ikc, n->g_csa, n->c_hca, n->g_hca, n->parent, n->n_nodes};
+  for (const void* p : base) if (!p) return TSV_ERR_NULL;
+  if (attn && (!n->q || !n->iq || !n->iw)) return TSV_ERR_NULL;
+  const void* vec[] = {n->kv, n->c_csa, n->ikc, n->c_hca, n->q, n->iq};
+  for (const void* p : vec) if (p && !al16(p)) return TSV_ERR_ALIGN;
+  return TSV_OK;
+}
+
+static int check_scratch(const tsv_scratch* s) {
+  if (!s) return TSV_ERR_NULL;
+  const void* all[] = {s->csa_mx, s->csa_s, s->csa_acc_kv, s->csa_acc_ik, s->hca_mx, s->hca_s, s->hca_acc_kv,
+                       s->new_csa_kv, s->new_csa_ik, s->new_hca_kv, s->csa_done, s->hca_done};
+  for (const void* p : all) if (!p) return TSV_ERR_NULL;
+  const void* vec[] = {s->csa_acc_kv, s->csa_acc_ik, s->hca_acc_kv, s->new_csa_kv, s->new_csa_ik, s->new_hca_kv};
+  for (const void* p : vec) if (!al16(p)) return TSV_ERR_ALIGN;
+  return TSV_OK;
+}
+
+}  // namespace tsv
+
+using namespace tsv;
+
+extern "C" {
+
+int tsv_version(void) { return 1000; }
+
+uint64_t tsv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* tsv_error_string(int code) {
+  switch (code) {
+    case TSV_OK: return "ok";
+    case TSV_ERR_NULL: return "a required pointer is NULL";
+    case TSV_ERR_ALIGN: return "a vector pointer is not 16-byte aligned";
+    case TSV_ERR_SHAPE: return "unsupported shape";
+    case TSV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TSV_ERR_CUDA: return "a CUDA runtime call failed";
+    case TSV_ERR_LIMIT: return "size beyond a built-in maximum of this entry point";
+    default: return "unknown error code";
+  }
+}
+
+size_t tsv_workspace_bytes(const tsv_shape* shape) {
+  if (!shape_ok(shape)) return 0;
+  TvaPlan p;
+  make_tva_plan(resolved(shape), p);
+  return p.total;
+}
+
+int branch_state_build(const tsv_shape* shape, const tsv_cache* cache, const tsv_nodes* nodes, const tsv_scratch* scratch,
+                       int32_t* status, void* stream) {
+  if (!shape || !status) return TSV_ERR_NULL;
+  if (!shape_ok(shape)) return TSV_ERR_SHAPE;
+  int r;
+  if ((r = check_cache(cache)) || (r = check_nodes(nodes, false)) || (r = check_scratch(scratch))) return r;
+  return launch_bsb(resolved(shape), *cache, *nodes, *scratch, status, (cudaStream_t)stream);
+}
+
+int tree_verify_attn(const tsv_shape* shape, const tsv_cache* cache, const tsv_nodes* nodes, const tsv_scratch* scratch,
+                     void* out, int32_t* topk_idx, void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+  if (!shape || !status || !out) return TSV_ERR_NULL;
+  if (!shape_ok(shape)) return TSV_ERR_SHAPE;
+  int r;
+  if ((r = check_cache(cache)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
+  if (!al16(out)) return TSV_ERR_ALIGN;
+  const tsv_shape s = resolved(shape);
+  TvaPlan p;
+  make_tva_plan(s, p);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < p.total) return TSV_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!(s.flags & TSV_FLAG_SKIP_SELECT))
+    if ((r = launch_tva_select(s, p, *cache, *nodes, *scratch, topk_idx, (char*)workspace, status, st))) return r;
+  if (s.flags & TSV_FLAG_SKIP_ATTN) return TSV_OK;
+  return launch_tva_simt(s, p, *cache, *nodes, *scratch, out, (char*)workspace, status, st);
+}
+
+int accept_and_refresh(const tsv_shape* shape, int32_t n_layers, const tsv_cache* const* caches, const tsv_nodes* const* nodes,
+                       const tsv_scratch* const* scratch, const int32_t* draft_tok, const int32_t* target_tok,
+                       int32_t* accept_len, int32_t* accept_path, int32_t* bonus_tok, int32_t* status, void* stream) {
+  if (!shape || !caches || !nodes || !scratch || !draft_tok || !target_tok || !accept_len || !accept_path || !bonus_tok || !status)
+    return TSV_ERR_NULL;
+  if (!shape_ok(shape)) return TSV_ERR_SHAPE;
+  if (n_layers < 1 || n_layers > 4096) return TSV_ERR_SHAPE;
+  AarLayer stackbuf[64];
+  AarLayer* ls = n_layers <= 64 ? stackbuf : new AarLayer[n_layers];
+  int r = TSV_OK;
+  for (int l = 0; l < n_layers && !r; ++l) {
+    if ((r = check_cache(caches[l])) || (r = check_nodes(nodes[l], false)) || (r = check_scratch(scratch[l]))) break;
+    ls[l].c = *caches[l];
+    ls[l].node_kv = nodes[l]->kv;
+    ls[l].sc = *scratch[l];
+  }
+  if (!r)
+    r = launch_aar(resolved(shape), n_layers, ls, nodes[0]->parent, nodes[0]->n_nodes, draft_tok, target_tok, accept_len,
+                   accept_path, bonus_tok, status, (cudaStream_t)stream);
+  if (ls != stackbuf) delete[] ls;
+  return r;
+}
+
+}  // extern "C"

@@ -1,0 +1,101 @@
+// Shared device helpers of the tree-verify kernels: storage-dtype access, tree metadata
+// derived on the device from the raw parent array (depth, ancestor masks, validity).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tsv.h"
+
+namespace tsv {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- storage dtype access
+template <typename T> struct Vec;   // 16-byte vector of storage elements
+template <> struct Vec<float> { static constexpr int N = 4; };
+template <> struct Vec<bf16> { static constexpr int N = 8; };
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(bf16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+// 16-byte load of Vec<T>::N storage elements, widened to fp32.
+__device__ __forceinline__ void ld16(const float* p, float* o) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+__device__ __forceinline__ void ld16(const bf16* p, float* o) {
+  uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    o[2 * i] = __uint_as_float(w[i] << 16);
+    o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void st16(float* p, const float* v) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void st16(bf16* p, const float* v) {
+  uint4 o;
+  uint32_t* w = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&h);
+  }
+  *reinterpret_cast<uint4*>(p) = o;
+}
+
+// ---------------------------------------------------------------- tree metadata
+// Built by ONE thread of a CTA into shared memory, then read by all after a barrier.
+struct TreeMeta {
+  int32_t L;            // committed length of this sequence in this layer
+  int32_t nn;           // valid nodes
+  int32_t status;       // TSV_ST_* found here (0 = usable)
+  int32_t n_csa, n_hca; // committed entries
+  int32_t depth[TSV_MAX_D];
+  int32_t parent[TSV_MAX_D];
+  uint32_t anc[TSV_MAX_D];   // bit j set iff j == n or j is an ancestor of n
+};
+
+// Validates and derives the per-sequence tree facts.  `caps` may be null (capacity unchecked).
+__device__ inline void build_tree_meta(TreeMeta& tm, const tsv_shape& s, int32_t L, const int32_t* parent_b,
+                                       int32_t nn, const int32_t* csa_cap_b, const int32_t* hca_cap_b) {
+  int st = 0;
+  if (nn < 1 || nn > s.D) { st |= TSV_ST_NODES; nn = 0; }
+  if (L < 0 || (int64_t)L + s.D > s.max_L) { st |= TSV_ST_LENGTH; L = 0; }
+  for (int n = 0; n < TSV_MAX_D; ++n) { tm.depth[n] = 0; tm.parent[n] = -1; tm.anc[n] = 0; }
+  for (int n = 0; n < nn; ++n) {
+    int p = parent_b[n];
+    if (n == 0) {
+      if (p != -1) st |= TSV_ST_PARENT;
+      tm.anc[0] = 1u;
+    } else if (p < 0 || p >= n) {
+      st |= TSV_ST_PARENT;
+    } else {
+      tm.parent[n] = p;
+      tm.depth[n] = tm.depth[p] + 1;
+      tm.anc[n] = tm.anc[p] | (1u << n);
+    }
+  }
+  if (csa_cap_b && (L + s.D) / s.m_csa > *csa_cap_b) st |= TSV_ST_CSA_CAP;
+  if (hca_cap_b && (L + s.D) / s.m_hca > *hca_cap_b) st |= TSV_ST_HCA_CAP;
+  tm.L = L; tm.nn = nn; tm.status = st;
+  tm.n_csa = L / s.m_csa; tm.n_hca = L / s.m_hca;
+}
+
+__device__ __forceinline__ float softmax_scale(const tsv_shape& s) {
+  return s.sm_scale > 0.f ? s.sm_scale : rsqrtf((float)s.d);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace tsv

@@ -1,0 +1,42 @@
+// Internal interface between the C-ABI front end (api.cu) and the kernel files.
+#pragma once
+#include "common.cuh"
+
+namespace tsv {
+
+void count_launch(int n = 1);   // bumps the reporting counter behind tsv_kernel_launches()
+
+// Per-layer pointers accept_and_refresh needs, packed so that a group of layers fits in
+// kernel-parameter space.
+struct AarLayer {
+  tsv_cache c;
+  const void* node_kv;
+  tsv_scratch sc;
+};
+constexpr int kAarLayersPerLaunch = 12;
+struct AarLayers {
+  AarLayer l[kAarLayersPerLaunch];
+  int32_t n;
+};
+
+// Workspace carve-up of tree_verify_attn (byte offsets from a 256-byte aligned base).
+struct TvaPlan {
+  int32_t cand_cap;      // max CSA candidates per node (committed + in-tree)
+  int32_t need_scores;   // cand_cap > topk: some node may have to rank its candidates
+  int32_t keys_max;      // max keys one node can attend to
+  int32_t ks;            // keys per split (CUDA-core path)
+  int32_t nsplit;        // max splits per node
+  size_t off_selcnt, off_sel, off_scores, off_po, off_pml, total;
+};
+bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
+
+int launch_bsb(const tsv_shape& s, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, int32_t* status, cudaStream_t st);
+int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const int32_t* parent, const int32_t* n_nodes,
+               const int32_t* draft, const int32_t* target, int32_t* accept_len, int32_t* accept_path,
+               int32_t* bonus, int32_t* status, cudaStream_t st);
+int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
+int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                    void* out, char* ws, int32_t* status, cudaStream_t st);
+
+}  // namespace tsv

@@ -1,0 +1,247 @@
+// CSA selection for tree_verify_attn: indexer scores of the committed entries and the exact
+// per-node top-k (ties to the lower block index, ascending output).
+//
+//   idx_score_kernel  thread-per-entry; the entry's indexer key stays in flight in registers
+//                     16 bytes at a time, the indexer queries of a group of nodes sit in shared
+//                     memory (broadcast reads).  Skipped (early exit) for sequences where every
+//                     node has at most topk candidates -- then the selection is "everything".
+//   topk_kernel       one CTA per (sequence, node): 4-pass 8-bit radix select on the order-
+//                     preserving integer image of the fp32 score, then one ordered compaction
+//                     pass.  In-tree entries (closed at strict ancestors) are scored here.
+#include "kernels.h"
+
+namespace tsv {
+
+// Strict ancestors of n that closed a CSA / HCA block, root first (ascending block index).
+struct PathEntries {
+  int32_t n_newc, n_newh;
+  int32_t newc[TSV_MAX_D], newc_blk[TSV_MAX_D];
+  int32_t newh[TSV_MAX_D];
+};
+
+__device__ inline void path_entries(PathEntries& pe, const TreeMeta& tm, const tsv_shape& s, int n,
+                                    const uint8_t* csa_done_b, const uint8_t* hca_done_b) {
+  pe.n_newc = pe.n_newh = 0;
+  const uint32_t a = tm.anc[n] & ~(1u << n);
+  for (int j = 0; j < n; ++j) {
+    if (!((a >> j) & 1u)) continue;
+    if (csa_done_b[j]) { pe.newc[pe.n_newc] = j; pe.newc_blk[pe.n_newc++] = (tm.L + tm.depth[j]) / s.m_csa; }
+    if (hca_done_b[j]) pe.newh[pe.n_newh++] = j;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                        const tsv_scratch sc, char* __restrict__ ws) {
+  extern __shared__ float iq_s[];                 // [<=32 (node, head) pairs][di]
+  __shared__ TreeMeta tm;
+  __shared__ int need_any;
+  __shared__ uint32_t need_mask;
+  const int b = blockIdx.y, D = s.D, di = s.di, HI = s.HI;
+  if (threadIdx.x == 0) {
+    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], nullptr, nullptr);
+    uint32_t m = 0;
+    if (!tm.status)
+      for (int n = 0; n < tm.nn; ++n) {
+        int extra = 0;
+        for (int j = 0; j < n; ++j)
+          if (((tm.anc[n] >> j) & 1u) && sc.csa_done[(size_t)b * D + j]) ++extra;
+        if (tm.n_csa + extra > s.topk) m |= 1u << n;
+      }
+    need_mask = m; need_any = m != 0;
+  }
+  __syncthreads();
+  if (!need_any || (int)(blockIdx.x * blockDim.x) >= tm.n_csa) return;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool live = e < tm.n_csa;
+  const T* ikrow = reinterpret_cast<const T*>(c.csa_ik) + ((size_t)c.csa_row0[b] + (live ? e : 0)) * di;
+  float* scores = reinterpret_cast<float*>(ws + pl.off_scores) + (size_t)b * D * pl.cand_cap;
+  constexpr int V = Vec<T>::N;
+  const int npg = 32 / HI;                        // nodes per group
+  for (int n0 = 0; n0 < tm.nn; n0 += npg) {
+    const int gn = min(npg, tm.nn - n0), G = gn * HI;
+    __syncthreads();
+    for (int i = threadIdx.x; i < G * di; i += blockDim.x)
+      iq_s[i] = to_f(reinterpret_cast<const T*>(nd.iq)[((size_t)b * D + n0) * HI * di + i]);
+    __syncthreads();
+    if (!((need_mask >> n0) & ((gn >= 32 ? 0xffffffffu : ((1u << gn) - 1u))))) continue;
+    float acc[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+    for (int cidx = 0; cidx < di / V; ++cidx) {
+      float kk[V];
+      ld16(ikrow + cidx * V, kk);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if (j < G) {
+          const float* qv = iq_s + j * di + cidx * V;
+#pragma unroll
+          for (int t = 0; t < V; ++t) acc[j] = fmaf(qv[t], kk[t], acc[j]);
+        }
+      }
+    }
+    if (live) {
+      for (int g = 0; g < gn; ++g) {
+        float sc_ = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if (j / HI == g && j < G) sc_ = fmaf(nd.iw[((size_t)b * D + n0 + g) * HI + (j % HI)], fmaxf(acc[j], 0.f), sc_);
+        }
+        scores[(size_t)(n0 + g) * pl.cand_cap + e] = sc_;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t order_key(float f) {       // larger float -> larger key
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive block scan of one int per thread (256 threads); returns the thread's offset and the total.
+__device__ __forceinline__ int block_excl_scan(int v, int* wsum /* shared[9] */, int& total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) wsum[w] = x;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int i = 0; i < 8; ++i) { const int t = wsum[i]; wsum[i] = run; run += t; }
+    wsum[8] = run;
+  }
+  __syncthreads();
+  total = wsum[8];
+  return wsum[w] + x - v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                   const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
+                                                   int32_t* __restrict__ status) {
+  __shared__ TreeMeta tm;
+  __shared__ PathEntries pe;
+  __shared__ float extra[TSV_MAX_D];
+  __shared__ int hist[256];
+  __shared__ int wsum[9];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_remaining;
+  const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk;
+  int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
+  int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
+  int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
+  if (threadIdx.x == 0) {
+    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], c.csa_cap + b, c.hca_cap + b);
+    if (tm.status && n == 0) atomicOr(status + b, tm.status);
+    if (!tm.status && n < tm.nn) path_entries(pe, tm, s, n, sc.csa_done + (size_t)b * D, sc.hca_done + (size_t)b * D);
+  }
+  __syncthreads();
+  if (tm.status || n >= tm.nn) {
+    for (int i = threadIdx.x; i < k; i += blockDim.x) { sel[i] = -1; if (usr) usr[i] = -1; }
+    if (threadIdx.x == 0) *selcnt = 0;
+    return;
+  }
+  const int n_csa = tm.n_csa, n_cand = n_csa + pe.n_newc;
+  if (n_cand <= k) {                                           // everything is selected: no ranking
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+      const int v = i < n_csa ? i : (i < n_cand ? pe.newc_blk[i - n_csa] : -1);
+      sel[i] = v; if (usr) usr[i] = v;
+    }
+    if (threadIdx.x == 0) *selcnt = n_cand;
+    return;
+  }
+  // scores of the in-tree entries on this node's path: warp w takes entries w, w+8, ...
+  {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * s.HI * s.di;
+    for (int i = w; i < pe.n_newc; i += 8) {
+      const T* ik = reinterpret_cast<const T*>(sc.new_csa_ik) + ((size_t)b * D + pe.newc[i]) * s.di;
+      float tot = 0.f;
+      for (int h = 0; h < s.HI; ++h) {
+        float p = 0.f;
+        for (int t = lane; t < s.di; t += 32) p = fmaf(to_f(iq[h * s.di + t]), to_f(ik[t]), p);
+        p = warp_sum(p);
+        tot = fmaf(nd.iw[((size_t)b * D + n) * s.HI + h], fmaxf(p, 0.f), tot);
+      }
+      if (lane == 0) extra[i] = tot;
+    }
+  }
+  if (threadIdx.x == 0) { sh_prefix = 0; sh_remaining = k; }
+  __syncthreads();
+  const float* scores = reinterpret_cast<const float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+  auto key_of = [&](int i) { return order_key(i < n_csa ? scores[i] : extra[i - n_csa]); };
+  uint32_t mask = 0;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t prefix = sh_prefix;
+    for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
+      const uint32_t key = key_of(i);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int rem = sh_remaining, cum = 0, bin = 255;
+      for (; bin > 0; --bin) {
+        if (cum + hist[bin] >= rem) break;
+        cum += hist[bin];
+      }
+      sh_prefix = prefix | ((uint32_t)bin << shift);
+      sh_remaining = rem - cum;
+    }
+    mask |= 0xFFu << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = sh_prefix;       // key of the k-th largest score
+  const int r = sh_remaining;           // how many of the scores equal to it are taken (lowest indices)
+  int eq_base = 0, out_base = 0;
+  for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
+    const int i = i0 + threadIdx.x;
+    uint32_t key = 0;
+    if (i < n_cand) key = key_of(i);
+    const int eq = (i < n_cand) && key == thr, gt = (i < n_cand) && key > thr;
+    int tot_eq, tot_take;
+    const int eq_rank = eq_base + block_excl_scan(eq, wsum, tot_eq);
+    const int take = gt || (eq && eq_rank < r);
+    const int pos = out_base + block_excl_scan(take, wsum, tot_take);
+    if (take) {
+      const int v = i < n_csa ? i : pe.newc_blk[i - n_csa];
+      sel[pos] = v; if (usr) usr[pos] = v;
+    }
+    eq_base += tot_eq; out_base += tot_take;
+  }
+  if (threadIdx.x == 0) *selcnt = k;
+}
+
+int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st) {
+  const bool bf = s.dtype == TSV_BF16;
+  if (p.need_scores) {
+    const int pref_cap = (int)(s.max_L / s.m_csa);
+    dim3 grid((pref_cap + 255) / 256, s.B);
+    const size_t sm = (size_t)32 * s.di * sizeof(float);
+    if (grid.x > 0) {
+      if (bf) {
+        cudaFuncSetAttribute(idx_score_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        idx_score_kernel<bf16><<<grid, 256, sm, st>>>(s, p, c, nd, sc, ws);
+      } else {
+        cudaFuncSetAttribute(idx_score_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        idx_score_kernel<float><<<grid, 256, sm, st>>>(s, p, c, nd, sc, ws);
+      }
+      count_launch();
+    }
+  }
+  dim3 g2(s.D, s.B);
+  if (bf) topk_kernel<bf16><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
+  else topk_kernel<float><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
+}
+
+}  // namespace tsv
