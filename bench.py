@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the verify-side hot path (one step = one full verify cycle over all layers:
+branch_state_build + tree_verify_attn per layer, then accept_and_refresh).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg4]
+
+Prints ONE JSON line (rank 0).  `value` is verified tree tokens per second (B*D tokens per cycle)
+with inputs resident in HBM and the cycle replayed from a CUDA graph; `e2e` is the same metric
+with every step's inputs copied from pinned host memory and the acceptance result read back.
+N > 1 runs N independent replicas (the path has no exchange step): weak scaling, no collective
+on the data path; only the barrier and the MAX-over-ranks of the device time use the process group.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+# dram bytes per tree_verify_attn attention launch at the bench workload, from the ncu capture
+# summarised under profiles/ (None until measured for the current kernel).
+NCU_ATTN_TRAFFIC_BYTES = None
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return {"hbm_gbs": float(j["hbm_gbs"]), "bf16_tflops": float(j["bf16_tflops"]),
+                "bf16_tflops_sustained": float(j.get("bf16_tflops_sustained", j["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill(); out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_sample(cfg, n_layers_sample: int, n_seq_sample: int, steps: int, warmup: int):
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload: the first
+    n_seq_sample sequences x n_layers_sample layers of the same seeded inputs, one verify cycle per step.
+    Returns verified tokens/s scaled to the full layer count, and a description of the sample."""
+    from oracle import tsv_oracle as O
+    from paper_2609_24698_b200 import synth
+    from paper_2609_24698_b200.workload import direct_arrays
+    sh = cfg.shape
+    lengths = synth.prefix_lengths(cfg)
+
+    def fresh_states():
+        st = []
+        for l in range(n_layers_sample):
+            row = []
+            for b in range(n_seq_sample):
+                a = direct_arrays(cfg, l, b, int(lengths[b]))
+                row.append(O.SeqState(int(lengths[b]), a["csa_kv"].astype(np.float64), a["csa_ik"].astype(np.float64),
+                                      a["hca_kv"].astype(np.float64), a["win"].astype(np.float64),
+                                      O.Partial(a["csa_mx"], a["csa_s"], [a["csa_acc_kv"].astype(np.float64), a["csa_acc_ik"].astype(np.float64)]),
+                                      O.Partial(a["hca_mx"], a["hca_s"], [a["hca_acc_kv"].astype(np.float64)])))
+            st.append(row)
+        return st
+
+    states = fresh_states()
+    times = []
+    n_sets = min(3, warmup + steps)
+    node_sets = [[{k: v[:n_seq_sample] for k, v in synth.node_inputs(cfg, l, c).items()} for l in range(n_layers_sample)]
+                 for c in range(n_sets)]
+    for it in range(warmup + steps):
+        c = it % n_sets
+        nodes = node_sets[c]
+        parent, n_nodes = synth.trees(cfg, c)
+        draft, target = synth.tokens(cfg, c, parent, n_nodes)
+        t0 = time.perf_counter()
+        O.verify_cycle(states, sh, nodes, parent[:n_seq_sample], n_nodes[:n_seq_sample], draft[:n_seq_sample], target[:n_seq_sample])
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    t_cycle_full_layers = float(np.mean(times)) * cfg.layers / n_layers_sample
+    tok_s = n_seq_sample * sh.D / t_cycle_full_layers
+    try:
+        import threadpoolctl
+        cores = max([p["num_threads"] for p in threadpoolctl.threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = (f"{n_seq_sample} of {sh.B} sequences x {n_layers_sample} of {cfg.layers} layers of {cfg.name}, "
+              f"{steps} verify cycles (mean {np.mean(times):.3f} s each), time scaled to {cfg.layers} layers")
+    return tok_s, float(np.mean(times)) * 1e3, cores, sample
+
+
+def run_reference(args, cfg):
+    """Reference arm = the fp64 CPU oracle on the host cores, bounded sample, same metric and config."""
+    from paper_2609_24698_b200 import dist as D
+    rank, _, world = D.env_world()
+    if rank != 0:
+        return
+    steps, warmup = max(1, min(args.steps, 5)), max(0, min(args.warmup, 1))
+    tok_s, ms, cores, sample = oracle_sample(cfg, n_layers_sample=min(2, cfg.layers), n_seq_sample=min(32, cfg.shape.B), steps=steps, warmup=warmup)
+    line = {"impl": "reference", "metric": "verified_tree_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": workload_config(cfg, args),
+            "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, args):
+    sh = cfg.shape
+    return {"workload": f"{cfg.name}: {cfg.layers}-layer stack, {sh.dtype}, batch {sh.B}, D={sh.D} random trees, prefixes "
+                        f"U[{cfg.L_min},{cfg.L_max}], H={sh.H}, d={sh.d}, CSA m={sh.m_csa} top-k={sh.topk} (indexer {sh.HI}x{sh.di}), "
+                        f"HCA m'={sh.m_hca}, window {sh.window}",
+            "global_batch": sh.B * max(1, args.gpus), "tree_nodes": sh.D, "layers": cfg.layers,
+            "parallelism": "single GPU" if args.gpus <= 1 else f"{args.gpus} independent replicas (no collective)",
+            "l2_policy": "inputs larger than L2: every cycle reads a different input set (q alone is 268 MB per cycle)",
+            "launch": "one CUDA graph replay per cycle"}
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def run_ours(args, cfg):
+    import torch
+    from paper_2609_24698_b200 import binding as tsv, dist as D, synth, workload as W
+
+    rank, local_rank, world = D.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the tree-verify path has no CPU fallback")
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    D.init("nccl")
+    if world > 1:                                     # replicas differ only by seed
+        from dataclasses import replace
+        cfg = replace(cfg, seed=cfg.seed + rank)
+    sh = cfg.shape
+    K, Wm = args.steps, max(3, args.warmup)
+    n_sets = 3
+    wl = W.build(cfg, cycles_headroom=2 * (K + Wm) + 8, n_sets=n_sets, device=dev)
+    eng = wl.engine
+    snap = eng.snapshot()
+    stream = torch.cuda.current_stream()
+
+    # ---- launch bookkeeping (our kernels per cycle) and graphs
+    n0 = tsv.kernel_launches()
+    eng.launch_cycle(wl.inputs[0])
+    torch.cuda.synchronize()
+    launches_per_cycle = tsv.kernel_launches() - n0
+    assert int(eng.status.sum()) == 0, "workload flagged by the device-side validation"
+    eng.restore(snap)
+    graphs = [eng.capture(inp) for inp in wl.inputs] if not args.no_graph else None
+
+    def step(i):
+        if graphs is not None:
+            graphs[i % n_sets].replay()
+        else:
+            eng.launch_cycle(wl.inputs[i % n_sets])
+
+    # ---- timed region: K cycles, inputs resident in HBM
+    for i in range(Wm):
+        step(i)
+    torch.cuda.synchronize(); D.barrier(); torch.cuda.synchronize()
+    clk = ClockSampler(torch.cuda.current_device()); clk.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(K):
+        step(Wm + i)
+    e1.record(stream)
+    torch.cuda.synchronize(); D.barrier(); torch.cuda.synchronize()
+    clocks = clk.stop()
+    sec_local = e0.elapsed_time(e1) * 1e-3
+    accepted = float(eng.accept_len.sum().item())
+    assert int(eng.status.sum()) == 0
+    value, sec = D.whole_job_throughput(sh.B * sh.D * K, sec_local, dev)
+
+    # ---- per-kernel pass (eager, CUDA events on the launching stream): attention kernel alone
+    eng.restore(snap)
+    sel_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_ATTN)
+    att_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_SELECT)
+    ev = []
+    t_parts = {"branch_state_build": [], "select": [], "attention": [], "accept_and_refresh": []}
+    for i in range(Wm + K):
+        inp = wl.inputs[i % n_sets]
+        eng.status.zero_()
+        marks = []
+        for l in range(eng.n_layers):
+            m = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            m[0].record(stream)
+            tsv.branch_state_build(eng.cshape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.status)
+            m[1].record(stream)
+            tsv.tree_verify_attn(sel_shape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+            m[2].record(stream)
+            tsv.tree_verify_attn(att_shape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+            m[3].record(stream)
+            marks.append(m)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path, eng.bonus, eng.status)
+        a1.record(stream)
+        if i >= Wm:
+            ev.append((marks, a0, a1))
+    torch.cuda.synchronize()
+    for marks, a0, a1 in ev:
+        for m in marks:
+            t_parts["branch_state_build"].append(m[0].elapsed_time(m[1]))
+            t_parts["select"].append(m[1].elapsed_time(m[2]))
+            t_parts["attention"].append(m[2].elapsed_time(m[3]))
+        t_parts["accept_and_refresh"].append(a0.elapsed_time(a1))
+    attn_ms = float(np.mean(t_parts["attention"]))
+
+    # ---- algorithmic work and roofline of the dominant kernel (attention)
+    parents = wl.inputs[0].layers[0].parent.cpu().numpy()
+    work = W.algorithmic_work(sh, cfg.layers, wl.lengths, parents)
+    pk = peaks()
+    attn_gbs = work["attn_bytes_per_layer"] / (attn_ms * 1e-3) / 1e9
+    attn_tf = work["attn_flops_per_layer"] / (attn_ms * 1e-3) / 1e12
+    roofline = {"bound": "hbm", "kernel": "tree_verify_attn attention kernel (one layer, all sequences)",
+                "achieved": attn_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / pk["hbm_gbs"],
+                "traffic": NCU_ATTN_TRAFFIC_BYTES, "peak_source": pk["source"], "launch_ms": attn_ms,
+                "algorithmic_bytes_per_launch": work["attn_bytes_per_layer"],
+                "tensor": {"achieved": attn_tf, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                           "frac": attn_tf / pk["bf16_tflops_sustained"], "flops_per_launch": work["attn_flops_per_layer"]}}
+    cycle_s = sec / K
+    cycle = {"full_bytes": work["full_bytes"], "cache_bytes": work["cache_bytes"], "flops": work["flops"],
+             "frac_hbm_full": work["full_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
+             "frac_hbm_cache": work["cache_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
+             "frac_tensor_sustained": work["flops"] / cycle_s / 1e12 / pk["bf16_tflops_sustained"],
+             "stage_ms_per_call_eager": {k: float(np.mean(v)) for k, v in t_parts.items()},
+             "accepted_tokens_per_cycle_last": accepted}
+
+    # ---- end to end: host buffers in, acceptance result out, every step
+    eng.restore(snap)
+    host_sets = [inp.pinned_host_copy() for inp in wl.inputs]
+    slot = wl.inputs[0]
+    g_slot = graphs[0] if graphs is not None else None
+    res_dev = [eng.accept_len, eng.accept_path, eng.bonus, eng.status]
+    res_host = [torch.empty_like(t, device="cpu").pin_memory() for t in res_dev]
+    h2d = d2h = 0
+
+    def e2e_step(i):
+        nonlocal h2d, d2h
+        h2d = slot.load_from_host(host_sets[i % n_sets])
+        if g_slot is not None:
+            g_slot.replay()
+        else:
+            eng.launch_cycle(slot)
+        d2h = 0
+        for hdst, dsrc in zip(res_host, res_dev):
+            hdst.copy_(dsrc, non_blocking=True)
+            d2h += dsrc.numel() * dsrc.element_size()
+        torch.cuda.synchronize()
+
+    for i in range(Wm):
+        e2e_step(i)
+    torch.cuda.synchronize(); D.barrier(); torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(K):
+        e2e_step(Wm + i)
+    e1.record(stream)
+    torch.cuda.synchronize(); D.barrier(); torch.cuda.synchronize()
+    e2e_value, _ = D.whole_job_throughput(sh.B * sh.D * K, e0.elapsed_time(e1) * 1e-3, dev)
+
+    line = {"metric": "verified_tree_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": sec / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": sh.dtype, "data": "synthetic", "config": workload_config(cfg, args), "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches_per_cycle * K), "roofline": roofline, "cycle": cycle}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            tok_s, ms, cores, sample = oracle_sample(cfg, n_layers_sample=min(2, cfg.layers), n_seq_sample=min(32, sh.B), steps=4, warmup=1)
+            line["cpu_baseline"] = {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample}
+        print(json.dumps(line), flush=True)
+    D.finalize()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2609_24698_b200 import synth
+    cfg = synth.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
