@@ -209,6 +209,31 @@ int accept_and_refresh(const tsv_shape *shape, int32_t n_layers, const tsv_cache
                        const int32_t *draft_tok, const int32_t *target_tok, int32_t *accept_len,
                        int32_t *accept_path, int32_t *bonus_tok, int32_t *status, void *stream);
 
+/*
+ * tree_verify_attn_static -- tree_verify_attn without a caller-provided workspace.
+ * (No counterpart in the paper: this is a convenience of this library.)
+ *
+ * For callers that cannot allocate device memory at the point of the call -- an engine that
+ * gives out all device memory from its own pool at start-up, a plug-in that must leave its
+ * host's allocator alone, a request loop where an allocation would stall the device.  The
+ * workspace lives in a device array of TSV_STATIC_WORKSPACE_BYTES built into the library
+ * (each GPU that loads the library holds that much until the process exits).  The call runs
+ * no cudaMalloc / cudaFree and no allocating library routine; inputs and outputs are still the
+ * caller's.  Arguments, results and status handling are those of tree_verify_attn.
+ *   - Shapes whose tsv_workspace_bytes() exceeds TSV_STATIC_WORKSPACE_BYTES are refused with
+ *     TSV_ERR_LIMIT and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last call left in
+ *     it.  Nothing in it has to start at zero -- every region is written before it is read
+ *     within a call -- but two calls that overlap on the GPU (different streams, no
+ *     dependency between them) race on it: order them.
+ */
+#define TSV_STATIC_WORKSPACE_BYTES (16u << 20)
+int tree_verify_attn_static(const tsv_shape *shape, const tsv_cache *cache, const tsv_nodes *nodes,
+                            const tsv_scratch *scratch, void *out, int32_t *topk_idx,
+                            int32_t *status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -248,3 +248,23 @@ def accept_and_refresh(shape: CShape, pack: LayerPack, draft_tok: torch.Tensor, 
                                 _ptr(accept_len), _ptr(accept_path), _ptr(bonus_tok), _ptr(status), _stream(stream))
     if r:
         raise TsvError(r, "accept_and_refresh")
+
+
+STATIC_WORKSPACE_BYTES = 16 << 20
+_lib.tree_verify_attn_static.restype = C.c_int
+_lib.tree_verify_attn_static.argtypes = [C.POINTER(CShape), C.POINTER(CCache), C.POINTER(CNodes), C.POINTER(CScratch),
+                                         _p, _p, _p, _p]
+
+
+def tree_verify_attn_static(shape: CShape, cache: LayerCache, nodes: NodeInputs, scratch: Scratch, out: torch.Tensor,
+                            topk_idx: Optional[torch.Tensor], status: torch.Tensor, stream=None) -> None:
+    """tree_verify_attn for callers that cannot allocate device memory (a serving engine that owns
+    the whole memory pool, a plug-in, a latency-critical loop): the workspace is an array built into
+    the library, so no workspace tensor is passed and the call allocates nothing.  Shapes that need
+    more than STATIC_WORKSPACE_BYTES raise TsvError(ERR_LIMIT).  Calls share that array: do not let
+    two of them overlap on the GPU, and make the first call on a device outside stream capture."""
+    cs, ns, ss = cache.struct(), nodes.struct(), scratch.struct()
+    r = _lib.tree_verify_attn_static(C.byref(shape), C.byref(cs), C.byref(ns), C.byref(ss), _ptr(out), _ptr(topk_idx),
+                                     _ptr(status), _stream(stream))
+    if r:
+        raise TsvError(r, "tree_verify_attn_static")

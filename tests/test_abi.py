@@ -18,7 +18,7 @@ def lib():
 def declared_functions():
     src = open(os.path.join(ROOT, "include", "tsv.h")).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"^\s*(?:const\s+)?(?:int|size_t|char\s*\*)\s*\*?\s*([a-z_][a-z0-9_]*)\s*\(", src, flags=re.M)))
+    return sorted(set(re.findall(r"^\s*(?:const\s+)?(?:int|size_t|uint64_t|char\s*\*)\s*\*?\s*([a-z_][a-z0-9_]*)\s*\(", src, flags=re.M)))
 
 
 def test_every_declared_symbol_is_exported(lib):
