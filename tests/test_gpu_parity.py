@@ -103,7 +103,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
                 if committed is not None:
                     for k in committed[l][b]:
                         committed[l][b][k] = np.concatenate([committed[l][b][k], nodes[l][k][b][path]], 0)
-        compare_caches(eng, states, sh, tol, committed)
+        compare_caches(eng, states, sh, tol, committed if (check_recompress is True or cyc == cycles - 1) else None)
     return (worst, eng, states) if return_engine else worst
 
 
@@ -193,6 +193,32 @@ def test_cfg3_peaked():
     from dataclasses import replace
     cfg = synth.CONFIGS["cfg3"]
     cfg = replace(cfg, shape=replace(cfg.shape, B=4, sm_scale=1.5), cfg_id=33, L_min=600, L_max=3000)
+    lockstep(cfg, cycles=2)
+
+
+def test_cfg4_full_size_stack_lockstep():
+    """8 layers x 64 sequences, the launch configuration the benchmark times.  Every cycle: branch states,
+    acceptance, committed caches of ALL (layer, sequence) pairs; attention outputs of all pairs on cycle 0 and of
+    a rotating sample later; recompression-from-scratch check of every pair after the last cycle."""
+    cfg = synth.CONFIGS["cfg4"]
+    rng = np.random.default_rng(4)
+    def pairs(cyc):
+        if cyc == 0:
+            return [(l, b) for l in range(cfg.layers) for b in range(cfg.shape.B)]
+        return [(int(rng.integers(0, cfg.layers)), int(rng.integers(0, cfg.shape.B))) for _ in range(24)]
+    lockstep(cfg, cycles=5, out_pairs=pairs, check_recompress="final")
+
+
+def test_cfg5_long_context():
+    """131072-token prefixes, top-k 2048 of 32768 candidates: ranked selection, split key lists, combine."""
+    lockstep(synth.CONFIGS["cfg5"], cycles=3, check_recompress="final")
+
+
+@pytest.mark.parametrize("D,B", [(5, 1), (6, 2), (7, 64), (8, 4)])
+def test_budget_and_batch_sweep(D, B):
+    """The paper's budgets D=5..8 and batch sizes from 1 to 64 on the benchmark's head shape, short prefixes."""
+    cfg = synth.Config(f"sweep_d{D}_b{B}", 60 + D, synth.Shape("bf16", B, D, 64, 512, 4, 512, 4, 128, 128, 128),
+                       L_min=100, L_max=420, seed=D)
     lockstep(cfg, cycles=2)
 
 
