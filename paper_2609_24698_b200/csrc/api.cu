@@ -53,6 +53,18 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   p.off_scores = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.cand_cap * sizeof(float));
   p.off_po = off;     if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * s.d * sizeof(float));
   p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
+  p.tc = tva_tc_eligible(s);
+  p.tc_nt = p.tc_maxk = p.tc_chmax = 0;
+  p.off_kptr = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = off;
+  if (p.tc) {
+    tva_tc_plan_sizes(s, p);
+    const size_t tiles = (size_t)s.B * p.tc_nt;
+    p.off_kptr = off;  off = up256(off + tiles * p.tc_maxk * sizeof(uint64_t));
+    p.off_kmask = off; off = up256(off + tiles * p.tc_maxk);
+    p.off_nkeys = off; off = up256(off + tiles * sizeof(int32_t));
+    p.off_tpo = off;   if (p.tc_chmax > 1) off = up256(off + tiles * p.tc_chmax * 128 * s.d * sizeof(float));
+    p.off_tpml = off;  if (p.tc_chmax > 1) off = up256(off + tiles * p.tc_chmax * 128 * 2 * sizeof(float));
+  }
   p.total = off;
   return true;
 }
@@ -143,6 +155,7 @@ int tree_verify_attn(const tsv_shape* shape, const tsv_cache* cache, const tsv_n
   if (!(s.flags & TSV_FLAG_SKIP_SELECT))
     if ((r = launch_tva_select(s, p, *cache, *nodes, *scratch, topk_idx, (char*)workspace, status, st))) return r;
   if (s.flags & TSV_FLAG_SKIP_ATTN) return TSV_OK;
+  if (p.tc) return launch_tva_tc(s, p, *cache, *nodes, *scratch, out, (char*)workspace, status, st);
   return launch_tva_simt(s, p, *cache, *nodes, *scratch, out, (char*)workspace, status, st);
 }
 

@@ -98,4 +98,26 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Exclusive block scan of one int per thread (256 threads); returns the thread's offset and the total.
+__device__ __forceinline__ int block_excl_scan_256(int v, int* wsum /* shared[9] */, int& total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) wsum[w] = x;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    for (int i = 0; i < 8; ++i) { const int t = wsum[i]; wsum[i] = run; run += t; }
+    wsum[8] = run;
+  }
+  __syncthreads();
+  total = wsum[8];
+  return wsum[w] + x - v;
+}
+
 }  // namespace tsv

@@ -27,6 +27,9 @@ struct TvaPlan {
   int32_t ks;            // keys per split (CUDA-core path)
   int32_t nsplit;        // max splits per node
   size_t off_selcnt, off_sel, off_scores, off_po, off_pml, total;
+  // tensor-core path (bf16, d = 512): row tiles per sequence, key-list capacity per tile, max chunks per tile
+  int32_t tc, tc_nt, tc_maxk, tc_chmax;
+  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml;
 };
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
 
@@ -38,5 +41,10 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
+
+bool tva_tc_eligible(const tsv_shape& s);
+void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                  void* out, char* ws, int32_t* status, cudaStream_t st);
 
 }  // namespace tsv

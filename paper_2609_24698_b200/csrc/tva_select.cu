@@ -98,28 +98,6 @@ __device__ __forceinline__ uint32_t order_key(float f) {       // larger float -
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Exclusive block scan of one int per thread (256 threads); returns the thread's offset and the total.
-__device__ __forceinline__ int block_excl_scan(int v, int* wsum /* shared[9] */, int& total) {
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  int x = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, x, o);
-    if (lane >= o) x += y;
-  }
-  __syncthreads();
-  if (lane == 31) wsum[w] = x;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int run = 0;
-    for (int i = 0; i < 8; ++i) { const int t = wsum[i]; wsum[i] = run; run += t; }
-    wsum[8] = run;
-  }
-  __syncthreads();
-  total = wsum[8];
-  return wsum[w] + x - v;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
@@ -207,9 +185,9 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     if (i < n_cand) key = key_of(i);
     const int eq = (i < n_cand) && key == thr, gt = (i < n_cand) && key > thr;
     int tot_eq, tot_take;
-    const int eq_rank = eq_base + block_excl_scan(eq, wsum, tot_eq);
+    const int eq_rank = eq_base + block_excl_scan_256(eq, wsum, tot_eq);
     const int take = gt || (eq && eq_rank < r);
-    const int pos = out_base + block_excl_scan(take, wsum, tot_take);
+    const int pos = out_base + block_excl_scan_256(take, wsum, tot_take);
     if (take) {
       const int v = i < n_csa ? i : pe.newc_blk[i - n_csa];
       sel[pos] = v; if (usr) usr[pos] = v;

@@ -1,0 +1,591 @@
+// tree_verify_attn on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 storage, d = 512.
+//
+// One CTA = (sequence, row tile, key chunk).  A row tile is 128 query rows = 128/H consecutive
+// tree nodes x H heads; all of them attend over the SAME staged key rows (key == value, MQA), so
+// S = Q K^T and O = P K are dense 128 x N x 512 contractions.  Which node sees which key is a
+// per-key bitmask applied to the S fragment after it is read back from tensor memory.
+//
+//   tc_plan_kernel   per (sequence, tile): the list of key rows visible to at least one node of
+//                    the tile (union of the nodes' CSA selections, HCA entries, window slots,
+//                    tree nodes, in-tree entries) as row pointers + node bitmasks.
+//   tc_attn_kernel   per (sequence, tile, chunk of <= 512 keys):
+//       phase 1  S[128 x CL] = Q K^T      tcgen05.mma kind::f16, A = Q sub-tile (smem, K-major),
+//                                         B = 256 key rows x 64 dims (smem, K-major), D in TMEM
+//       phase 2  exact softmax of the chunk on the fp32 S read with tcgen05.ld; P (bf16) is
+//                written back into TMEM over S with tcgen05.st
+//       phase 3  O[128 x 256] = P K[:, half]  twice; A = P from TMEM, B = 64 key rows x 256 dims
+//                (smem, MN-major); epilogue reads O with tcgen05.ld and stores bf16 rows
+//     Operand tiles stream through a ring of seven 32 KiB slots filled with 16-byte cp.async
+//     copies written in the 128-byte swizzle pattern (any row from any of the six source arrays,
+//     zero fill for padding), four stages ahead of the MMA issue; slots are released by
+//     tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
+//   tc_combine_kernel merges the chunks of tiles that needed more than one (fixed order).
+#include "kernels.h"
+
+namespace tsv {
+
+namespace tc {
+
+constexpr int DH = 512;             // head dim handled by this path
+constexpr int BM = 128;             // rows per tile
+constexpr int NC = 512;             // max keys per chunk (S columns in TMEM)
+constexpr int SLOT = 32768;
+constexpr int NS = 7;               // ring slots
+constexpr int LOOK = NS - 3;        // stages loaded ahead of the MMA issue
+constexpr int THREADS = 256;
+constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
+constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
+constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls before a wait gives up (then no later wait of the thread is attempted)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
+  // D fp32, A/B bf16, A K-major, M = 128
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Bounded wait on an mbarrier phase; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t a = smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;      // src-size 0: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, "
+      "%20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+        "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
+        "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+               "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Small {                       // first SMALL bytes of dynamic shared memory
+  uint64_t slot_free[NS];
+  uint64_t acc_bar;
+  uint32_t tmem_base;
+  uint32_t pad;
+  uint8_t kmask[NC];
+  float xch[2][BM];                   // row max, later row sum, exchanged between the two column halves
+};
+static_assert(sizeof(Small) <= SMALL, "small region overflow");
+
+// chunking of a tile's key list: nch chunks of CL keys (CL a multiple of 128, <= NC)
+__device__ __host__ __forceinline__ void chunking(int nk, int& nch, int& CL) {
+  nch = (nk + NC - 1) / NC;
+  if (nch < 1) nch = 1;
+  CL = (((nk + nch - 1) / nch) + 127) / 128 * 128;
+  if (CL < 128) CL = 128;
+}
+
+}  // namespace tc
+
+// ------------------------------------------------------------------------------------------------ plan
+__global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                      const tsv_scratch sc, char* __restrict__ ws) {
+  extern __shared__ uint8_t cmask[];                   // [cand_cap] node bits per committed CSA entry (ranked case only)
+  __shared__ TreeMeta tm;
+  __shared__ int wsum[9];
+  __shared__ int n_cand[8], win_lo[8];
+  __shared__ int dense;
+  const int tile = blockIdx.x, b = blockIdx.y, D = s.D, H = s.H;
+  const int npt = tc::BM / H, n0 = tile * npt;
+  const size_t tix = (size_t)b * pl.tc_nt + tile;
+  uint64_t* kptr = reinterpret_cast<uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
+  uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
+  int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
+  const int32_t* selcnt = reinterpret_cast<const int32_t*>(ws + pl.off_selcnt) + (size_t)b * D;
+  const int32_t* sel = reinterpret_cast<const int32_t*>(ws + pl.off_sel) + (size_t)b * D * s.topk;
+  const uint8_t* cdone = sc.csa_done + (size_t)b * D;
+  const uint8_t* hdone = sc.hca_done + (size_t)b * D;
+  if (threadIdx.x == 0) {
+    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], c.csa_cap + b, c.hca_cap + b);
+    int dn = 1;
+    for (int nl = 0; nl < npt; ++nl) {
+      const int n = n0 + nl;
+      int extra = 0;
+      if (n < tm.nn)
+        for (int j = 0; j < n; ++j) if (((tm.anc[n] >> j) & 1u) && cdone[j]) ++extra;
+      n_cand[nl] = tm.n_csa + extra;
+      if (n < tm.nn && n_cand[nl] > s.topk) dn = 0;
+      win_lo[nl] = max(0, tm.L + tm.depth[n < tm.nn ? n : 0] - s.window + 1);
+    }
+    dense = dn;
+  }
+  __syncthreads();
+  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) *nkeys = 0; return; }
+  const int nvalid = min(npt, tm.nn - n0);
+  const uint32_t validbits = (1u << nvalid) - 1u;
+  const int n_csa = tm.n_csa;
+  const size_t rowb = (size_t)s.d * 2;
+  if (!dense) {
+    for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] = 0;
+    __syncthreads();
+    for (int nl = 0; nl < nvalid; ++nl) {
+      const int n = n0 + nl, cnt = selcnt[n];
+      if (n_cand[nl] <= s.topk) { for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)(1u << nl); }
+      else for (int j = threadIdx.x; j < cnt; j += blockDim.x) { const int idx = sel[(size_t)n * s.topk + j]; if (idx < n_csa) cmask[idx] |= (uint8_t)(1u << nl); }
+      __syncthreads();
+    }
+  }
+  // committed CSA entries, in index order
+  int base = 0;
+  for (int i0 = 0; i0 < n_csa; i0 += blockDim.x) {
+    const int i = i0 + threadIdx.x;
+    const uint32_t m = i < n_csa ? (dense ? validbits : cmask[i]) : 0u;
+    int tot;
+    const int pos = base + block_excl_scan_256(m != 0, wsum, tot);
+    if (m) { kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)c.csa_row0[b] + i) * rowb); kmask[pos] = (uint8_t)m; }
+    base += tot;
+  }
+  // committed HCA entries
+  for (int i = threadIdx.x; i < tm.n_hca; i += blockDim.x) {
+    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + ((size_t)c.hca_row0[b] + i) * rowb); kmask[base + i] = (uint8_t)validbits;
+  }
+  base += tm.n_hca;
+  // committed window positions seen by at least one node of the tile
+  int lo = tm.L;
+  for (int nl = 0; nl < nvalid; ++nl) lo = min(lo, win_lo[nl]);
+  for (int i = threadIdx.x; i < tm.L - lo; i += blockDim.x) {
+    const int pos = lo + i;
+    uint32_t m = 0;
+    for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
+    kptr[base + i] = (uint64_t)((const char*)c.win_kv + ((size_t)b * s.window + pos % s.window) * rowb); kmask[base + i] = (uint8_t)m;
+  }
+  base += max(0, tm.L - lo);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    // tree nodes (ancestors-or-self) and the entries closed inside the tree at strict ancestors
+    for (int j = 0; j < tm.nn; ++j) {
+      uint32_t mt = 0, mc = 0, mh = 0;
+      for (int nl = 0; nl < nvalid; ++nl) {
+        const int n = n0 + nl;
+        if (!((tm.anc[n] >> j) & 1u)) continue;
+        mt |= 1u << nl;
+        if (j == n) continue;
+        if (hdone[j]) mh |= 1u << nl;
+        if (cdone[j]) {
+          bool in = n_cand[nl] <= s.topk;
+          if (!in) {                                         // ranked: is the entry's block index in the node's selection?
+            const int blk = (tm.L + tm.depth[j]) / s.m_csa, cnt = selcnt[n];
+            const int32_t* sl = sel + (size_t)n * s.topk;
+            int a = 0, z = cnt - 1;
+            while (a <= z) { const int mid = (a + z) >> 1; const int v = sl[mid]; if (v == blk) { in = true; break; } if (v < blk) a = mid + 1; else z = mid - 1; }
+          }
+          if (in) mc |= 1u << nl;
+        }
+      }
+      const size_t nrow = (size_t)b * D + j;
+      if (mt) { kptr[base] = (uint64_t)((const char*)nd.kv + nrow * rowb); kmask[base++] = (uint8_t)mt; }
+      if (mc) { kptr[base] = (uint64_t)((const char*)sc.new_csa_kv + nrow * rowb); kmask[base++] = (uint8_t)mc; }
+      if (mh) { kptr[base] = (uint64_t)((const char*)sc.new_hca_kv + nrow * rowb); kmask[base++] = (uint8_t)mh; }
+    }
+    *nkeys = base;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ attention
+namespace tc {
+
+// 16 key-row pointers per thread: keys (tid>>3) + 32 j of the chunk, j = 0..15.  They serve the
+// K stages of phase 1 (key tile kt, rows 32 i: j = 8 kt + i) and the V stages of phase 3
+// (64-key block kb, rows 32 i: j = 2 kb + i).
+struct KeyPtrs { const char* p[16]; uint32_t valid; };
+
+template <int KT>
+__device__ __forceinline__ void load_k_stage(const KeyPtrs& kp, uint32_t slot, int dk, int ntk, int tid) {
+  const int r0 = tid >> 3, c = tid & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (i * 32 < ntk) {
+      const int r = r0 + 32 * i;
+      cp16(slot + r * 128 + ((c ^ (r & 7)) << 4), kp.p[8 * KT + i] + dk * 128 + c * 16, (kp.valid >> (8 * KT + i)) & 1u);
+    }
+  }
+}
+template <int KB>
+__device__ __forceinline__ void load_v_stage(const KeyPtrs& kp, uint32_t slot, int half, int tid) {
+  const int r0 = tid >> 3, c = tid & 7;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int r = r0 + 32 * i;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      cp16(slot + j * 8192 + r * 128 + ((c ^ (r & 7)) << 4), kp.p[2 * KB + i] + (half * 4 + j) * 128 + c * 16, (kp.valid >> (2 * KB + i)) & 1u);
+  }
+}
+
+}  // namespace tc
+
+__global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape s, const TvaPlan pl, const tsv_nodes nd, void* __restrict__ out_,
+                                                                 char* __restrict__ ws, int32_t* __restrict__ status) {
+  using namespace tc;
+  extern __shared__ unsigned char smem_raw[];
+  const int chunk = blockIdx.x, tile = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int D = s.D, H = s.H;
+  const size_t tix = (size_t)b * pl.tc_nt + tile;
+  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
+  const int rows_seq = D * H;
+  const int row0 = tile * BM;                                   // first row of the tile within the sequence
+  bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
+  if (nk <= 0) {                                                // flagged sequence or padding-only tile: zeros
+    if (chunk == 0)
+      for (int i = tid; i < BM * DH / 8; i += THREADS)
+        if (row0 + i / (DH / 8) < rows_seq) reinterpret_cast<uint4*>(out)[i] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  int nch, CL;
+  chunking(nk, nch, CL);
+  if (chunk >= nch) return;
+  const int cbeg = chunk * CL, cend = min(nk, cbeg + CL);
+
+  // ---- shared memory carve-up (tiles need 1024-byte alignment for the 128-byte swizzle)
+  unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Small& sm = *reinterpret_cast<Small*>(base);
+  const uint32_t ring = smem_u32(base + SMALL);
+  int fail = 0;
+
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.slot_free[i])));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.acc_bar)));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // key masks of the chunk and this thread's 16 key-row pointers
+  const uint64_t* kptr_g = reinterpret_cast<const uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
+  const uint8_t* kmask_g = reinterpret_cast<const uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
+  for (int i = tid; i < NC; i += THREADS) sm.kmask[i] = (cbeg + i < cend) ? kmask_g[cbeg + i] : (uint8_t)0;
+  KeyPtrs kp;
+  kp.valid = 0;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const int key = cbeg + (tid >> 3) + 32 * j;
+    const bool v = key < cend;
+    kp.p[j] = v ? reinterpret_cast<const char*>(kptr_g[key]) : reinterpret_cast<const char*>(nd.q);
+    kp.valid |= (uint32_t)v << j;
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tm = sm.tmem_base;
+
+  // ---- stage stream
+  const int nkt = (CL + 255) / 256;                 // key tiles of <= 256 keys
+  const int per_dk = 1 + nkt;                       // one Q stage + nkt K stages per 64-wide slice of d
+  const int G1 = 8 * per_dk;                        // stages of phase 1
+  const int nvs = CL / 64;                          // V stages per half of d
+  const int GT = G1 + 2 * nvs;
+  const char* qsrc = reinterpret_cast<const char*>(nd.q) + ((size_t)b * rows_seq + row0) * DH * 2;
+
+  auto load_stage = [&](int g) {
+    if (g < GT) {
+      const uint32_t slot = ring + (uint32_t)(g % NS) * SLOT;
+      if (g < G1) {
+        const int dk = g / per_dk, r = g % per_dk;
+        if (r == 0) {                               // Q slice: 128 rows x 64 dims
+          const int r0 = tid >> 3, c = tid & 7;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int row = r0 + 32 * i;
+            cp16(slot + row * 128 + ((c ^ (row & 7)) << 4), qsrc + (size_t)row * DH * 2 + dk * 128 + c * 16, row0 + row < rows_seq);
+          }
+        } else {
+          const int kt = r - 1, ntk = min(256, CL - kt * 256);
+          if (kt == 0) load_k_stage<0>(kp, slot, dk, ntk, tid); else load_k_stage<1>(kp, slot, dk, ntk, tid);
+        }
+      } else {
+        const int gv = g - G1, half = gv / nvs, kb = gv % nvs;
+        switch (kb) {
+          case 0: load_v_stage<0>(kp, slot, half, tid); break;
+          case 1: load_v_stage<1>(kp, slot, half, tid); break;
+          case 2: load_v_stage<2>(kp, slot, half, tid); break;
+          case 3: load_v_stage<3>(kp, slot, half, tid); break;
+          case 4: load_v_stage<4>(kp, slot, half, tid); break;
+          case 5: load_v_stage<5>(kp, slot, half, tid); break;
+          case 6: load_v_stage<6>(kp, slot, half, tid); break;
+          default: load_v_stage<7>(kp, slot, half, tid); break;
+        }
+      }
+    }
+    cp_commit();
+  };
+
+  const uint32_t idesc_k256 = make_idesc(256, 0), idesc_k128 = make_idesc(128, 0), idesc_v = make_idesc(256, 1);
+  const int q4 = warp & 3, hh = warp >> 2;          // TMEM lane quarter of this warp; column half it works on
+  const int row = q4 * 32 + lane;
+  const uint32_t tlane = tm + ((uint32_t)(q4 * 32) << 16);
+  const uint32_t mybit = 1u << (row / H);
+  const float scale2 = s.sm_scale * 1.4426950408889634f;
+  float m_row = 0.f, l_row = 0.f;
+  uint32_t acc_parity = 0;
+
+  // epilogue of one half of d: O[128 x 256] in TMEM columns 256..511
+  auto epilogue = [&](int half) {
+    if (!fail && !mbar_wait(&sm.acc_bar, acc_parity)) fail = 1;
+    acc_parity ^= 1u;
+    fence_after();
+    const bool rowok = row0 + row < rows_seq;
+    if (nch == 1) {
+      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+      bf16* orow = out + (size_t)row * DH + half * 256 + hh * 128;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tlane + 256 + hh * 128 + c0, r);
+        if (rowok) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float f[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(r[v * 8 + t]) * inv;
+            st16(orow + c0 + v * 8, f);
+          }
+        }
+      }
+    } else {
+      float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((tix * pl.tc_chmax + chunk) * BM + row) * DH + half * 256 + hh * 128;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tlane + 256 + hh * 128 + c0, r);
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          *reinterpret_cast<float4*>(po + c0 + v * 4) = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                                                    __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+      }
+      if (half == 0 && hh == 0)
+        reinterpret_cast<float2*>(ws + pl.off_tpml)[(tix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_row, l_row);
+    }
+    fence_before();
+    __syncthreads();                                 // O columns may be overwritten by the next half
+    fence_after();
+  };
+
+  // exact softmax of the chunk: S (fp32, columns 0..CL) -> P (bf16 pairs, columns 0..CL/2)
+  auto softmax = [&]() {
+    if (!fail && !mbar_wait(&sm.acc_bar, acc_parity)) fail = 1;
+    acc_parity ^= 1u;
+    fence_after();
+    const int nblk = CL / 128;
+    float mx = -INFINITY;
+    for (int e = 0; e < 2; ++e) {
+      const int jb = 2 * e + hh;
+      if (jb < nblk) {
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(tlane + jb * 128 + c0, r);
+#pragma unroll
+          for (int t = 0; t < 32; ++t)
+            if (sm.kmask[jb * 128 + c0 + t] & mybit) mx = fmaxf(mx, __uint_as_float(r[t]));
+        }
+      }
+    }
+    sm.xch[hh][row] = mx;
+    __syncthreads();
+    mx = fmaxf(sm.xch[0][row], sm.xch[1][row]);
+    m_row = mx * scale2;                              // scale2 > 0
+    const float moff = (mx == -INFINITY) ? 0.f : m_row;
+    float sum = 0.f;
+    for (int e = 0; e < 2; ++e) {
+      const int jb = 2 * e + hh;
+      uint32_t pk[64];
+      if (jb < nblk) {
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(tlane + jb * 128 + c0, r);
+#pragma unroll
+          for (int t = 0; t < 32; t += 2) {
+            const uint32_t mk0 = sm.kmask[jb * 128 + c0 + t] & mybit, mk1 = sm.kmask[jb * 128 + c0 + t + 1] & mybit;
+            const float p0 = mk0 ? ex2(fmaf(__uint_as_float(r[t]), scale2, -moff)) : 0.f;
+            const float p1 = mk1 ? ex2(fmaf(__uint_as_float(r[t + 1]), scale2, -moff)) : 0.f;
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);       // low half = even key
+            const float2 back = __bfloat1622float2(h2);
+            sum += back.x + back.y;
+            pk[(c0 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        }
+      }
+      fence_before();
+      __syncthreads();                                // every warp has read S blocks 2e and 2e+1
+      fence_after();
+      if (jb < nblk) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) tmem_st16(tlane + jb * 64 + v * 16, pk + v * 16);
+      }
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    sm.xch[hh][row] = sum;
+    fence_before();
+    __syncthreads();
+    fence_after();
+    l_row = sm.xch[0][row] + sm.xch[1][row];
+  };
+
+  // prologue: LOOK stages in flight
+  for (int g = 0; g < LOOK; ++g) load_stage(g);
+
+  for (int g = 0; g < GT; ++g) {
+    cp_wait<LOOK - 1>();                              // stage g has landed (this thread's copies)
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (g == G1) softmax();                           // S complete -> P in TMEM (also syncs the CTA)
+    else if (g == G1 + nvs) epilogue(0);
+    fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      fence_after();
+      const uint32_t slot = ring + (uint32_t)(g % NS) * SLOT;
+      if (g < G1) {
+        const int dk = g / per_dk, r = g % per_dk;
+        if (r > 0) {
+          const int kt = r - 1, ntk = min(256, CL - kt * 256);
+          const uint32_t qslot = ring + (uint32_t)((dk * per_dk) % NS) * SLOT;
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_ss(tm + kt * 256, make_desc(qslot + ks * 32, 16, 1024), make_desc(slot + ks * 32, 16, 1024),
+                   ntk == 256 ? idesc_k256 : idesc_k128, (dk | ks) != 0);
+          mma_commit(&sm.slot_free[g % NS]);
+          if (r == per_dk - 1) mma_commit(&sm.slot_free[(dk * per_dk) % NS]);        // Q slice no longer needed
+          if (g == G1 - 1) mma_commit(&sm.acc_bar);
+        }
+      } else {
+        const int gv = g - G1, kb = gv % nvs;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_ts(tm + 256, tm + kb * 32 + ks * 8, make_desc(slot + ks * 2048, 8192, 1024), idesc_v, (kb | ks) != 0);
+        mma_commit(&sm.slot_free[g % NS]);
+        if (kb == nvs - 1) mma_commit(&sm.acc_bar);
+      }
+    }
+    // refill the slot of stage g-3 (its release was committed at least two iterations ago) with stage g+LOOK
+    const int rs = g - 3;
+    if (rs >= 0 && rs + NS < GT) {
+      if (!fail && !mbar_wait(&sm.slot_free[rs % NS], (uint32_t)(rs / NS) & 1u)) fail = 1;
+    }
+    load_stage(g + LOOK);
+  }
+  epilogue(1);
+  cp_wait<0>();
+  if (fail && lane == 0) atomicOr(status + b, TSV_ST_INTERNAL);
+  fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tm) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------ combine
+__global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, const TvaPlan pl, void* __restrict__ out_, const char* __restrict__ ws) {
+  using namespace tc;
+  const int tile = blockIdx.x, b = blockIdx.y;
+  const size_t tix = (size_t)b * pl.tc_nt + tile;
+  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
+  int nch, CL;
+  chunking(nk, nch, CL);
+  if (nk <= 0 || nch <= 1) return;
+  const int rows_seq = s.D * s.H, row0 = tile * BM;
+  bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
+  const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + tix * pl.tc_chmax * BM * DH;
+  const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + tix * pl.tc_chmax * BM;
+  for (int i = threadIdx.x; i < BM * DH / 8; i += blockDim.x) {
+    const int row = i / (DH / 8), c8 = i % (DH / 8);
+    if (row0 + row >= rows_seq) continue;
+    float m = -INFINITY;
+    for (int ch = 0; ch < nch; ++ch) { const float2 ml = pml[ch * BM + row]; if (ml.y > 0.f) m = fmaxf(m, ml.x); }
+    float l = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int ch = 0; ch < nch; ++ch) {
+      const float2 ml = pml[ch * BM + row];
+      if (!(ml.y > 0.f)) continue;
+      const float w = exp2f(ml.x - m);
+      l = fmaf(ml.y, w, l);
+      const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + row) * DH + c8 * 8);
+      const float4 a = p4[0], bq = p4[1];
+      o[0] = fmaf(a.x, w, o[0]); o[1] = fmaf(a.y, w, o[1]); o[2] = fmaf(a.z, w, o[2]); o[3] = fmaf(a.w, w, o[3]);
+      o[4] = fmaf(bq.x, w, o[4]); o[5] = fmaf(bq.y, w, o[5]); o[6] = fmaf(bq.z, w, o[6]); o[7] = fmaf(bq.w, w, o[7]);
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) o[t] *= inv;
+    st16(out + (size_t)row * DH + c8 * 8, o);
+  }
+}
+
+bool tva_tc_eligible(const tsv_shape& s) {
+  return s.dtype == TSV_BF16 && s.d == tc::DH && s.H >= 16 && s.H <= 128 && (128 % s.H) == 0 && !(s.flags & TSV_FLAG_FORCE_SIMT);
+}
+
+void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
+  const int npt = tc::BM / s.H;
+  p.tc_nt = (s.D * s.H + tc::BM - 1) / tc::BM;
+  const int64_t ksel = p.cand_cap < s.topk ? p.cand_cap : s.topk;
+  int64_t uni = (int64_t)npt * ksel;
+  if (uni > p.cand_cap) uni = p.cand_cap;
+  int64_t mk = uni + s.max_L / s.m_hca + s.window + 3 * (int64_t)s.D + 8;
+  p.tc_maxk = (int32_t)((mk + 127) / 128 * 128);
+  p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
+}
+
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                  void* out, char* ws, int32_t* status, cudaStream_t st) {
+  const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
+  if (plan_sm > 48 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
+    return TSV_ERR_CUDA;
+  tc_plan_kernel<<<dim3(p.tc_nt, s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);
+  count_launch();
+  if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
+  tc_attn_kernel<<<dim3(p.tc_chmax, p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
+  count_launch();
+  if (p.tc_chmax > 1) {
+    tc_combine_kernel<<<dim3(p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
+    count_launch();
+  }
+  return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
+}
+
+}  // namespace tsv
