@@ -17,6 +17,9 @@
  *     partial-block accumulators, gates and weights are fp32.
  *   - Row-major, innermost dimension contiguous, no padding.  Vector pointers must be
  *     16-byte aligned and d, di multiples of 8.
+ *   - Cache buffers (csa_kv, csa_ik, hca_kv, win_kv) must hold finite numbers in EVERY allocated
+ *     row, also in rows not committed yet (allocate them zero-filled): the tensor-core kernels
+ *     fetch whole 32-row boxes and multiply the unused rows by an exact zero weight.
  *   - Node n of sequence b sits at depth delta_n (root = node 0 = depth 0) and at position
  *     p_n = L[b] + delta_n.  n_csa = L / m_csa and n_hca = L / m_hca committed entries.
  *   - Return value: 0 or a negative TSV_ERR_* for problems the host can see BEFORE any
@@ -103,6 +106,8 @@ typedef struct tsv_cache {
   float *csa_acc_ik;          /* [B][di] weighted sum of indexer-key vectors                */
   float *hca_mx, *hca_s;      /* [B] open HCA block                                         */
   float *hca_acc_kv;          /* [B][d]                                                     */
+  int64_t csa_rows;           /* HOST value: rows allocated in csa_kv / csa_ik (all slabs)  */
+  int64_t hca_rows;           /* HOST value: rows allocated in hca_kv                       */
 } tsv_cache;
 
 /* Per-cycle inputs of ONE layer for all tree nodes; read-only. */

@@ -40,7 +40,11 @@ class CShape(C.Structure):
 
 class CCache(C.Structure):
     _fields_ = [(n, _p) for n in ("L", "csa_kv", "csa_ik", "csa_row0", "csa_cap", "hca_kv", "hca_row0", "hca_cap",
-                                  "win_kv", "csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")]
+                                  "win_kv", "csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")] + \
+               [("csa_rows", C.c_int64), ("hca_rows", C.c_int64)]
+
+
+CACHE_TENSORS = tuple(n for n, t in CCache._fields_ if t is _p)
 
 
 class CNodes(C.Structure):
@@ -121,10 +125,10 @@ class LayerCache:
     hca_acc_kv: torch.Tensor
 
     def struct(self) -> CCache:
-        return CCache(*[_ptr(getattr(self, n)) for n, _ in CCache._fields_])
+        return CCache(*[_ptr(getattr(self, n)) for n in CACHE_TENSORS], int(self.csa_kv.shape[0]), int(self.hca_kv.shape[0]))
 
     def clone(self) -> "LayerCache":
-        return LayerCache(*[getattr(self, n).clone() for n, _ in CCache._fields_])
+        return LayerCache(*[getattr(self, n).clone() for n in CACHE_TENSORS])
 
 
 @dataclass

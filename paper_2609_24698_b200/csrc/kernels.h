@@ -29,7 +29,8 @@ struct TvaPlan {
   size_t off_selcnt, off_sel, off_scores, off_po, off_pml, total;
   // tensor-core path (bf16, d = 512): row tiles per sequence, key-list capacity per tile, max chunks per tile
   int32_t tc, tc_nt, tc_maxk, tc_chmax;
-  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml;
+  int32_t tc_tma, tc_misc_rows;      // contiguous-run tiles go through TMA; rows of the per-sequence packed buffer
+  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc;
 };
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
 
@@ -42,7 +43,11 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
 
+constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
+bool tva_tc_tma_usable(const tsv_cache& c);
+int launch_tva_tc_tma(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
+                      int32_t* status, cudaStream_t st);
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                   void* out, char* ws, int32_t* status, cudaStream_t st);

@@ -1,0 +1,117 @@
+// Shared pieces of the tensor-core (tcgen05) attention kernels: PTX wrappers, descriptors,
+// the small shared-memory control block and the chunking rule.
+#pragma once
+#include "kernels.h"
+
+namespace tsv {
+
+namespace tc {
+
+constexpr int DH = 512;             // head dim handled by this path
+constexpr int BM = 128;             // rows per tile
+constexpr int NC = 512;             // max keys per chunk (S columns in TMEM)
+constexpr int SLOT = 32768;
+constexpr int NS = 7;               // ring slots
+constexpr int LOOK = NS - 3;        // stages loaded ahead of the MMA issue
+constexpr int THREADS = 256;
+constexpr int kHcaMiscMaxTc = 32;
+constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
+constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
+constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls before a wait gives up (then no later wait of the thread is attempted)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
+  // D fp32, A/B bf16, A K-major, M = 128
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Bounded wait on an mbarrier phase; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t a = smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;      // src-size 0: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, "
+      "%20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+        "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
+        "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+               "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct Small {                       // first SMALL bytes of dynamic shared memory
+  uint64_t slot_free[NS];
+  uint64_t acc_bar;
+  uint32_t tmem_base;
+  uint32_t pad;
+  uint8_t kmask[NC];
+  float xch[2][BM];                   // row max, later row sum, exchanged between the two column halves
+};
+static_assert(sizeof(Small) <= SMALL, "small region overflow");
+
+// chunking of a tile's key list: nch chunks of CL keys (CL a multiple of 128, <= NC)
+__device__ __host__ __forceinline__ void chunking(int nk, int& nch, int& CL) {
+  nch = (nk + NC - 1) / NC;
+  if (nch < 1) nch = 1;
+  CL = (((nk + nch - 1) / nch) + 127) / 128 * 128;
+  if (CL < 128) CL = 128;
+}
+
+constexpr int NCX = 768;             // max keys per chunk of the TMA kernel: P (bf16) takes 384 TMEM columns, an O quarter 128
+// chunking of the TMA kernel: nch chunks of CL keys, CL a multiple of 128 and <= NCX
+__device__ __host__ __forceinline__ void chunking_x(int nk, int& nch, int& CL) {
+  nch = (nk + NCX - 1) / NCX;
+  if (nch < 1) nch = 1;
+  CL = (((nk + nch - 1) / nch) + 127) / 128 * 128;
+  if (CL < 128) CL = 128;
+}
+
+}  // namespace tc
+
+}  // namespace tsv

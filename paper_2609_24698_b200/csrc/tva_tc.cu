@@ -20,108 +20,10 @@
 //     zero fill for padding), four stages ahead of the MMA issue; slots are released by
 //     tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
 //   tc_combine_kernel merges the chunks of tiles that needed more than one (fixed order).
-#include "kernels.h"
+#include "tc_common.cuh"
 
 namespace tsv {
 
-namespace tc {
-
-constexpr int DH = 512;             // head dim handled by this path
-constexpr int BM = 128;             // rows per tile
-constexpr int NC = 512;             // max keys per chunk (S columns in TMEM)
-constexpr int SLOT = 32768;
-constexpr int NS = 7;               // ring slots
-constexpr int LOOK = NS - 3;        // stages loaded ahead of the MMA issue
-constexpr int THREADS = 256;
-constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
-constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls before a wait gives up (then no later wait of the thread is attempted)
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  // shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
-  // D fp32, A/B bf16, A K-major, M = 128
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Bounded wait on an mbarrier phase; false if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  const uint32_t a = smem_u32(bar);
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
-__device__ __forceinline__ void cp16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;      // src-size 0: the 16 bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, "
-      "%20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
-        "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
-        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]),
-        "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-               "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-struct Small {                       // first SMALL bytes of dynamic shared memory
-  uint64_t slot_free[NS];
-  uint64_t acc_bar;
-  uint32_t tmem_base;
-  uint32_t pad;
-  uint8_t kmask[NC];
-  float xch[2][BM];                   // row max, later row sum, exchanged between the two column halves
-};
-static_assert(sizeof(Small) <= SMALL, "small region overflow");
-
-// chunking of a tile's key list: nch chunks of CL keys (CL a multiple of 128, <= NC)
-__device__ __host__ __forceinline__ void chunking(int nk, int& nch, int& CL) {
-  nch = (nk + NC - 1) / NC;
-  if (nch < 1) nch = 1;
-  CL = (((nk + nch - 1) / nch) + 127) / 128 * 128;
-  if (CL < 128) CL = 128;
-}
-
-}  // namespace tc
 
 // ------------------------------------------------------------------------------------------------ plan
 __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
@@ -156,11 +58,79 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
     dense = dn;
   }
   __syncthreads();
-  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) *nkeys = 0; return; }
+  int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
+  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = pl.tc_tma ? 1 : 0; } return; }
   const int nvalid = min(npt, tm.nn - n0);
   const uint32_t validbits = (1u << nvalid) - 1u;
   const int n_csa = tm.n_csa;
   const size_t rowb = (size_t)s.d * 2;
+  if (pl.tc_tma) {
+    // rows that are small and scattered (few HCA entries, tree nodes, entries closed inside the tree) are packed
+    // into one contiguous per-sequence buffer so that TMA boxes can fetch them: written by the CTA of tile 0
+    const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
+    int ncd = 0, nhd = 0;
+    for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
+    const int n_misc = nh_in + tm.nn + ncd + nhd;
+    if (tile == 0) {
+      uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
+      const int rows_out = (n_misc + 31) / 32 * 32, cpr = (int)(rowb / 16);
+      for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
+        const int r = i / cpr, cc = i % cpr;
+        const char* src = nullptr;
+        if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)c.hca_row0[b] + r) * rowb;
+        else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
+        else if (r < n_misc) {
+          int ord = r - nh_in - tm.nn;
+          const bool isc = ord < ncd;
+          if (!isc) ord -= ncd;
+          const uint8_t* dn = isc ? cdone : hdone;
+          int a = 0;
+          for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
+          src = (const char*)(isc ? sc.new_csa_kv : sc.new_hca_kv) + ((size_t)b * D + a) * rowb;
+        }
+        dst[i] = src ? reinterpret_cast<const uint4*>(src)[cc] : make_uint4(0, 0, 0, 0);
+      }
+    }
+    if (dense) {
+      int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / 32);
+      int kb = 0;
+      auto emit = [&](int map, int64_t start, int count, int seg) {
+        const int nb = (count + 31) / 32;
+        for (int i = threadIdx.x; i < nb; i += blockDim.x) box[kb / 32 + i] = make_int2(map, (int)(start + 32 * i));
+        for (int i = threadIdx.x; i < nb * 32; i += blockDim.x) {
+          uint32_t m = 0;
+          if (i < count) {
+            if (seg == 0 || seg == 1) m = validbits;
+            else if (seg == 2) {
+              const int pos = tm.L - 1 - ((tm.L - 1 - i) % s.window);
+              for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
+            } else if (i < nh_in) m = validbits;
+            else if (i < nh_in + tm.nn) {
+              const int j = i - nh_in;
+              for (int nl = 0; nl < nvalid; ++nl) if ((tm.anc[n0 + nl] >> j) & 1u) m |= 1u << nl;
+            } else {
+              int ord = i - nh_in - tm.nn;
+              const bool isc = ord < ncd;
+              if (!isc) ord -= ncd;
+              const uint8_t* dn = isc ? cdone : hdone;
+              int a = 0;
+              for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
+              for (int nl = 0; nl < nvalid; ++nl) if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u)) m |= 1u << nl;
+            }
+          }
+          kmask[kb + i] = (uint8_t)m;
+        }
+        kb += nb * 32;
+      };
+      emit(0, c.csa_row0[b], n_csa, 0);
+      if (tm.n_hca > kHcaMiscMax) emit(1, c.hca_row0[b], tm.n_hca, 1);
+      emit(2, (int64_t)b * s.window, min(tm.L, s.window), 2);
+      emit(3, (int64_t)b * pl.tc_misc_rows, n_misc, 3);
+      if (threadIdx.x == 0) { *nkeys = kb; *mode = 1; }
+      return;
+    }
+  }
+  if (threadIdx.x == 0) *mode = 0;
   if (!dense) {
     for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] = 0;
     __syncthreads();
@@ -268,6 +238,7 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int D = s.D, H = s.H;
   const size_t tix = (size_t)b * pl.tc_nt + tile;
+  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 0) return;      // a contiguous-run tile: the TMA kernel's
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   const int rows_seq = D * H;
   const int row0 = tile * BM;                                   // first row of the tile within the sequence
@@ -527,7 +498,7 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   const size_t tix = (size_t)b * pl.tc_nt + tile;
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   int nch, CL;
-  chunking(nk, nch, CL);
+  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] == 1) chunking_x(nk, nch, CL); else chunking(nk, nch, CL);
   if (nk <= 0 || nch <= 1) return;
   const int rows_seq = s.D * s.H, row0 = tile * BM;
   bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
@@ -567,20 +538,31 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   int64_t uni = (int64_t)npt * ksel;
   if (uni > p.cand_cap) uni = p.cand_cap;
   int64_t mk = uni + s.max_L / s.m_hca + s.window + 3 * (int64_t)s.D + 8;
+  p.tc_misc_rows = (kHcaMiscMax + 3 * s.D + 31) / 32 * 32;
+  const int64_t runs = (p.cand_cap + 31) / 32 * 32 + (s.max_L / s.m_hca + 31) / 32 * 32 + (s.window + 31) / 32 * 32 + p.tc_misc_rows;
+  if (runs > mk) mk = runs;
   p.tc_maxk = (int32_t)((mk + 127) / 128 * 128);
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
 }
 
-int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
+  TvaPlan p = p_in;
+  p.tc_tma = tva_tc_tma_usable(c) ? 1 : 0;
   const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
   if (plan_sm > 48 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
     return TSV_ERR_CUDA;
   tc_plan_kernel<<<dim3(p.tc_nt, s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);
   count_launch();
-  if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
-  tc_attn_kernel<<<dim3(p.tc_chmax, p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
-  count_launch();
+  if (p.tc_tma) {
+    const int r = launch_tva_tc_tma(s, p, c, nd, out, ws, status, st);
+    if (r != TSV_OK) return r;
+  }
+  if (!p.tc_tma || p.need_scores) {            // tiles with ranked selections (or no TMA): pointer-gather kernel
+    if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
+    tc_attn_kernel<<<dim3(p.tc_chmax, p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
+    count_launch();
+  }
   if (p.tc_chmax > 1) {
     tc_combine_kernel<<<dim3(p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
     count_launch();

@@ -163,5 +163,5 @@ class VerifyEngine:
 
     def restore(self, snap: List[tsv.LayerCache]) -> None:
         for c, s in zip(self.caches, snap):
-            for name, _ in tsv.CCache._fields_:
+            for name in tsv.CACHE_TENSORS:
                 getattr(c, name).copy_(getattr(s, name))

@@ -53,7 +53,7 @@ def test_workspace_bytes_and_shape_validation(lib):
 def test_host_errors_return_before_any_launch(lib):
     from paper_2609_24698_b200 import binding as tsv
     fake = 0x10000                                           # never dereferenced: validation fails first
-    cache = tsv.CCache(*[fake] * len(tsv.CCache._fields_))
+    cache = tsv.CCache(*[fake] * len(tsv.CACHE_TENSORS), 1 << 20, 1 << 20)
     nodes = tsv.CNodes(*[fake] * len(tsv.CNodes._fields_))
     scr = tsv.CScratch(*[fake] * len(tsv.CScratch._fields_))
     s = _shape()
@@ -62,7 +62,7 @@ def test_host_errors_return_before_any_launch(lib):
     assert f(C.byref(s), None, C.byref(nodes), C.byref(scr), fake, None) == tsv.ERR_NULL
     assert f(C.byref(s), C.byref(cache), C.byref(nodes), C.byref(scr), None, None) == tsv.ERR_NULL
     assert f(C.byref(_shape(D=40)), C.byref(cache), C.byref(nodes), C.byref(scr), fake, None) == tsv.ERR_SHAPE
-    c2 = tsv.CCache(*[fake] * len(tsv.CCache._fields_)); c2.csa_kv = fake + 8
+    c2 = tsv.CCache(*[fake] * len(tsv.CACHE_TENSORS), 1 << 20, 1 << 20); c2.csa_kv = fake + 8
     assert f(C.byref(s), C.byref(c2), C.byref(nodes), C.byref(scr), fake, None) == tsv.ERR_ALIGN
     n2 = tsv.CNodes(*[fake] * len(tsv.CNodes._fields_)); n2.parent = None
     assert f(C.byref(s), C.byref(cache), C.byref(n2), C.byref(scr), fake, None) == tsv.ERR_NULL

@@ -55,7 +55,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
         torch.cuda.synchronize()
         # isolation: the first two calls leave every persistent byte unchanged
         for c0, c1 in zip(before, eng.caches):
-            for name, _ in tsv.CCache._fields_:
+            for name in tsv.CACHE_TENSORS:
                 assert torch.equal(getattr(c0, name), getattr(c1, name)), f"{name} changed before acceptance"
         tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path,
                                eng.bonus, eng.status)
