@@ -98,12 +98,14 @@ int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const i
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
     for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
     const int last = l0 + ls.n >= n_layers;
+    TSV_PREP(aar_walk_kernel);
     aar_walk_kernel<<<s.B, 32, 0, st>>>(s, ls, parent, n_nodes, draft, target, accept_len, accept_path, bonus, status, last);
     count_launch();
   }
   for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
     for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
+    TSV_PREP(aar_commit_kernel);
     aar_commit_kernel<<<dim3(s.B, ls.n), 128, 0, st>>>(s, ls, accept_len, accept_path, status);
     count_launch();
   }

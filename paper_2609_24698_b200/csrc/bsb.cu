@@ -1,8 +1,11 @@
 // branch_state_build: chain-private online compression along every root-to-node path.
-// One CTA per sequence.  Thread 0 derives the tree facts and the scalar part of every fold
-// (max gate, sum of weights, the two blend coefficients); then each thread owns a fixed set
-// of vector elements and walks the nodes in index order (parents first), so the parent's
-// post-fold value of an element is always one this same thread wrote earlier.
+//
+// Grid (sequence, element slab).  The scalar part of every fold (max gate, sum of weights, the two
+// blend coefficients, done flags) is a chain over at most 32 nodes: thread 0 of each CTA loads all
+// gates and parents up front (independent loads, one memory latency) and walks the chain in
+// registers.  Each thread then owns ONE vector element: it loads that element of every node's
+// compression vector up front, folds along the tree with the inherited values kept in shared
+// memory (indexed by parent), and stores states and closed entries.  No load depends on a store.
 #include "kernels.h"
 
 namespace tsv {
@@ -13,7 +16,7 @@ struct FoldCoef {
   int32_t empty;     // the inherited block holds no token (inherited numbers are ignored)
 };
 
-__device__ inline void scalar_fold(FoldCoef& fc, float& mx_out, float& s_out, int p, int blk, float mxp, float sp, float g) {
+__device__ __forceinline__ void scalar_fold(FoldCoef& fc, float& mx_out, float& s_out, int p, int blk, float mxp, float sp, float g) {
   const bool empty = (p % blk) == 0;
   float mx2, a, b, s2;
   if (empty) { mx2 = g; a = 0.f; b = 1.f; s2 = 1.f; }
@@ -29,67 +32,110 @@ __device__ inline void scalar_fold(FoldCoef& fc, float& mx_out, float& s_out, in
   s_out = fc.done ? 0.f : s2;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(128) bsb_kernel(const tsv_shape s, const tsv_cache c, const tsv_nodes nd,
-                                                  const tsv_scratch sc, int32_t* __restrict__ status) {
+constexpr int kBsbThreads = 128;
+
+template <typename T, int DMAX>
+__global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, const tsv_cache c, const tsv_nodes nd,
+                                                          const tsv_scratch sc, int32_t* __restrict__ status) {
+  extern __shared__ float hist[];                      // [D][kBsbThreads] post-fold value of this thread's element per node
   __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
   __shared__ FoldCoef fcs[TSV_MAX_D], fhs[TSV_MAX_D];
+  __shared__ float cmx[TSV_MAX_D], cs[TSV_MAX_D], hmx[TSV_MAX_D], hs[TSV_MAX_D];   // thread 0's chain state per node
   const int b = blockIdx.x, D = s.D;
+  const int d = s.d, di = s.di;
+  const int e = blockIdx.y * kBsbThreads + threadIdx.x;   // element index: [0,d) CSA kv | [d,d+di) CSA indexer key | [d+di,2d+di) HCA kv
+  const bool live = e < 2 * d + di;
+  const int which = e < d ? 0 : (e < d + di ? 1 : 2);
+  const int el = which == 0 ? e : (which == 1 ? e - d : e - d - di);
+  const int dim = which == 1 ? di : d;
+  const T* cin = reinterpret_cast<const T*>(which == 0 ? nd.c_csa : (which == 1 ? nd.ikc : nd.c_hca));
+  const float* pers = which == 0 ? c.csa_acc_kv : (which == 1 ? c.csa_acc_ik : c.hca_acc_kv);
+  // issue this thread's loads before the scalar chain is known (padding slots load too: the memory is there)
+  float cv[DMAX];
+#pragma unroll
+  for (int n = 0; n < DMAX; ++n) cv[n] = (live && n < D) ? to_f(cin[((size_t)b * D + n) * dim + el]) : 0.f;
+  const float pv = live ? pers[(size_t)b * dim + el] : 0.f;
+  float gcl = 0.f, ghl = 0.f;                        // lane n of warp 0 fetches node n's gates; thread 0 collects them by shuffle
+  if (threadIdx.x < D) { gcl = nd.g_csa[(size_t)b * D + threadIdx.x]; ghl = nd.g_hca[(size_t)b * D + threadIdx.x]; }
+  float pcm = 0.f, pcs = 0.f, phm = 0.f, phs = 0.f;
+  if (threadIdx.x == 0) { pcm = c.csa_mx[b]; pcs = c.csa_s[b]; phm = c.hca_mx[b]; phs = c.hca_s[b]; }
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  float gc[DMAX], gh[DMAX];
+  if (threadIdx.x < 32) {
+#pragma unroll
+    for (int n = 0; n < DMAX; ++n) { gc[n] = __shfl_sync(0xffffffffu, gcl, n); gh[n] = __shfl_sync(0xffffffffu, ghl, n); }
+  }
+
   if (threadIdx.x == 0) {
-    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], c.csa_cap + b, c.hca_cap + b);
-    if (tm.status) atomicOr(status + b, tm.status);
+    const bool writer = blockIdx.y == 0;
+    if (tm.status && writer) atomicOr(status + b, tm.status);
     const int nn = tm.status ? 0 : tm.nn;
-    float cmx[TSV_MAX_D], cs[TSV_MAX_D], hmx[TSV_MAX_D], hs[TSV_MAX_D];
-    for (int n = 0; n < D; ++n) {
-      float m1 = 0.f, s1 = 0.f, m2 = 0.f, s2 = 0.f;
-      if (n < nn) {
-        const int p = tm.L + tm.depth[n], par = tm.parent[n];
-        scalar_fold(fcs[n], m1, s1, p, s.m_csa, n ? cmx[par] : c.csa_mx[b], n ? cs[par] : c.csa_s[b], nd.g_csa[(size_t)b * D + n]);
-        scalar_fold(fhs[n], m2, s2, p, s.m_hca, n ? hmx[par] : c.hca_mx[b], n ? hs[par] : c.hca_s[b], nd.g_hca[(size_t)b * D + n]);
-      } else {
-        fcs[n].done = fhs[n].done = 0;
+#pragma unroll
+    for (int n = 0; n < DMAX; ++n) {
+      if (n < D) {
+        float m1 = 0.f, s1 = 0.f, m2 = 0.f, s2 = 0.f;
+        if (n < nn) {
+          const int p = tm.L + tm.depth[n], par = tm.parent[n];
+          float mp = pcm, sp = pcs, mq = phm, sq = phs;
+          if (n) { mp = cmx[par]; sp = cs[par]; mq = hmx[par]; sq = hs[par]; }
+          scalar_fold(fcs[n], m1, s1, p, s.m_csa, mp, sp, gc[n]);
+          scalar_fold(fhs[n], m2, s2, p, s.m_hca, mq, sq, gh[n]);
+        } else {
+          fcs[n].done = fhs[n].done = 0;
+        }
+        cmx[n] = m1; cs[n] = s1; hmx[n] = m2; hs[n] = s2;
+        if (writer) {
+          sc.csa_mx[(size_t)b * D + n] = m1; sc.csa_s[(size_t)b * D + n] = s1;
+          sc.hca_mx[(size_t)b * D + n] = m2; sc.hca_s[(size_t)b * D + n] = s2;
+          sc.csa_done[(size_t)b * D + n] = (uint8_t)fcs[n].done;
+          sc.hca_done[(size_t)b * D + n] = (uint8_t)fhs[n].done;
+        }
       }
-      cmx[n] = m1; cs[n] = s1; hmx[n] = m2; hs[n] = s2;
-      sc.csa_mx[(size_t)b * D + n] = m1; sc.csa_s[(size_t)b * D + n] = s1;
-      sc.hca_mx[(size_t)b * D + n] = m2; sc.hca_s[(size_t)b * D + n] = s2;
-      sc.csa_done[(size_t)b * D + n] = (uint8_t)fcs[n].done;
-      sc.hca_done[(size_t)b * D + n] = (uint8_t)fhs[n].done;
     }
   }
   __syncthreads();
+  if (!live) return;
   const int nn = tm.status ? 0 : tm.nn;
-  const int d = s.d, di = s.di;
-  // element index space: [0, d) CSA kv | [d, d+di) CSA indexer key | [d+di, 2d+di) HCA kv
-  for (int e = threadIdx.x; e < 2 * d + di; e += blockDim.x) {
-    const int which = e < d ? 0 : (e < d + di ? 1 : 2);
-    const int el = which == 0 ? e : (which == 1 ? e - d : e - d - di);
-    const int dim = which == 1 ? di : d;
-    const float* pers = which == 0 ? c.csa_acc_kv : (which == 1 ? c.csa_acc_ik : c.hca_acc_kv);
-    float* sacc = which == 0 ? sc.csa_acc_kv : (which == 1 ? sc.csa_acc_ik : sc.hca_acc_kv);
-    const T* cin = reinterpret_cast<const T*>(which == 0 ? nd.c_csa : (which == 1 ? nd.ikc : nd.c_hca));
-    T* newe = reinterpret_cast<T*>(which == 0 ? sc.new_csa_kv : (which == 1 ? sc.new_csa_ik : sc.new_hca_kv));
-    const FoldCoef* fc = which == 2 ? fhs : fcs;
-    for (int n = 0; n < D; ++n) {
+  float* sacc = which == 0 ? sc.csa_acc_kv : (which == 1 ? sc.csa_acc_ik : sc.hca_acc_kv);
+  T* newe = reinterpret_cast<T*>(which == 0 ? sc.new_csa_kv : (which == 1 ? sc.new_csa_ik : sc.new_hca_kv));
+  const FoldCoef* fc = which == 2 ? fhs : fcs;
+#pragma unroll
+  for (int n = 0; n < DMAX; ++n) {
+    if (n < D) {
       const size_t o = ((size_t)b * D + n) * dim + el;
-      if (n >= nn) { sacc[o] = 0.f; newe[o] = from_f<T>(0.f); continue; }
-      const FoldCoef f = fc[n];
-      const float cv = to_f(cin[o]);
-      float acc;
-      if (f.empty) acc = cv;
-      else {
-        const float ap = n ? sacc[((size_t)b * D + tm.parent[n]) * dim + el] : pers[(size_t)b * dim + el];
-        acc = fmaf(f.a, ap, f.b * cv);
+      float acc = 0.f, ent = 0.f;
+      if (n < nn) {
+        const FoldCoef f = fc[n];
+        if (f.empty) acc = cv[n];
+        else {
+          const float ap = n ? hist[tm.parent[n] * kBsbThreads + threadIdx.x] : pv;
+          acc = fmaf(f.a, ap, f.b * cv[n]);
+        }
+        if (f.done) { ent = acc / f.s; acc = 0.f; }
       }
-      if (f.done) { newe[o] = from_f<T>(acc / f.s); acc = 0.f; }
-      else newe[o] = from_f<T>(0.f);
+      hist[n * kBsbThreads + threadIdx.x] = acc;
       sacc[o] = acc;
+      newe[o] = from_f<T>(ent);
     }
   }
 }
 
 int launch_bsb(const tsv_shape& s, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, int32_t* status, cudaStream_t st) {
-  if (s.dtype == TSV_BF16) bsb_kernel<bf16><<<s.B, 128, 0, st>>>(s, c, nd, sc, status);
-  else bsb_kernel<float><<<s.B, 128, 0, st>>>(s, c, nd, sc, status);
+  const int elems = 2 * s.d + s.di;
+  const dim3 grid(s.B, (elems + kBsbThreads - 1) / kBsbThreads);
+  const size_t sm = (size_t)s.D * kBsbThreads * sizeof(float);
+  TSV_PREP((bsb_kernel<bf16, 8>));
+  TSV_PREP((bsb_kernel<float, 8>));
+  TSV_PREP((bsb_kernel<bf16, TSV_MAX_D>));
+  TSV_PREP((bsb_kernel<float, TSV_MAX_D>));
+  if (s.D <= 8) {
+    if (s.dtype == TSV_BF16) bsb_kernel<bf16, 8><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+    else bsb_kernel<float, 8><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+  } else {
+    if (s.dtype == TSV_BF16) bsb_kernel<bf16, TSV_MAX_D><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+    else bsb_kernel<float, TSV_MAX_D><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+  }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }

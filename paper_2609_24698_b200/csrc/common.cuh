@@ -88,6 +88,23 @@ __device__ inline void build_tree_meta(TreeMeta& tm, const tsv_shape& s, int32_t
   tm.n_csa = L / s.m_csa; tm.n_hca = L / s.m_hca;
 }
 
+// Cooperative front end of build_tree_meta: the first threads of the CTA fetch the parent array and the per-sequence
+// scalars in parallel (one memory latency instead of a chain of dependent loads), then thread 0 derives the tree facts.
+// Must be called by all threads of the CTA (contains two barriers); needs blockDim.x >= 64.
+struct TreeStage { int32_t parent[TSV_MAX_D]; int32_t scal[4]; };
+__device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, const tsv_shape& s, const int32_t* L_b, const int32_t* parent_b,
+                                               const int32_t* nn_b, const int32_t* csa_cap_b, const int32_t* hca_cap_b) {
+  const int t = threadIdx.x;
+  if (t < s.D) st.parent[t] = parent_b[t];
+  if (t == 32) st.scal[0] = *L_b;
+  if (t == 33) st.scal[1] = *nn_b;
+  if (t == 34 && csa_cap_b) st.scal[2] = *csa_cap_b;
+  if (t == 35 && hca_cap_b) st.scal[3] = *hca_cap_b;
+  __syncthreads();
+  if (t == 0) build_tree_meta(tm, s, st.scal[0], st.parent, st.scal[1], csa_cap_b ? &st.scal[2] : nullptr, hca_cap_b ? &st.scal[3] : nullptr);
+  __syncthreads();
+}
+
 __device__ __forceinline__ float softmax_scale(const tsv_shape& s) {
   return s.sm_scale > 0.f ? s.sm_scale : rsqrtf((float)s.d);
 }

@@ -4,7 +4,18 @@
 
 namespace tsv {
 
-void count_launch(int n = 1);   // bumps the reporting counter behind tsv_kernel_launches()
+void count_launch(int n = 1);
+
+// Every kernel of the library asks for the same (maximal) shared-memory carve-out: consecutive kernels with different
+// carve-outs make the SMs drain and reconfigure between launches, which costs far more than these kernels run.
+#define TSV_PREP(kernel)                                                                                          \
+  do {                                                                                                            \
+    static bool done_ = false;                                                                                    \
+    if (!done_) {                                                                                                 \
+      cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared); \
+      done_ = true;                                                                                               \
+    }                                                                                                             \
+  } while (0)   // bumps the reporting counter behind tsv_kernel_launches()
 
 // Per-layer pointers accept_and_refresh needs, packed so that a group of layers fits in
 // kernel-parameter space.
@@ -43,6 +54,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
 
+constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs are padded to a multiple of it
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
 bool tva_tc_tma_usable(const tsv_cache& c);

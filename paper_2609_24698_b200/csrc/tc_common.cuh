@@ -17,7 +17,7 @@ constexpr int THREADS = 256;
 constexpr int kHcaMiscMaxTc = 32;
 constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
 constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 20;   // polls before a wait gives up (then no later wait of the thread is attempted)
+constexpr uint32_t WAIT_LIMIT = 1u << 16;   // polls before a wait gives up (then no later wait of the thread is attempted)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

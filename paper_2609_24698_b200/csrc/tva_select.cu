@@ -35,11 +35,16 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
                                                         const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ float iq_s[];                 // [<=32 (node, head) pairs][di]
   __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
   __shared__ int need_any;
   __shared__ uint32_t need_mask;
   const int b = blockIdx.y, D = s.D, di = s.di, HI = s.HI;
+  {   // cheap exit: even with every ancestor closing a block, no node of this sequence has more than topk candidates
+    const int L0 = c.L[b];
+    if (L0 < 0 || L0 / s.m_csa + D <= s.topk || (int)(blockIdx.x * blockDim.x) >= L0 / s.m_csa) return;
+  }
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, nullptr, nullptr);
   if (threadIdx.x == 0) {
-    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], nullptr, nullptr);
     uint32_t m = 0;
     if (!tm.status)
       for (int n = 0; n < tm.nn; ++n) {
@@ -57,9 +62,10 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
   const T* ikrow = reinterpret_cast<const T*>(c.csa_ik) + ((size_t)c.csa_row0[b] + (live ? e : 0)) * di;
   float* scores = reinterpret_cast<float*>(ws + pl.off_scores) + (size_t)b * D * pl.cand_cap;
   constexpr int V = Vec<T>::N;
-  const int npg = 32 / HI;                        // nodes per group
-  for (int n0 = 0; n0 < tm.nn; n0 += npg) {
-    const int gn = min(npg, tm.nn - n0), G = gn * HI;
+  const int npg = min(32 / HI, (D + (int)gridDim.z - 1) / (int)gridDim.z);   // nodes per group; blockIdx.z owns a slab of nodes
+  const int nz0 = blockIdx.z * ((D + (int)gridDim.z - 1) / (int)gridDim.z), nz1 = min(tm.nn, nz0 + (D + (int)gridDim.z - 1) / (int)gridDim.z);
+  for (int n0 = nz0; n0 < nz1; n0 += npg) {
+    const int gn = min(npg, nz1 - n0), G = gn * HI;
     __syncthreads();
     for (int i = threadIdx.x; i < G * di; i += blockDim.x)
       iq_s[i] = to_f(reinterpret_cast<const T*>(nd.iq)[((size_t)b * D + n0) * HI * di + i]);
@@ -103,6 +109,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
                                                    int32_t* __restrict__ status) {
   __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
   __shared__ PathEntries pe;
   __shared__ float extra[TSV_MAX_D];
   __shared__ int hist[256];
@@ -113,8 +120,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
   if (threadIdx.x == 0) {
-    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], c.csa_cap + b, c.hca_cap + b);
     if (tm.status && n == 0) atomicOr(status + b, tm.status);
     if (!tm.status && n < tm.nn) path_entries(pe, tm, s, n, sc.csa_done + (size_t)b * D, sc.hca_done + (size_t)b * D);
   }
@@ -164,14 +171,22 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int rem = sh_remaining, cum = 0, bin = 255;
-      for (; bin > 0; --bin) {
-        if (cum + hist[bin] >= rem) break;
-        cum += hist[bin];
+    if (threadIdx.x < 32) {                           // warp 0 finds the bin holding the rem-th largest key: lane l owns bins 255-8l .. 248-8l
+      const int lane = threadIdx.x, rem = sh_remaining;
+      int h[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { h[j] = hist[255 - (lane * 8 + j)]; tot += h[j]; }
+      int incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+      const int excl = incl - tot;
+      if (excl < rem && incl >= rem) {
+        int cum = excl, bin = 255 - lane * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { if (cum + h[j] >= rem) { bin = 255 - (lane * 8 + j); break; } cum += h[j]; }
+        sh_prefix = prefix | ((uint32_t)bin << shift);
+        sh_remaining = rem - cum;
       }
-      sh_prefix = prefix | ((uint32_t)bin << shift);
-      sh_remaining = rem - cum;
     }
     mask |= 0xFFu << shift;
     __syncthreads();
@@ -202,20 +217,24 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   const bool bf = s.dtype == TSV_BF16;
   if (p.need_scores) {
     const int pref_cap = (int)(s.max_L / s.m_csa);
-    dim3 grid((pref_cap + 255) / 256, s.B);
+    dim3 grid((pref_cap + 255) / 256, s.B, s.D <= 8 ? s.D : 8);        // z: slabs of nodes, so a ranked sequence is scored by many CTAs
     const size_t sm = (size_t)32 * s.di * sizeof(float);
     if (grid.x > 0) {
       if (bf) {
         cudaFuncSetAttribute(idx_score_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        TSV_PREP(idx_score_kernel<bf16>);
         idx_score_kernel<bf16><<<grid, 256, sm, st>>>(s, p, c, nd, sc, ws);
       } else {
         cudaFuncSetAttribute(idx_score_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        TSV_PREP(idx_score_kernel<float>);
         idx_score_kernel<float><<<grid, 256, sm, st>>>(s, p, c, nd, sc, ws);
       }
       count_launch();
     }
   }
   dim3 g2(s.D, s.B);
+  TSV_PREP(topk_kernel<bf16>);
+  TSV_PREP(topk_kernel<float>);
   if (bf) topk_kernel<bf16><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
   else topk_kernel<float><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
   count_launch();

@@ -258,6 +258,8 @@ static int launch_one(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   const size_t sm = ((size_t)kHeadsPerCta * s.d + (size_t)kKeyTile * (s.d + V)) * sizeof(T) + kHeadsPerCta * kKeyTile * sizeof(float);
   if (cudaFuncSetAttribute(attn_simt_kernel<T, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) != cudaSuccess) return TSV_ERR_CUDA;
   dim3 grid(p.nsplit, s.D * hgroups, s.B);
+  TSV_PREP((attn_simt_kernel<T, NCH>));
+  TSV_PREP(attn_combine_kernel<T>);
   attn_simt_kernel<T, NCH><<<grid, 256, sm, st>>>(s, p, c, nd, sc, out, ws);
   count_launch();
   if (p.nsplit > 1) { attn_combine_kernel<T><<<dim3(s.D, s.B), 256, 0, st>>>(s, p, c, nd, sc, out, ws); count_launch(); }

@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask[];                   // [cand_cap] node bits per committed CSA entry (ranked case only)
   __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
   __shared__ int wsum[9];
   __shared__ int n_cand[8], win_lo[8];
   __shared__ int dense;
@@ -43,8 +44,8 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   const int32_t* sel = reinterpret_cast<const int32_t*>(ws + pl.off_sel) + (size_t)b * D * s.topk;
   const uint8_t* cdone = sc.csa_done + (size_t)b * D;
   const uint8_t* hdone = sc.hca_done + (size_t)b * D;
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
   if (threadIdx.x == 0) {
-    build_tree_meta(tm, s, c.L[b], nd.parent + (size_t)b * D, nd.n_nodes[b], c.csa_cap + b, c.hca_cap + b);
     int dn = 1;
     for (int nl = 0; nl < npt; ++nl) {
       const int n = n0 + nl;
@@ -64,6 +65,25 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   const uint32_t validbits = (1u << nvalid) - 1u;
   const int n_csa = tm.n_csa;
   const size_t rowb = (size_t)s.d * 2;
+  if (!dense) {
+    for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] = 0;
+    __syncthreads();
+    for (int nl = 0; nl < nvalid; ++nl) {
+      const int n = n0 + nl, cnt = selcnt[n];
+      if (n_cand[nl] <= s.topk) { for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)(1u << nl); }
+      else for (int j = threadIdx.x; j < cnt; j += blockDim.x) { const int idx = sel[(size_t)n * s.topk + j]; if (idx < n_csa) cmask[idx] |= (uint8_t)(1u << nl); }
+      __syncthreads();
+    }
+  }
+  // is the entry closed at node a (a strict ancestor of node n0 + nl) among that node's selected CSA entries?
+  auto newc_selected = [&](int nl, int a) {
+    if (n_cand[nl] <= s.topk) return true;
+    const int n = n0 + nl, blk = (tm.L + tm.depth[a]) / s.m_csa, cnt = selcnt[n];
+    const int32_t* sl = sel + (size_t)n * s.topk;
+    int lo_ = 0, hi_ = cnt - 1;
+    while (lo_ <= hi_) { const int mid = (lo_ + hi_) >> 1; const int v = sl[mid]; if (v == blk) return true; if (v < blk) lo_ = mid + 1; else hi_ = mid - 1; }
+    return false;
+  };
   if (pl.tc_tma) {
     // rows that are small and scattered (few HCA entries, tree nodes, entries closed inside the tree) are packed
     // into one contiguous per-sequence buffer so that TMA boxes can fetch them: written by the CTA of tile 0
@@ -73,7 +93,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     if (tile == 0) {
       uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
-      const int rows_out = (n_misc + 31) / 32 * 32, cpr = (int)(rowb / 16);
+      const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows, cpr = (int)(rowb / 16);
       for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
         const int r = i / cpr, cc = i % cpr;
         const char* src = nullptr;
@@ -91,16 +111,19 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
         dst[i] = src ? reinterpret_cast<const uint4*>(src)[cc] : make_uint4(0, 0, 0, 0);
       }
     }
-    if (dense) {
-      int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / 32);
+    // Ranked nodes still take the contiguous-run path while the run is at most twice the selection size: all committed
+    // entries are staged and the unselected ones are masked per node.
+    if (dense || n_csa <= 2 * s.topk) {
+      int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
       int kb = 0;
       auto emit = [&](int map, int64_t start, int count, int seg) {
-        const int nb = (count + 31) / 32;
-        for (int i = threadIdx.x; i < nb; i += blockDim.x) box[kb / 32 + i] = make_int2(map, (int)(start + 32 * i));
-        for (int i = threadIdx.x; i < nb * 32; i += blockDim.x) {
+        const int nb = (count + kBoxRows - 1) / kBoxRows;
+        for (int i = threadIdx.x; i < nb; i += blockDim.x) box[kb / kBoxRows + i] = make_int2(map, (int)(start + kBoxRows * i));
+        for (int i = threadIdx.x; i < nb * kBoxRows; i += blockDim.x) {
           uint32_t m = 0;
           if (i < count) {
-            if (seg == 0 || seg == 1) m = validbits;
+            if (seg == 0) m = dense ? validbits : cmask[i];
+            else if (seg == 1) m = validbits;
             else if (seg == 2) {
               const int pos = tm.L - 1 - ((tm.L - 1 - i) % s.window);
               for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
@@ -115,12 +138,13 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
               const uint8_t* dn = isc ? cdone : hdone;
               int a = 0;
               for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
-              for (int nl = 0; nl < nvalid; ++nl) if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u)) m |= 1u << nl;
+              for (int nl = 0; nl < nvalid; ++nl)
+                if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && (!isc || newc_selected(nl, a))) m |= 1u << nl;
             }
           }
           kmask[kb + i] = (uint8_t)m;
         }
-        kb += nb * 32;
+        kb += nb * kBoxRows;
       };
       emit(0, c.csa_row0[b], n_csa, 0);
       if (tm.n_hca > kHcaMiscMax) emit(1, c.hca_row0[b], tm.n_hca, 1);
@@ -131,16 +155,6 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
     }
   }
   if (threadIdx.x == 0) *mode = 0;
-  if (!dense) {
-    for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] = 0;
-    __syncthreads();
-    for (int nl = 0; nl < nvalid; ++nl) {
-      const int n = n0 + nl, cnt = selcnt[n];
-      if (n_cand[nl] <= s.topk) { for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)(1u << nl); }
-      else for (int j = threadIdx.x; j < cnt; j += blockDim.x) { const int idx = sel[(size_t)n * s.topk + j]; if (idx < n_csa) cmask[idx] |= (uint8_t)(1u << nl); }
-      __syncthreads();
-    }
-  }
   // committed CSA entries, in index order
   int base = 0;
   for (int i0 = 0; i0 < n_csa; i0 += blockDim.x) {
@@ -538,8 +552,9 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   int64_t uni = (int64_t)npt * ksel;
   if (uni > p.cand_cap) uni = p.cand_cap;
   int64_t mk = uni + s.max_L / s.m_hca + s.window + 3 * (int64_t)s.D + 8;
-  p.tc_misc_rows = (kHcaMiscMax + 3 * s.D + 31) / 32 * 32;
-  const int64_t runs = (p.cand_cap + 31) / 32 * 32 + (s.max_L / s.m_hca + 31) / 32 * 32 + (s.window + 31) / 32 * 32 + p.tc_misc_rows;
+  const int64_t br = kBoxRows;
+  p.tc_misc_rows = (int32_t)((kHcaMiscMax + 3 * s.D + br - 1) / br * br);
+  const int64_t runs = (p.cand_cap + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + p.tc_misc_rows;
   if (runs > mk) mk = runs;
   p.tc_maxk = (int32_t)((mk + 127) / 128 * 128);
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
@@ -552,6 +567,9 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
   const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
   if (plan_sm > 48 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
     return TSV_ERR_CUDA;
+  TSV_PREP(tc_plan_kernel);
+  TSV_PREP(tc_attn_kernel);
+  TSV_PREP(tc_combine_kernel);
   tc_plan_kernel<<<dim3(p.tc_nt, s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);
   count_launch();
   if (p.tc_tma) {
