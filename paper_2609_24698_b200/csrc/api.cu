@@ -65,8 +65,8 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
     p.off_kptr = off;  off = up256(off + tiles * p.tc_maxk * sizeof(uint64_t));
     p.off_kmask = off; off = up256(off + tiles * p.tc_maxk);
     p.off_nkeys = off; off = up256(off + tiles * sizeof(int32_t));
-    p.off_tpo = off;   if (p.tc_chmax > 1) off = up256(off + tiles * p.tc_chmax * 128 * s.d * sizeof(float));
-    p.off_tpml = off;  if (p.tc_chmax > 1) off = up256(off + tiles * p.tc_chmax * 128 * 2 * sizeof(float));
+    p.off_tpo = off;   if (p.tc_chmax > 1) off = up256(off + 2 * tiles * p.tc_chmax * 128 * s.d * sizeof(float));
+    p.off_tpml = off;  if (p.tc_chmax > 1) off = up256(off + 2 * tiles * p.tc_chmax * 128 * 2 * sizeof(float));
     p.off_box = off;   off = up256(off + tiles * (p.tc_maxk / 32) * 2 * sizeof(int32_t));
     p.off_mode = off;  off = up256(off + tiles * sizeof(int32_t));
     p.off_misc = off;  off = up256(off + (size_t)s.B * p.tc_misc_rows * s.d * 2);

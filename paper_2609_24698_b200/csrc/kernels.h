@@ -57,8 +57,8 @@ int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, co
 constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs are padded to a multiple of it
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
-bool tva_tc_tma_usable(const tsv_cache& c);
-int launch_tva_tc_tma(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
+bool tva_tc_pair_usable(const tsv_cache& c);
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
                       int32_t* status, cudaStream_t st);
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,

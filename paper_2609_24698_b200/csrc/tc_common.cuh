@@ -8,7 +8,8 @@ namespace tsv {
 namespace tc {
 
 constexpr int DH = 512;             // head dim handled by this path
-constexpr int BM = 128;             // rows per tile
+constexpr int BM = 128;             // rows per CTA
+constexpr int PR = 256;             // rows per plan tile: two row tiles (one CTA pair) share one key list
 constexpr int NC = 512;             // max keys per chunk (S columns in TMEM)
 constexpr int SLOT = 32768;
 constexpr int NS = 7;               // ring slots
@@ -17,7 +18,7 @@ constexpr int THREADS = 256;
 constexpr int kHcaMiscMaxTc = 32;
 constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
 constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 16;   // polls before a wait gives up (then no later wait of the thread is attempted)
+constexpr uint32_t WAIT_LIMIT = 1u << 14;   // polls before a wait gives up (then no later wait of the thread is attempted)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -44,13 +45,16 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Bounded wait on an mbarrier phase; false if the limit ran out.
+// Bounded wait on an mbarrier phase; false if the limit ran out.  Each try suspends the warp in hardware for up to
+// SUSPEND_NS (it wakes as soon as the phase completes), so waiting warps do not compete for issue slots or for the
+// shared-memory pipe with the warps that feed the tensor core.
+constexpr uint32_t SUSPEND_NS = 4000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   const uint32_t a = smem_u32(bar);
   for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity), "r"(SUSPEND_NS) : "memory");
     if (ok) return true;
   }
   return false;

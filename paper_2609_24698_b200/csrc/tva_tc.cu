@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   __shared__ int n_cand[8], win_lo[8];
   __shared__ int dense;
   const int tile = blockIdx.x, b = blockIdx.y, D = s.D, H = s.H;
-  const int npt = tc::BM / H, n0 = tile * npt;
+  const int npt = tc::PR / H, n0 = tile * npt;
   const size_t tix = (size_t)b * pl.tc_nt + tile;
   uint64_t* kptr = reinterpret_cast<uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
@@ -248,14 +248,16 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
                                                                  char* __restrict__ ws, int32_t* __restrict__ status) {
   using namespace tc;
   extern __shared__ unsigned char smem_raw[];
-  const int chunk = blockIdx.x, tile = blockIdx.y, b = blockIdx.z;
+  const int chunk = blockIdx.x, rt = blockIdx.y, tile = rt >> 1, b = blockIdx.z;     // rt: 128-row tile; tile: its plan tile
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int D = s.D, H = s.H;
   const size_t tix = (size_t)b * pl.tc_nt + tile;
+  const size_t rix = (size_t)b * 2 * pl.tc_nt + rt;
   if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 0) return;      // a contiguous-run tile: the TMA kernel's
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   const int rows_seq = D * H;
-  const int row0 = tile * BM;                                   // first row of the tile within the sequence
+  if (rt * BM >= rows_seq) return;                              // second half of a plan tile that ends before it
+  const int row0 = rt * BM;                                     // first row of the CTA's tile within the sequence
   bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
   if (nk <= 0) {                                                // flagged sequence or padding-only tile: zeros
     if (chunk == 0)
@@ -346,7 +348,7 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
   const int q4 = warp & 3, hh = warp >> 2;          // TMEM lane quarter of this warp; column half it works on
   const int row = q4 * 32 + lane;
   const uint32_t tlane = tm + ((uint32_t)(q4 * 32) << 16);
-  const uint32_t mybit = 1u << (row / H);
+  const uint32_t mybit = 1u << ((rt & 1) * (BM / H) + row / H);
   const float scale2 = s.sm_scale * 1.4426950408889634f;
   float m_row = 0.f, l_row = 0.f;
   uint32_t acc_parity = 0;
@@ -375,7 +377,7 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
         }
       }
     } else {
-      float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((tix * pl.tc_chmax + chunk) * BM + row) * DH + half * 256 + hh * 128;
+      float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((rix * pl.tc_chmax + chunk) * BM + row) * DH + half * 256 + hh * 128;
 #pragma unroll
       for (int c0 = 0; c0 < 128; c0 += 32) {
         uint32_t r[32];
@@ -386,7 +388,7 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
                                                                     __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
       }
       if (half == 0 && hh == 0)
-        reinterpret_cast<float2*>(ws + pl.off_tpml)[(tix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_row, l_row);
+        reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_row, l_row);
     }
     fence_before();
     __syncthreads();                                 // O columns may be overwritten by the next half
@@ -508,16 +510,16 @@ __global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape
 // ------------------------------------------------------------------------------------------------ combine
 __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, const TvaPlan pl, void* __restrict__ out_, const char* __restrict__ ws) {
   using namespace tc;
-  const int tile = blockIdx.x, b = blockIdx.y;
-  const size_t tix = (size_t)b * pl.tc_nt + tile;
+  const int rt = blockIdx.x, tile = rt >> 1, b = blockIdx.y;
+  const size_t tix = (size_t)b * pl.tc_nt + tile, rix = (size_t)b * 2 * pl.tc_nt + rt;
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   int nch, CL;
   if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] == 1) chunking_x(nk, nch, CL); else chunking(nk, nch, CL);
   if (nk <= 0 || nch <= 1) return;
-  const int rows_seq = s.D * s.H, row0 = tile * BM;
+  const int rows_seq = s.D * s.H, row0 = rt * BM;
   bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
-  const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + tix * pl.tc_chmax * BM * DH;
-  const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + tix * pl.tc_chmax * BM;
+  const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + rix * pl.tc_chmax * BM * DH;
+  const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM;
   for (int i = threadIdx.x; i < BM * DH / 8; i += blockDim.x) {
     const int row = i / (DH / 8), c8 = i % (DH / 8);
     if (row0 + row >= rows_seq) continue;
@@ -542,12 +544,12 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
 }
 
 bool tva_tc_eligible(const tsv_shape& s) {
-  return s.dtype == TSV_BF16 && s.d == tc::DH && s.H >= 16 && s.H <= 128 && (128 % s.H) == 0 && !(s.flags & TSV_FLAG_FORCE_SIMT);
+  return s.dtype == TSV_BF16 && s.d == tc::DH && s.H >= 32 && s.H <= 128 && (128 % s.H) == 0 && !(s.flags & TSV_FLAG_FORCE_SIMT);
 }
 
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
-  const int npt = tc::BM / s.H;
-  p.tc_nt = (s.D * s.H + tc::BM - 1) / tc::BM;
+  const int npt = tc::PR / s.H;
+  p.tc_nt = (s.D * s.H + tc::PR - 1) / tc::PR;
   const int64_t ksel = p.cand_cap < s.topk ? p.cand_cap : s.topk;
   int64_t uni = (int64_t)npt * ksel;
   if (uni > p.cand_cap) uni = p.cand_cap;
@@ -563,7 +565,7 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
   TvaPlan p = p_in;
-  p.tc_tma = tva_tc_tma_usable(c) ? 1 : 0;
+  p.tc_tma = tva_tc_pair_usable(c) ? 1 : 0;
   const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
   if (plan_sm > 48 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
     return TSV_ERR_CUDA;
@@ -573,16 +575,16 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
   tc_plan_kernel<<<dim3(p.tc_nt, s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);
   count_launch();
   if (p.tc_tma) {
-    const int r = launch_tva_tc_tma(s, p, c, nd, out, ws, status, st);
+    const int r = launch_tva_tc_pair(s, p, c, nd, out, ws, status, st);
     if (r != TSV_OK) return r;
   }
   if (!p.tc_tma || p.need_scores) {            // tiles with ranked selections (or no TMA): pointer-gather kernel
     if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
-    tc_attn_kernel<<<dim3(p.tc_chmax, p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
+    tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
   }
   if (p.tc_chmax > 1) {
-    tc_combine_kernel<<<dim3(p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
+    tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
     count_launch();
   }
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;

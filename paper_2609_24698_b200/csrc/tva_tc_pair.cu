@@ -1,34 +1,39 @@
-// tree_verify_attn, tensor-core kernel for tiles whose key rows form contiguous runs
-// (every node of the tile selects all of its CSA candidates: the common short-prefix case).
+// tree_verify_attn, tensor-core kernel for key lists made of contiguous runs, run by PAIRS of CTAs
+// (thread-block cluster of 2, tcgen05 cta_group::2).
 //
-// Same math and the same stage stream as tc_attn_kernel (Q slice | K tiles per 64-wide slice of d,
-// then 64-key V stages per half of d), but operands arrive by TMA (cp.async.bulk.tensor, 128-byte
-// swizzle, boxes of 32 rows x 64 dims) and the CTA is warp-specialised:
-//   warp 0     producer: waits for a free ring slot, arms its mbarrier with the byte count and
-//              issues the box copies of the stage (one elected lane)
-//   warp 1     MMA issuer: waits for the slot to fill, issues tcgen05.mma, releases the slot
-//              with tcgen05.commit (one elected lane)
-//   warps 2-9  softmax on S read from TMEM, P written back to TMEM, epilogue of O
-// The key list of a tile is a list of boxes {tensor map, first row}; runs are padded to 32 rows
-// and the padding rows carry a zero node mask.  No block-wide barrier inside the main loop.
+// A pair covers 256 query rows of one sequence (256/H consecutive tree nodes x H heads); each CTA owns
+// 128 of them in its own tensor memory.  The two SMs execute every MMA together (M = 256): the B operand
+// -- the staged key rows -- is split between the two shared memories, so each SM fetches only HALF of
+// the K tile (S = Q K^T: half of the keys) and half of the V tile (O = P K: half of the columns of d).
+// That halves the bytes each SM pulls from L2, which is what bounds this kernel.
+//   warp 0     producer: TMA boxes (cp.async.bulk.tensor, 128-byte swizzle) into a ring of 16 KiB slots; the
+//              copies of BOTH CTAs complete on the mbarrier of the leader (rank 0) CTA
+//   warp 1     MMA issuer (leader CTA only): tcgen05.mma.cta_group::2, slot release and accumulator
+//              events by tcgen05.commit multicast to both CTAs
+//   warps 2-9  softmax on the CTA's own S rows (TMEM), P written back to TMEM, epilogue of O through
+//              swizzled shared-memory tiles and TMA stores; events to the leader's MMA warp by remote arrive
+// Stage stream, TMEM column plan, running-max rule and chunking are those described at the kernel.
 #include <cuda.h>
+#include <stdio.h>
 #include <cudaTypedefs.h>
 
 #include "tc_common.cuh"
 
 namespace tsv {
 
-namespace tma {
+namespace pair {
 
 using namespace tc;
 
-constexpr int TTHREADS = 320;
+constexpr int TTHREADS = 352;               // warps 0 and 10: producers (even / odd stages); 1: MMA issuer; 2-9: softmax and epilogue
 constexpr int BOXB = kBoxRows * 128;       // bytes of one box: kBoxRows rows x 128 bytes
 constexpr float RESCALE_GAP = 16.f;        // log2 units a later piece's row max may exceed the running reference
 
+constexpr int NSX = 12;                    // ring slots; a 32 KiB area after the ring stages the output tiles
+
 struct Ctl {                               // control block at the start of dynamic shared memory
-  uint64_t full[NS];
-  uint64_t empty[NS];
+  uint64_t full[NSX];
+  uint64_t empty[NSX];
   uint64_t acc_ev[7];                      // MMA -> compute warps, one barrier per event, each used once:
                                            //   [pc] S of piece pc is complete   [3 + p] part p of O is complete
   uint64_t cmp_ev[6];                      // compute warps -> MMA, one barrier per event, each used once:
@@ -40,45 +45,86 @@ struct Ctl {                               // control block at the start of dyna
   float xch[2][BM];
 };
 constexpr int CTLB = 3072;                 // control block bytes; the ring follows (needs a 1024-byte aligned base)
-constexpr int NSX = 6;                     // ring slots of this kernel; the seventh 32 KiB area stages the output tiles
-constexpr int SMEM_X = CTLB + (NSX + 1) * SLOT;
+constexpr int SLOTP = 16384;               // ring slot: every stage of a CTA is at most 16 KiB
+constexpr int SMEM_X = CTLB + NSX * SLOTP + 32768;
 static_assert(sizeof(Ctl) <= CTLB, "control block overflow");
 
 __device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
-}
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+// shared::cluster address of the same variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA box copy into this CTA's shared memory; completion is counted on an mbarrier given by its cluster address
+__device__ __forceinline__ void tma_box2(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// arrives on the same barrier (same shared-memory offset) in both CTAs of the pair once all prior MMAs have completed:
+// one commit per destination CTA, each addressed through its cluster address
+__device__ __forceinline__ void mma2_commit(uint64_t* bar) {
+  const uint32_t a = smem_u32(bar);
+#pragma unroll
+  for (uint32_t r = 0; r < 2; ++r)
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_rank(a, r)) : "memory");
+}
+__device__ __forceinline__ uint32_t make_idesc2(int N, int b_mn_major) {      // M = 256 over the pair
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
+// Tensor maps of one call: every source array with boxes of 32, 64 and 128 rows (64 columns, 128-byte swizzle), so that
+// a stage whose key rows are consecutive rows of one array is fetched by ONE large request.
+struct alignas(64) MapSet {
+  CUtensorMap q;          // 128-row boxes
+  CUtensorMap out;        // 32-row boxes (stores)
+  CUtensorMap src[4][3];  // [csa, hca, window, packed misc][32, 64, 128 rows]
+};
+
 constexpr uint32_t OOB_BOX = 0x3FFFFF00u;   // map 0, a row beyond every tensor: the box is zero-filled
 
-}  // namespace tma
+}  // namespace pair
 
-// Stage stream of one chunk (CL keys, pieces of 256 keys, the last one may hold 128):
-//   for piece: for dk in 0..7:  [Q slice dk: 128 rows x 64]  [K: piece keys x 64 dims of slice dk]     (S piece += Q K^T)
-//   for quarter of d in 0..3: for kb in 0..CL/128-1:  [V: 128 keys x 128 dims]                         (O quarter += P V)
-__global__ void __launch_bounds__(tma::TTHREADS, 1)
-tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_csa,
-                   const __grid_constant__ CUtensorMap map_hca, const __grid_constant__ CUtensorMap map_win,
-                   const __grid_constant__ CUtensorMap map_misc, const __grid_constant__ CUtensorMap map_out, const tsv_shape s, const TvaPlan pl, void* __restrict__ out_,
-                   char* __restrict__ ws, int32_t* __restrict__ status) {
-  using namespace tma;
+// Per CTA (rank r of the pair), for a chunk of CL keys (pieces of 256 keys, the last may hold 128):
+//   S stages: pass A = pieces 0 and 1, pass B = piece 2; per pass and 64-wide slice dk of d:
+//       [Q: this CTA's 128 rows x 64 dims]  then per piece  [K: this CTA's half of the piece's keys x 64 dims]
+//   V stages: CL <= 512: per half of d, per 64 keys:  [64 keys x this CTA's 128 of the half's 256 dims]
+//             else       per quarter of d, per 128 keys: [128 keys x this CTA's 64 of the quarter's 128 dims]
+__global__ void __launch_bounds__(pair::TTHREADS, 1)
+tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s,
+                    const TvaPlan pl, void* __restrict__ out_, char* __restrict__ ws, int32_t* __restrict__ status) {
+  using namespace pair;
   extern __shared__ unsigned char smem_raw[];
-  const int chunk = blockIdx.x, tile = blockIdx.y, b = blockIdx.z;
+  const int chunk = blockIdx.y, tile = blockIdx.x >> 1, b = blockIdx.z;       // the two CTAs of a pair are neighbours in x
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const size_t tix = (size_t)b * pl.tc_nt + tile;
+  const size_t rix = (size_t)b * 2 * pl.tc_nt + blockIdx.x;      // this CTA's 128-row tile (partials of multi-chunk tiles)
+  // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
   if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 1) return;      // not a contiguous-run tile
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
-  const int rows_seq = s.D * s.H, row0 = tile * BM;
+  const int rows_seq = s.D * s.H, row0 = tile * PR + (int)rank * BM;           // first of this CTA's rows within the sequence
   if (nk <= 0) {                                               // flagged sequence or padding-only tile: zeros
     if (chunk == 0) {
       uint4* o4 = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH);
@@ -92,22 +138,19 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   if (chunk >= nch) return;
   const int cbeg = chunk * CL, cend = min(nk, cbeg + CL);
 
-  if (smem_u32(smem_raw) & 1023u) {                            // the swizzled tiles need a 1024-byte aligned base
-    if (tid == 0) atomicOr(status + b, TSV_ST_INTERNAL);
-    return;
-  }
   Ctl& sm = *reinterpret_cast<Ctl*>(smem_raw);
   const uint32_t ring = smem_u32(smem_raw + CTLB);
+  int fail = (smem_u32(smem_raw) & 1023u) ? 1 : 0;             // the swizzled tiles need a 1024-byte aligned base
 
   if (tid == 0) {
     for (int i = 0; i < NSX; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
     for (int i = 0; i < 7; ++i) mbar_init(&sm.acc_ev[i], 1);
-    for (int i = 0; i < 6; ++i) mbar_init(&sm.cmp_ev[i], 8);
+    for (int i = 0; i < 6; ++i) mbar_init(&sm.cmp_ev[i], 16);   // 8 compute warps of each CTA
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   {
     const int2* box_g = reinterpret_cast<const int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
@@ -121,28 +164,26 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   }
   fence_before();
   __syncthreads();
+  cluster_sync_all();                                            // barriers of both CTAs exist before anyone signals them
   fence_after();
   const uint32_t tm = sm.tmem_base;
 
-  // TMEM columns.  S piece 0 -> [0,256), pieces 1 and 2 -> [256,512) (fp32); P piece pc (bf16 pairs) -> [128 pc, 128 pc + 128).
-  // CL <= 512: two pieces at most, O is computed in two halves of 256 columns at [256,512) (N = 256);
-  // CL <= 768: three pieces, O in four quarters of 128 columns at [384,512) (N = 128).
+  // TMEM columns (per CTA, its own 128 rows).  S piece 0 -> [0,256), pieces 1 and 2 -> [256,512) (fp32);
+  // P piece pc (bf16 pairs) -> [128 pc, 128 pc + 128).  CL <= 512: O in two halves of 256 columns at [256,512);
+  // CL <= 768: O in four quarters of 128 columns at [384,512).
   const int npc = (CL + 255) / 256;                 // S pieces
   const int NQ = CL <= 512 ? 2 : 4;                 // parts of d the PV product is computed in
   const int OW = DH / NQ;                           // columns of one part
   const uint32_t OCOL = 512 - OW;
-  const int vkeys = 16384 / OW;                     // keys per V stage (32 KiB slot): 64 or 128
-  // S stages: pass A covers pieces 0 and 1 (their S columns coexist), pass B piece 2; per pass and 64-wide slice dk of d:
-  // one Q stage followed by one K stage per piece of the pass
+  const int vkeys = 16384 / OW;                     // keys per V stage: 64 or 128
   const int npA = npc < 2 ? npc : 2, perA = 1 + npA;
   const int GA = 8 * perA;
   const int G1 = GA + (npc > 2 ? 16 : 0);
   const int nvb = CL / vkeys;                       // V stages per part
   const int GT = G1 + NQ * nvb;
-  int fail = 0;
 #ifdef TSV_TIMELINE
-  long long* tl = reinterpret_cast<long long*>(ws);
-  const bool tlon = (blockIdx.x == 0 && blockIdx.y == 1 && blockIdx.z == 0);
+  long long* tl = reinterpret_cast<long long*>(ws) + (rank ? 400 : 0);
+  const bool tlon = (blockIdx.x < 2 && blockIdx.y == 0 && blockIdx.z == 0);
 #define TL(i) do { if (tlon) tl[i] = clock64(); } while (0)
   if (tlon && tid == 0) { tl[0] = clock64(); tl[1] = CL; tl[2] = GT; }
 #else
@@ -155,54 +196,75 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     else { const int h = g - GA; dk = h >> 1; r = h & 1; pc = 2; gq = GA + 2 * dk; lastk = r == 1; }
   };
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer (lane 0 arms the barrier, lanes 0..7 each copy one box)
-    const CUtensorMap* maps[4] = {&map_csa, &map_hca, &map_win, &map_misc};
-    for (int g = 0; g < GT; ++g) {
+  if (warp == 0 || warp == 10) {
+    // ------------------------------------------------------------------ producers (both CTAs): warp 0 takes the even stages, warp 10 the odd ones
+    const int pw = warp == 0 ? 0 : 1;
+    // consecutive: do the nb boxes starting at list index i0 name consecutive rows of one array?
+    auto consecutive = [&](int i0, int nb) {
+      const uint32_t b0 = sm.box[i0];
+      if ((b0 & 0x3FFFFFFFu) >= (OOB_BOX & 0x3FFFFFFFu)) return false;
+      for (int i = 1; i < nb; ++i) if (sm.box[i0 + i] != b0 + (uint32_t)(i * kBoxRows)) return false;
+      return true;
+    };
+    for (int g = pw; g < GT; g += 2) {
       const int sl = g % NSX, use = g / NSX;
-      const uint32_t slot = ring + (uint32_t)sl * SLOT;
-      uint64_t* fb = &sm.full[sl];
-      int nbox;
+      const uint32_t slot = ring + (uint32_t)sl * SLOTP;
+      const uint32_t fb_leader = map_to_rank(smem_u32(&sm.full[sl]), 0);     // both CTAs' copies complete on the leader's barrier
       int dk = 0, r = 0, pc = 0, gq = 0; bool lastk = false;
-      if (g < G1) { dec(g, dk, r, pc, gq, lastk); nbox = r ? min(256, CL - pc * 256) / kBoxRows : BM / kBoxRows; } else nbox = SLOT / BOXB;
+      int bytes;                                                             // bytes THIS CTA copies in the stage
+      if (g < G1) { dec(g, dk, r, pc, gq, lastk); bytes = r ? min(256, CL - pc * 256) * 64 : SLOTP; } else bytes = SLOTP;
       if (lane == 0) {
         if (use > 0 && !fail && !mbar_wait(&sm.empty[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
         TL(100 + g);
-        mbar_expect_tx(fb, nbox * BOXB);
+        if (rank == 0) mbar_expect_tx(&sm.full[sl], 2 * bytes);               // bytes of both CTAs
       }
       __syncwarp();
-      if (lane < nbox) {
-        if (g < G1) {
-          if (r == 0) tma_box(slot + lane * BOXB, &map_q, dk * 64, b * rows_seq + row0 + kBoxRows * lane, fb);
-          else {
-            const uint32_t bx = sm.box[pc * (256 / kBoxRows) + lane];
-            tma_box(slot + lane * BOXB, maps[bx >> 30], dk * 64, (int)(bx & 0x3FFFFFFFu), fb);
+      if (g < G1) {
+        if (r == 0) {                                                        // Q: this CTA's 128 rows, one request
+          if (lane == 0) tma_box2(slot, &maps.q, dk * 64, b * rows_seq + row0, fb_leader);
+        } else {      // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
+          const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
+          const bool one = consecutive(i0, nb);                              // nb = 4 (128 rows) or 2 (64 rows)
+          if (one) {
+            if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+          } else if (lane < nb) {
+            const uint32_t bx = sm.box[i0 + lane];
+            tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
           }
-        } else {
-          const int gv = g - G1, part = gv / nvb, kb = gv % nvb;
-          if (NQ == 2) {          // 64 keys x 256 dims: boxes (i = key box, j = 64-wide slice 0..3)
-            const int i = lane >> 2, j = lane & 3;
-            const uint32_t bx = sm.box[kb * (64 / kBoxRows) + i];
-            tma_box(slot + j * 8192 + i * BOXB, maps[bx >> 30], (part * 4 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb);
-          } else {                // 128 keys x 128 dims: boxes (i = key box, j = slice 0..1)
+        }
+      } else {
+        const int gv = g - G1, part = gv / nvb, kb = gv % nvb;
+        if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
+          const int i0 = kb * (64 / kBoxRows);
+          if (consecutive(i0, 2)) {
+            if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+          } else if (lane < 4) {
             const int i = lane >> 1, j = lane & 1;
-            const uint32_t bx = sm.box[kb * (128 / kBoxRows) + i];
-            tma_box(slot + j * 16384 + i * BOXB, maps[bx >> 30], (part * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb);
+            const uint32_t bx = sm.box[i0 + i];
+            tma_box2(slot + j * 8192 + i * BOXB, &maps.src[bx >> 30][0], (part * 4 + (int)rank * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+          }
+        } else {                  // 128 keys x this CTA's 64 dims: key boxes 0..3
+          const int i0 = kb * (128 / kBoxRows);
+          if (consecutive(i0, 4)) {
+            if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][2], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+          } else if (lane < 4) {
+            const uint32_t bx = sm.box[i0 + lane];
+            tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
           }
         }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc_k256 = make_idesc(256, 0), idesc_k128 = make_idesc(128, 0), idesc_v = make_idesc(OW, 1);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc_k256 = make_idesc2(256, 0), idesc_k128 = make_idesc2(128, 0), idesc_v = make_idesc2(OW, 1);
       auto need_ev = [&](int e) { if (!fail && !mbar_wait(&sm.cmp_ev[e], 0)) fail = 1; };
       for (int g = 0; g < GT; ++g) {
         const int sl = g % NSX;
         if (!fail && !mbar_wait(&sm.full[sl], (uint32_t)(g / NSX) & 1u)) fail = 1;
-        TL(300 + g);
-        const uint32_t slot = ring + (uint32_t)sl * SLOT;
+        TL(200 + g);
+        const uint32_t slot = ring + (uint32_t)sl * SLOTP;
         if (g < G1) {
           int dk, r, pc, gq; bool lastk;
           dec(g, dk, r, pc, gq, lastk);
@@ -211,17 +273,17 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (pc == 2 && dk == 0) need_ev(1);        // piece 2 reuses the S columns of piece 1
             fence_after();
             const int qsl = gq % NSX;
-            const uint32_t qslot = ring + (uint32_t)qsl * SLOT;
+            const uint32_t qslot = ring + (uint32_t)qsl * SLOTP;
             const uint32_t scol = tm + (pc == 0 ? 0 : 256);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-              mma_ss(scol, make_desc(qslot + ks * 32, 16, 1024), make_desc(slot + ks * 32, 16, 1024),
-                     ntk == 256 ? idesc_k256 : idesc_k128, (dk | ks) != 0);
-            mma_commit(&sm.empty[sl]);
+              mma2_ss(scol, make_desc(qslot + ks * 32, 16, 1024), make_desc(slot + ks * 32, 16, 1024),
+                      ntk == 256 ? idesc_k256 : idesc_k128, (dk | ks) != 0);
+            mma2_commit(&sm.empty[sl]);
             if (lastk) {
-              mma_commit(&sm.empty[qsl]);                 // the Q slice of this pass and dk is no longer needed
+              mma2_commit(&sm.empty[qsl]);                // the Q slices of this pass and dk are no longer needed
               if (dk == 7) {                              // the S pieces of this pass are complete
-                if (g < GA) { mma_commit(&sm.acc_ev[0]); if (npA == 2) mma_commit(&sm.acc_ev[1]); } else mma_commit(&sm.acc_ev[2]);
+                if (g < GA) { mma2_commit(&sm.acc_ev[0]); if (npA == 2) mma2_commit(&sm.acc_ev[1]); } else mma2_commit(&sm.acc_ev[2]);
               }
             }
           }
@@ -229,19 +291,18 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           const int gv = g - G1, part = gv / nvb, kb = gv % nvb;
           if (kb == 0) need_ev(part == 0 ? npc - 1 : 3 + part - 1);   // all of P is in TMEM / the previous part of O has been read out
           fence_after();
-          if (NQ == 2) {
+          if (NQ == 2) {          // per CTA: 64 keys x 128 dims = two [64 x 64] tiles
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-              mma_ts(tm + OCOL, tm + kb * 32 + ks * 8, make_desc(slot + ks * 2048, 8192, 1024), idesc_v, (kb | ks) != 0);
-          } else {
+              mma2_ts(tm + OCOL, tm + kb * 32 + ks * 8, make_desc(slot + ks * 2048, 8192, 1024), idesc_v, (kb | ks) != 0);
+          } else {                // per CTA: 128 keys x 64 dims = one [128 x 64] tile
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-              mma_ts(tm + OCOL, tm + kb * 64 + ks * 8, make_desc(slot + ks * 2048, 16384, 1024), idesc_v, (kb | ks) != 0);
+              mma2_ts(tm + OCOL, tm + kb * 64 + ks * 8, make_desc(slot + ks * 2048, 16384, 1024), idesc_v, (kb | ks) != 0);
           }
-          mma_commit(&sm.empty[sl]);
-          if (kb == nvb - 1) mma_commit(&sm.acc_ev[3 + part]);
+          mma2_commit(&sm.empty[sl]);
+          if (kb == nvb - 1) mma2_commit(&sm.acc_ev[3 + part]);
         }
-        TL(500 + g);
       }
     }
     __syncwarp();
@@ -250,14 +311,14 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int q4 = warp & 3, hh = (warp - 2) >> 2;
     const int row = q4 * 32 + lane;
     const uint32_t tlane = tm + ((uint32_t)(q4 * 32) << 16);
-    const uint32_t mybit = 1u << (row / s.H);
+    const uint32_t mybit = 1u << ((int)rank * (BM / s.H) + row / s.H);      // node of this row within the pair's plan tile
     const float scale2 = s.sm_scale * 1.4426950408889634f;
     float m_run = -INFINITY, l_part = 0.f;           // reference max (log2 units); this thread's share of the row sum
 
     for (int pc = 0; pc < npc; ++pc) {
       if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
       fence_after();
-      if (warp == 2 && lane == 0) TL(700 + 2 * pc);
+      if (warp == 2 && lane == 0) TL(300 + 2 * pc);
       const int pkeys = min(256, CL - pc * 256);
       const bool mine = hh * 128 < pkeys;            // this warp's 128-key block exists in the piece
       const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128;   // S block (fp32 columns)
@@ -358,8 +419,8 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.cmp_ev[pc]);    // this piece's P is in TMEM; its S columns may be reused
-      if (warp == 2 && lane == 0) TL(701 + 2 * pc);
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[pc]), 0));   // this piece's P is in TMEM (tells the leader's MMA warp)
+      if (warp == 2 && lane == 0) TL(301 + 2 * pc);
     }
     sm.xch[hh][row] = l_part;
     compute_sync();
@@ -369,12 +430,12 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const bool full_tile = row0 + BM <= rows_seq;     // whole tile inside the sequence: rows may be stored as 32-row boxes
     const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
     const int cw = OW / 2;                            // columns of the part this thread handles: 128 or 64
-    const uint32_t stage = ring + (uint32_t)NSX * SLOT + (uint32_t)(warp - 2) * 4096;   // this warp's 32 rows x 64 columns (bf16)
+    const uint32_t stage = ring + (uint32_t)NSX * SLOTP + (uint32_t)(warp - 2) * 4096;   // this warp's 32 rows x 64 columns (bf16)
     bool store_pending = false;
     for (int part = 0; part < NQ; ++part) {
       if (!fail && !mbar_wait(&sm.acc_ev[3 + part], 0)) fail = 1;
       fence_after();
-      if (warp == 2 && lane == 0) TL(720 + 2 * part);
+      if (warp == 2 && lane == 0) TL(320 + 2 * part);
       for (int c0 = 0; c0 < cw; c0 += 64) {
         uint32_t r0[32], r1[32];
         tmem_ld32(tlane + OCOL + hh * cw + c0, r0);
@@ -382,7 +443,7 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (c0 + 64 >= cw && part < NQ - 1) {         // last columns are in registers: the MMA may overwrite this part
           fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.cmp_ev[3 + part]);
+          if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[3 + part]), 0));
         }
         const int col = part * OW + hh * cw + c0;
         if (nch == 1 && full_tile) {
@@ -407,7 +468,7 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           __syncwarp();
           if (lane == 0) {
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(col), "r"(b * rows_seq + row0 + q4 * 32), "r"(stage) : "memory");
+                         ::"l"(reinterpret_cast<uint64_t>(&maps.out)), "r"(col), "r"(b * rows_seq + row0 + q4 * 32), "r"(stage) : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           store_pending = true;
@@ -426,7 +487,7 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
           }
         } else {
-          float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((tix * pl.tc_chmax + chunk) * BM + row) * DH + col;
+          float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((rix * pl.tc_chmax + chunk) * BM + row) * DH + col;
 #pragma unroll
           for (int v = 0; v < 8; ++v) {
             *reinterpret_cast<float4*>(po + v * 4) = make_float4(__uint_as_float(r0[v * 4]), __uint_as_float(r0[v * 4 + 1]),
@@ -437,16 +498,15 @@ tc_attn_tma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
       }
       if (nch > 1 && part == 0 && hh == 0)
-        reinterpret_cast<float2*>(ws + pl.off_tpml)[(tix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
+        reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
     }
     if (store_pending && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
-  if (warp == 2 && lane == 0) TL(740);
   if (fail) atomicOr(status + b, TSV_ST_INTERNAL);
   fence_before();
   __syncthreads();
-  if (tid == 0) TL(741);
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tm) : "memory");
+  cluster_sync_all();                                            // neither CTA leaves while the other may still signal it or read its memory
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tm) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -473,20 +533,46 @@ static bool make_map(CUtensorMap* m, const void* basep, int64_t rows, int box_ro
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool tva_tc_tma_usable(const tsv_cache& c) { return c.csa_rows > 0 && c.hca_rows > 0 && encode_fn() != nullptr; }
+bool tva_tc_pair_usable(const tsv_cache& c) { return c.csa_rows > 0 && c.hca_rows > 0 && encode_fn() != nullptr; }
 
-int launch_tva_tc_tma(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
                       int32_t* status, cudaStream_t st) {
-  CUtensorMap mq, mc, mh, mw, mm, mo;
-  if (!make_map(&mq, nd.q, (int64_t)s.B * s.D * s.H) || !make_map(&mc, c.csa_kv, c.csa_rows) || !make_map(&mh, c.hca_kv, c.hca_rows) ||
-      !make_map(&mw, c.win_kv, (int64_t)s.B * s.window) || !make_map(&mm, ws + p.off_misc, (int64_t)s.B * p.tc_misc_rows) ||
-      !make_map(&mo, out, (int64_t)s.B * s.D * s.H, 32))
+  pair::MapSet ms;
+  const void* bases[4] = {c.csa_kv, c.hca_kv, c.win_kv, ws + p.off_misc};
+  const int64_t rows[4] = {c.csa_rows, c.hca_rows, (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
+  bool ok = make_map(&ms.q, nd.q, (int64_t)s.B * s.D * s.H, 128) && make_map(&ms.out, out, (int64_t)s.B * s.D * s.H, 32);
+  for (int a = 0; a < 4 && ok; ++a)
+    for (int k = 0; k < 3 && ok; ++k) ok = make_map(&ms.src[a][k], bases[a], rows[a], 32 << k);
+  if (!ok) {
+    fprintf(stderr, "tsv: cuTensorMapEncodeTiled failed\n");
     return TSV_ERR_CUDA;
-  if (cudaFuncSetAttribute(tc_attn_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tma::SMEM_X) != cudaSuccess) return TSV_ERR_CUDA;
-  TSV_PREP(tc_attn_tma_kernel);
-  tc_attn_tma_kernel<<<dim3(p.tc_chmax, p.tc_nt, s.B), tma::TTHREADS, tma::SMEM_X, st>>>(mq, mc, mh, mw, mm, mo, s, p, out, ws, status);
+  }
+  if (cudaFuncSetAttribute(tc_attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_X) != cudaSuccess) {
+    fprintf(stderr, "tsv: cannot set %d bytes of dynamic shared memory: %s\n", pair::SMEM_X, cudaGetErrorString(cudaGetLastError()));
+    return TSV_ERR_CUDA;
+  }
+  TSV_PREP(tc_attn_pair_kernel);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * p.tc_nt, p.tc_chmax, s.B);
+  cfg.blockDim = dim3(pair::TTHREADS, 1, 1);
+  cfg.dynamicSmemBytes = pair::SMEM_X;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel, ms, s, p, out, ws, status);
+  if (le != cudaSuccess) {
+    int ncl = -1;
+    cudaOccupancyMaxActiveClusters(&ncl, tc_attn_pair_kernel, &cfg);
+    fprintf(stderr, "tsv: cluster launch failed: %s (max active clusters %d, grid %d x %d x %d)\n", cudaGetErrorString(le), ncl,
+            cfg.gridDim.x, cfg.gridDim.y, cfg.gridDim.z);
+  }
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) fprintf(stderr, "tsv: launch of the paired attention kernel failed: %s\n", cudaGetErrorString(e));
+  return e == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }
 
 }  // namespace tsv
