@@ -48,9 +48,6 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   p.ks = (int32_t)ks;
   p.nsplit = (int32_t)((p.keys_max + ks - 1) / ks);
   size_t off = 0;
-#ifdef TSV_TIMELINE
-  off = 8192;   // experiment: first bytes of the workspace hold clock stamps of one CTA
-#endif
   p.off_selcnt = off; off = up256(off + (size_t)s.B * s.D * sizeof(int32_t));
   p.off_sel = off;    off = up256(off + (size_t)s.B * s.D * s.topk * sizeof(int32_t));
   p.off_scores = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.cand_cap * sizeof(float));
@@ -58,7 +55,7 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
   p.tc = tva_tc_eligible(s);
   p.tc_nt = p.tc_maxk = p.tc_chmax = p.tc_tma = p.tc_misc_rows = 0;
-  p.off_kptr = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = off;
+  p.off_kptr = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = p.off_order = p.off_counter = off;
   if (p.tc) {
     tva_tc_plan_sizes(s, p);
     const size_t tiles = (size_t)s.B * p.tc_nt;
@@ -70,6 +67,8 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
     p.off_box = off;   off = up256(off + tiles * (p.tc_maxk / 32) * 2 * sizeof(int32_t));
     p.off_mode = off;  off = up256(off + tiles * sizeof(int32_t));
     p.off_misc = off;  off = up256(off + (size_t)s.B * p.tc_misc_rows * s.d * 2);
+    p.off_order = off; off = up256(off + tiles * sizeof(int32_t));
+    p.off_counter = off; off = up256(off + sizeof(uint32_t));
   }
   p.total = off;
   return true;

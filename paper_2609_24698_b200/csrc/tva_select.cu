@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
+  if (pl.tc && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *reinterpret_cast<unsigned int*>(ws + pl.off_counter) = 0u;   // the plan kernel's finished-CTA counter
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
   if (threadIdx.x == 0) {
     if (tm.status && n == 0) atomicOr(status + b, tm.status);

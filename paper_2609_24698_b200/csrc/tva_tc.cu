@@ -26,9 +26,8 @@ namespace tsv {
 
 
 // ------------------------------------------------------------------------------------------------ plan
-__global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
-                                                      const tsv_scratch sc, char* __restrict__ ws) {
-  extern __shared__ uint8_t cmask[];                   // [cand_cap] node bits per committed CSA entry (ranked case only)
+__device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
+                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
   __shared__ int wsum[9];
@@ -209,6 +208,36 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
     }
     *nkeys = base;
   }
+}
+
+// Plan of every (sequence, 256-row tile).  The CTA that finishes last also orders the tiles by decreasing key count:
+// the paired attention kernel takes tiles in that order, so the long ones start first and the short ones fill the tail
+// (the grid is less than two waves of CTA pairs, and tile lengths differ by an order of magnitude).
+__global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                      const tsv_scratch sc, char* __restrict__ ws) {
+  extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
+  __shared__ int is_last;
+  tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
+  __threadfence();
+  __syncthreads();
+  unsigned int* counter = reinterpret_cast<unsigned int*>(ws + pl.off_counter);
+  if (threadIdx.x == 0) is_last = atomicAdd(counter, 1u) == gridDim.x * gridDim.y - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const int n = s.B * pl.tc_nt;
+  const volatile int32_t* nkeys = reinterpret_cast<const volatile int32_t*>(ws + pl.off_nkeys);
+  int32_t* order = reinterpret_cast<int32_t*>(ws + pl.off_order);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    int rank = i;
+    if (n <= 4096) {                                    // rank = tiles with more keys (ties: lower index first)
+      const int ki = nkeys[i];
+      rank = 0;
+      for (int j = 0; j < n; ++j) { const int kj = nkeys[j]; rank += (kj > ki) || (kj == ki && j < i); }
+    }
+    order[rank] = i;
+  }
+  if (threadIdx.x == 0) *counter = 0;                   // ready for the next call on this workspace
 }
 
 // ------------------------------------------------------------------------------------------------ attention

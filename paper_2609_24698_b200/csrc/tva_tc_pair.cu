@@ -25,7 +25,8 @@ namespace pair {
 
 using namespace tc;
 
-constexpr int TTHREADS = 352;               // warps 0 and 10: producers (even / odd stages); 1: MMA issuer; 2-9: softmax and epilogue
+constexpr int NPROD = 2;                    // producer warps: warp 0 and warps 10.., stage g belongs to producer g % NPROD
+constexpr int TTHREADS = 32 * (10 + NPROD - 1);   // warp 1: MMA issuer; warps 2-9: softmax and epilogue
 constexpr int BOXB = kBoxRows * 128;       // bytes of one box: kBoxRows rows x 128 bytes
 constexpr float RESCALE_GAP = 16.f;        // log2 units a later piece's row max may exceed the running reference
 
@@ -77,13 +78,10 @@ __device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
                ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
 }
-// arrives on the same barrier (same shared-memory offset) in both CTAs of the pair once all prior MMAs have completed:
-// one commit per destination CTA, each addressed through its cluster address
+// arrives on the same barrier (same shared-memory offset) in both CTAs of the pair once all prior MMAs have completed
 __device__ __forceinline__ void mma2_commit(uint64_t* bar) {
-  const uint32_t a = smem_u32(bar);
-#pragma unroll
-  for (uint32_t r = 0; r < 2; ++r)
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_rank(a, r)) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 __device__ __forceinline__ uint32_t make_idesc2(int N, int b_mn_major) {      // M = 256 over the pair
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
@@ -115,12 +113,16 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
                     const TvaPlan pl, void* __restrict__ out_, char* __restrict__ ws, int32_t* __restrict__ status) {
   using namespace pair;
   extern __shared__ unsigned char smem_raw[];
-  const int chunk = blockIdx.y, tile = blockIdx.x >> 1, b = blockIdx.z;       // the two CTAs of a pair are neighbours in x
+  // the two CTAs of a pair are neighbours in x; pairs take the (sequence, tile) items in the order the plan kernel left
+  // (most keys first)
+  const int chunk = blockIdx.y;
+  const int item = reinterpret_cast<const int32_t*>(ws + pl.off_order)[blockIdx.x >> 1];
+  const int b = item / pl.tc_nt, tile = item % pl.tc_nt;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const size_t tix = (size_t)b * pl.tc_nt + tile;
-  const size_t rix = (size_t)b * 2 * pl.tc_nt + blockIdx.x;      // this CTA's 128-row tile (partials of multi-chunk tiles)
+  const size_t rix = (size_t)b * 2 * pl.tc_nt + 2 * tile + rank;  // this CTA's 128-row tile (partials of multi-chunk tiles)
   // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
   if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 1) return;      // not a contiguous-run tile
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
@@ -181,14 +183,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   const int G1 = GA + (npc > 2 ? 16 : 0);
   const int nvb = CL / vkeys;                       // V stages per part
   const int GT = G1 + NQ * nvb;
-#ifdef TSV_TIMELINE
-  long long* tl = reinterpret_cast<long long*>(ws) + (rank ? 400 : 0);
-  const bool tlon = (blockIdx.x < 2 && blockIdx.y == 0 && blockIdx.z == 0);
-#define TL(i) do { if (tlon) tl[i] = clock64(); } while (0)
-  if (tlon && tid == 0) { tl[0] = clock64(); tl[1] = CL; tl[2] = GT; }
-#else
-#define TL(i) do { } while (0)
-#endif
 
   // S stage g -> slice dk of d, r (0 = Q stage, else K stage), piece pc of the K stage, index gq of the pass's Q stage for dk
   auto dec = [&](int g, int& dk, int& r, int& pc, int& gq, bool& lastk) {
@@ -196,9 +190,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     else { const int h = g - GA; dk = h >> 1; r = h & 1; pc = 2; gq = GA + 2 * dk; lastk = r == 1; }
   };
 
-  if (warp == 0 || warp == 10) {
-    // ------------------------------------------------------------------ producers (both CTAs): warp 0 takes the even stages, warp 10 the odd ones
-    const int pw = warp == 0 ? 0 : 1;
+  if (warp == 0 || warp >= 10) {
+    // ------------------------------------------------------------------ producers (both CTAs): stage g is issued by producer g % NPROD
+    const int pw = warp == 0 ? 0 : warp - 9;
     // consecutive: do the nb boxes starting at list index i0 name consecutive rows of one array?
     auto consecutive = [&](int i0, int nb) {
       const uint32_t b0 = sm.box[i0];
@@ -206,7 +200,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       for (int i = 1; i < nb; ++i) if (sm.box[i0 + i] != b0 + (uint32_t)(i * kBoxRows)) return false;
       return true;
     };
-    for (int g = pw; g < GT; g += 2) {
+    for (int g = pw; g < GT; g += NPROD) {
       const int sl = g % NSX, use = g / NSX;
       const uint32_t slot = ring + (uint32_t)sl * SLOTP;
       const uint32_t fb_leader = map_to_rank(smem_u32(&sm.full[sl]), 0);     // both CTAs' copies complete on the leader's barrier
@@ -215,7 +209,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       if (g < G1) { dec(g, dk, r, pc, gq, lastk); bytes = r ? min(256, CL - pc * 256) * 64 : SLOTP; } else bytes = SLOTP;
       if (lane == 0) {
         if (use > 0 && !fail && !mbar_wait(&sm.empty[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
-        TL(100 + g);
         if (rank == 0) mbar_expect_tx(&sm.full[sl], 2 * bytes);               // bytes of both CTAs
       }
       __syncwarp();
@@ -263,7 +256,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       for (int g = 0; g < GT; ++g) {
         const int sl = g % NSX;
         if (!fail && !mbar_wait(&sm.full[sl], (uint32_t)(g / NSX) & 1u)) fail = 1;
-        TL(200 + g);
         const uint32_t slot = ring + (uint32_t)sl * SLOTP;
         if (g < G1) {
           int dk, r, pc, gq; bool lastk;
@@ -318,7 +310,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     for (int pc = 0; pc < npc; ++pc) {
       if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
       fence_after();
-      if (warp == 2 && lane == 0) TL(300 + 2 * pc);
       const int pkeys = min(256, CL - pc * 256);
       const bool mine = hh * 128 < pkeys;            // this warp's 128-key block exists in the piece
       const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128;   // S block (fp32 columns)
@@ -337,18 +328,23 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         }
         vis[c] = v;
       }
+      // the thread's 128 S values are read from TMEM once and stay in registers for both passes (max, then exp)
+      uint32_t sv[128];
       float mx = -INFINITY;
       if (mine) {
 #pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32_nowait(scol + c * 32, sv + c * 32);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_regs_ready(sv + c * 32);
+#pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(scol + c * 32, r);
           if (vis[c] == 0xffffffffu) {
 #pragma unroll
-            for (int t = 0; t < 32; ++t) mx = fmaxf(mx, __uint_as_float(r[t]));
+            for (int t = 0; t < 32; ++t) mx = fmaxf(mx, __uint_as_float(sv[c * 32 + t]));
           } else {
 #pragma unroll
-            for (int t = 0; t < 32; ++t) if ((vis[c] >> t) & 1u) mx = fmaxf(mx, __uint_as_float(r[t]));
+            for (int t = 0; t < 32; ++t) if ((vis[c] >> t) & 1u) mx = fmaxf(mx, __uint_as_float(sv[c * 32 + t]));
           }
         }
       }
@@ -382,29 +378,26 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         l_part *= factor;
       }
       const float moff = (m_run == -INFINITY) ? 0.f : m_run;
-      uint32_t pk[64];
-      if (mine) {
+      if (mine) {                                    // P overwrites the S values pairwise: sv[0..63] then hold the packed bf16 pairs
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(scol + c * 32, r);
           if (vis[c] == 0xffffffffu) {
 #pragma unroll
             for (int t = 0; t < 32; t += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(r[t]), scale2, -moff));
-              const float p1 = ex2(fmaf(__uint_as_float(r[t + 1]), scale2, -moff));
+              const float p0 = ex2(fmaf(__uint_as_float(sv[c * 32 + t]), scale2, -moff));
+              const float p1 = ex2(fmaf(__uint_as_float(sv[c * 32 + t + 1]), scale2, -moff));
               l_part += p0 + p1;
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);     // low half = even key
-              pk[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+              sv[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
             }
           } else {
 #pragma unroll
             for (int t = 0; t < 32; t += 2) {
-              const float p0 = ((vis[c] >> t) & 1u) ? ex2(fmaf(__uint_as_float(r[t]), scale2, -moff)) : 0.f;
-              const float p1 = ((vis[c] >> (t + 1)) & 1u) ? ex2(fmaf(__uint_as_float(r[t + 1]), scale2, -moff)) : 0.f;
+              const float p0 = ((vis[c] >> t) & 1u) ? ex2(fmaf(__uint_as_float(sv[c * 32 + t]), scale2, -moff)) : 0.f;
+              const float p1 = ((vis[c] >> (t + 1)) & 1u) ? ex2(fmaf(__uint_as_float(sv[c * 32 + t + 1]), scale2, -moff)) : 0.f;
               l_part += p0 + p1;
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-              pk[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+              sv[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
             }
           }
         }
@@ -414,13 +407,12 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       fence_after();
       if (mine) {
 #pragma unroll
-        for (int v = 0; v < 4; ++v) tmem_st16(tlane + pc * 128 + hh * 64 + v * 16, pk + v * 16);
+        for (int v = 0; v < 4; ++v) tmem_st16(tlane + pc * 128 + hh * 64 + v * 16, sv + v * 16);
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[pc]), 0));   // this piece's P is in TMEM (tells the leader's MMA warp)
-      if (warp == 2 && lane == 0) TL(301 + 2 * pc);
     }
     sm.xch[hh][row] = l_part;
     compute_sync();
@@ -435,7 +427,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     for (int part = 0; part < NQ; ++part) {
       if (!fail && !mbar_wait(&sm.acc_ev[3 + part], 0)) fail = 1;
       fence_after();
-      if (warp == 2 && lane == 0) TL(320 + 2 * part);
       for (int c0 = 0; c0 < cw; c0 += 64) {
         uint32_t r0[32], r1[32];
         tmem_ld32(tlane + OCOL + hh * cw + c0, r0);
@@ -553,7 +544,7 @@ int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c,
   }
   TSV_PREP(tc_attn_pair_kernel);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * p.tc_nt, p.tc_chmax, s.B);
+  cfg.gridDim = dim3(2 * p.tc_nt * s.B, p.tc_chmax, 1);
   cfg.blockDim = dim3(pair::TTHREADS, 1, 1);
   cfg.dynamicSmemBytes = pair::SMEM_X;
   cfg.stream = st;
