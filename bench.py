@@ -25,9 +25,9 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# dram bytes per tree_verify_attn attention launch at the bench workload, from the ncu capture
-# summarised under profiles/ (None until measured for the current kernel).
-NCU_ATTN_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one tc_attn_pair_kernel launch on one layer of the bench workload
+# (ncu capture summarised in profiles/ncu_tc_attn_pair_kernel_cfg4.md): 65.25 MB read + 4.52 MB written.
+NCU_ATTN_TRAFFIC_BYTES = 69_774_592
 
 
 def peaks():
@@ -211,40 +211,50 @@ def run_ours(args, cfg):
     assert int(eng.status.sum()) == 0
     value, sec = D.whole_job_throughput(sh.B * sh.D * K, sec_local, dev)
 
-    # ---- per-kernel pass (eager, CUDA events on the launching stream): attention kernel alone
+    # ---- per-stage pass: each stage of the cycle captured alone in a CUDA graph (all layers) and replayed, timed with
+    # CUDA events on the launching stream.  Graph replay keeps the host out of the measurement; the attention stage is
+    # tree_verify_attn without its selection step (tile plan + paired attention kernel + merge of multi-chunk tiles).
     eng.restore(snap)
     sel_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_ATTN)
     att_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_SELECT)
-    ev = []
-    t_parts = {"branch_state_build": [], "select": [], "attention": [], "accept_and_refresh": []}
-    for i in range(Wm + K):
-        inp = wl.inputs[i % n_sets]
-        eng.status.zero_()
-        marks = []
-        for l in range(eng.n_layers):
-            m = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-            m[0].record(stream)
-            tsv.branch_state_build(eng.cshape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.status)
-            m[1].record(stream)
-            tsv.tree_verify_attn(sel_shape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
-            m[2].record(stream)
-            tsv.tree_verify_attn(att_shape, eng.caches[l], inp.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
-            m[3].record(stream)
-            marks.append(m)
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a0.record(stream)
-        tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path, eng.bonus, eng.status)
-        a1.record(stream)
-        if i >= Wm:
-            ev.append((marks, a0, a1))
+    inp0 = wl.inputs[0]
+    eng.launch_cycle(inp0, refresh=False)           # scratch pads and selections of inp0 are in place for the partial graphs
     torch.cuda.synchronize()
-    for marks, a0, a1 in ev:
-        for m in marks:
-            t_parts["branch_state_build"].append(m[0].elapsed_time(m[1]))
-            t_parts["select"].append(m[1].elapsed_time(m[2]))
-            t_parts["attention"].append(m[2].elapsed_time(m[3]))
-        t_parts["accept_and_refresh"].append(a0.elapsed_time(a1))
-    attn_ms = float(np.mean(t_parts["attention"]))
+
+    def stage_fn(name):
+        def f():
+            for l in range(eng.n_layers):
+                if name == "branch_state_build":
+                    tsv.branch_state_build(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.status)
+                elif name == "select":
+                    tsv.tree_verify_attn(sel_shape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+                elif name == "attention":
+                    tsv.tree_verify_attn(att_shape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+        return f
+
+    t_parts = {}
+    for name in ("branch_state_build", "select", "attention"):
+        sg = torch.cuda.Stream(); sg.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=sg):
+            stage_fn(name)()
+        stream.wait_stream(sg)
+        for _ in range(Wm):
+            g.replay()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(K):
+            g.replay()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        t_parts[name] = s0.elapsed_time(s1) / K / eng.n_layers          # ms per layer-call
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    tsv.accept_and_refresh(eng.cshape, eng._pack(inp0), inp0.draft, inp0.target, eng.accept_len, eng.accept_path, eng.bonus, eng.status)
+    a1.record(stream)
+    torch.cuda.synchronize()
+    t_parts["accept_and_refresh"] = a0.elapsed_time(a1)
+    attn_ms = float(t_parts["attention"])
 
     # ---- algorithmic work and roofline of the dominant kernel (attention)
     parents = wl.inputs[0].layers[0].parent.cpu().numpy()
@@ -252,7 +262,7 @@ def run_ours(args, cfg):
     pk = peaks()
     attn_gbs = work["attn_bytes_per_layer"] / (attn_ms * 1e-3) / 1e9
     attn_tf = work["attn_flops_per_layer"] / (attn_ms * 1e-3) / 1e12
-    roofline = {"bound": "hbm", "kernel": "tree_verify_attn attention kernel (one layer, all sequences)",
+    roofline = {"bound": "hbm", "kernel": "tree_verify_attn attention stage: tile plan + tc_attn_pair_kernel (one layer, all sequences)",
                 "achieved": attn_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / pk["hbm_gbs"],
                 "traffic": NCU_ATTN_TRAFFIC_BYTES, "peak_source": pk["source"], "launch_ms": attn_ms,
                 "algorithmic_bytes_per_launch": work["attn_bytes_per_layer"],
@@ -263,7 +273,7 @@ def run_ours(args, cfg):
              "frac_hbm_full": work["full_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
              "frac_hbm_cache": work["cache_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
              "frac_tensor_sustained": work["flops"] / cycle_s / 1e12 / pk["bf16_tflops_sustained"],
-             "stage_ms_per_call_eager": {k: float(np.mean(v)) for k, v in t_parts.items()},
+             "stage_ms_per_layer_call": {k: float(v) for k, v in t_parts.items()},
              "accepted_tokens_per_cycle_last": accepted}
 
     # ---- end to end: host buffers in, acceptance result out, every step

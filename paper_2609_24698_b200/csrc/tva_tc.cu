@@ -1,25 +1,24 @@
-// tree_verify_attn on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 storage, d = 512.
+// tree_verify_attn on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 storage, d = 512: the tile plan, the
+// pointer-gather attention kernel and the merge of multi-chunk tiles.  (The main attention kernel, for key lists made of
+// contiguous runs, is in tva_tc_pair.cu.)
 //
-// One CTA = (sequence, row tile, key chunk).  A row tile is 128 query rows = 128/H consecutive
-// tree nodes x H heads; all of them attend over the SAME staged key rows (key == value, MQA), so
-// S = Q K^T and O = P K are dense 128 x N x 512 contractions.  Which node sees which key is a
-// per-key bitmask applied to the S fragment after it is read back from tensor memory.
+// Rows are grouped in plan tiles of 256 query rows = 256/H consecutive tree nodes x H heads; all of them attend over the
+// SAME staged key rows (key == value, MQA), so S = Q K^T and O = P K are dense contractions.  Which node sees which key is
+// a per-key bitmask applied to the S fragment after it is read back from tensor memory.
 //
-//   tc_plan_kernel   per (sequence, tile): the list of key rows visible to at least one node of
-//                    the tile (union of the nodes' CSA selections, HCA entries, window slots,
-//                    tree nodes, in-tree entries) as row pointers + node bitmasks.
-//   tc_attn_kernel   per (sequence, tile, chunk of <= 512 keys):
-//       phase 1  S[128 x CL] = Q K^T      tcgen05.mma kind::f16, A = Q sub-tile (smem, K-major),
-//                                         B = 256 key rows x 64 dims (smem, K-major), D in TMEM
-//       phase 2  exact softmax of the chunk on the fp32 S read with tcgen05.ld; P (bf16) is
-//                written back into TMEM over S with tcgen05.st
-//       phase 3  O[128 x 256] = P K[:, half]  twice; A = P from TMEM, B = 64 key rows x 256 dims
-//                (smem, MN-major); epilogue reads O with tcgen05.ld and stores bf16 rows
-//     Operand tiles stream through a ring of seven 32 KiB slots filled with 16-byte cp.async
-//     copies written in the 128-byte swizzle pattern (any row from any of the six source arrays,
-//     zero fill for padding), four stages ahead of the MMA issue; slots are released by
-//     tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
-//   tc_combine_kernel merges the chunks of tiles that needed more than one (fixed order).
+//   tc_plan_kernel   per (sequence, plan tile): the keys visible to at least one node of the tile.
+//                    mode 1 (every node selects all CSA candidates, or the CSA slab is at most 2 x topk rows): contiguous
+//                    runs {CSA slab, HCA slab, window ring, packed misc rows} as 32-row TMA boxes + node masks;
+//                    mode 0 (selection far from dense): row pointers of the union of the nodes' selections + masks.
+//                    The last CTA to finish orders the tiles by key count for the paired kernel.
+//   tc_attn_kernel   mode-0 tiles, one CTA per 128 rows and chunk of <= 512 keys:
+//       phase 1  S[128 x CL] = Q K^T      tcgen05.mma kind::f16, A = Q slice (smem, K-major), B = 256 key rows x 64 dims
+//       phase 2  exact softmax of the chunk on the fp32 S read with tcgen05.ld; P (bf16) written back over S (tcgen05.st)
+//       phase 3  O[128 x 256] = P K[:, half] twice; A = P from TMEM, B = 64 key rows x 256 dims (smem, MN-major)
+//     Operand tiles stream through a ring of seven 32 KiB slots filled with 16-byte cp.async copies written in the
+//     128-byte swizzle pattern (any row from any source array, zero fill for padding), four stages ahead of the MMA
+//     issue; slots are released by tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
+//   tc_combine_kernel merges the chunks of tiles that needed more than one (fixed order), per 128 rows.
 #include "tc_common.cuh"
 
 namespace tsv {
