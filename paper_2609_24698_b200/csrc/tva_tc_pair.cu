@@ -253,48 +253,55 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     if (lane == 0 && rank == 0) {
       const uint32_t idesc_k256 = make_idesc2(256, 0), idesc_k128 = make_idesc2(128, 0), idesc_v = make_idesc2(OW, 1);
       auto need_ev = [&](int e) { if (!fail && !mbar_wait(&sm.cmp_ev[e], 0)) fail = 1; };
-      for (int g = 0; g < GT; ++g) {
-        const int sl = g % NSX;
-        if (!fail && !mbar_wait(&sm.full[sl], (uint32_t)(g / NSX) & 1u)) fail = 1;
-        const uint32_t slot = ring + (uint32_t)sl * SLOTP;
-        if (g < G1) {
-          int dk, r, pc, gq; bool lastk;
-          dec(g, dk, r, pc, gq, lastk);
-          if (r) {
-            const int ntk = min(256, CL - pc * 256);
-            if (pc == 2 && dk == 0) need_ev(1);        // piece 2 reuses the S columns of piece 1
+      // The issuing thread is the pacemaker of the tensor pipe: stages are walked with counters (no divisions), and the
+      // descriptors of a stage are the slot-0 descriptor plus a multiple of the slot size (the address field counts
+      // 16-byte units and cannot overflow within the ring).
+      const uint64_t dk0 = make_desc(ring, 16, 1024), dv0 = make_desc(ring, NQ == 2 ? 8192 : 16384, 1024);
+      int sl = 0; uint32_t ph = 0;                       // slot and parity of the next stage
+      auto wait_full = [&]() { if (!fail && !mbar_wait(&sm.full[sl], ph)) fail = 1; };
+      auto advance = [&]() { if (++sl == NSX) { sl = 0; ph ^= 1u; } };
+      // one pass over d for pieces [pc0, pc0 + np): per 64-wide slice the Q stage, then one K stage per piece
+      auto s_pass = [&](int pc0, int np) {
+        for (int dk = 0; dk < 8; ++dk) {
+          wait_full();
+          const int qsl = sl;
+          const uint64_t qd = dk0 + (uint64_t)(sl * (SLOTP >> 4));
+          advance();
+          for (int pc = pc0; pc < pc0 + np; ++pc) {
+            wait_full();
+            if (pc == 2 && dk == 0) need_ev(1);          // piece 2 reuses the S columns of piece 1
             fence_after();
-            const int qsl = gq % NSX;
-            const uint32_t qslot = ring + (uint32_t)qsl * SLOTP;
+            const uint64_t kd = dk0 + (uint64_t)(sl * (SLOTP >> 4));
             const uint32_t scol = tm + (pc == 0 ? 0 : 256);
+            const uint32_t idesc = CL - pc * 256 >= 256 ? idesc_k256 : idesc_k128;
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              mma2_ss(scol, make_desc(qslot + ks * 32, 16, 1024), make_desc(slot + ks * 32, 16, 1024),
-                      ntk == 256 ? idesc_k256 : idesc_k128, (dk | ks) != 0);
+            for (int ks = 0; ks < 4; ++ks) mma2_ss(scol, qd + 2 * ks, kd + 2 * ks, idesc, (dk | ks) != 0);
             mma2_commit(&sm.empty[sl]);
-            if (lastk) {
-              mma2_commit(&sm.empty[qsl]);                // the Q slices of this pass and dk are no longer needed
-              if (dk == 7) {                              // the S pieces of this pass are complete
-                if (g < GA) { mma2_commit(&sm.acc_ev[0]); if (npA == 2) mma2_commit(&sm.acc_ev[1]); } else mma2_commit(&sm.acc_ev[2]);
-              }
-            }
+            advance();
           }
-        } else {
-          const int gv = g - G1, part = gv / nvb, kb = gv % nvb;
-          if (kb == 0) need_ev(part == 0 ? npc - 1 : 3 + part - 1);   // all of P is in TMEM / the previous part of O has been read out
+          mma2_commit(&sm.empty[qsl]);                  // the Q slice of this pass and dk is no longer needed
+        }
+        for (int pc = pc0; pc < pc0 + np; ++pc) mma2_commit(&sm.acc_ev[pc]);   // the S pieces of this pass are complete
+      };
+      s_pass(0, npA);
+      if (npc > 2) s_pass(2, 1);
+      for (int part = 0; part < NQ; ++part) {
+        need_ev(part == 0 ? npc - 1 : 3 + part - 1);     // all of P is in TMEM / the previous part of O has been read out
+        for (int kb = 0; kb < nvb; ++kb) {
+          wait_full();
           fence_after();
+          const uint64_t vd = dv0 + (uint64_t)(sl * (SLOTP >> 4));
           if (NQ == 2) {          // per CTA: 64 keys x 128 dims = two [64 x 64] tiles
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              mma2_ts(tm + OCOL, tm + kb * 32 + ks * 8, make_desc(slot + ks * 2048, 8192, 1024), idesc_v, (kb | ks) != 0);
+            for (int ks = 0; ks < 4; ++ks) mma2_ts(tm + OCOL, tm + kb * 32 + ks * 8, vd + ks * (2048 >> 4), idesc_v, (kb | ks) != 0);
           } else {                // per CTA: 128 keys x 64 dims = one [128 x 64] tile
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              mma2_ts(tm + OCOL, tm + kb * 64 + ks * 8, make_desc(slot + ks * 2048, 16384, 1024), idesc_v, (kb | ks) != 0);
+            for (int ks = 0; ks < 8; ++ks) mma2_ts(tm + OCOL, tm + kb * 64 + ks * 8, vd + ks * (2048 >> 4), idesc_v, (kb | ks) != 0);
           }
           mma2_commit(&sm.empty[sl]);
-          if (kb == nvb - 1) mma2_commit(&sm.acc_ev[3 + part]);
+          advance();
         }
+        mma2_commit(&sm.acc_ev[3 + part]);
       }
     }
     __syncwarp();
