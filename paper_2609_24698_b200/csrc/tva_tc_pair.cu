@@ -122,6 +122,8 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const size_t tix = (size_t)b * pl.tc_nt + tile;
+  if (tid < 14)      // the descriptors of all 14 tensor maps are fetched while the plan is read
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps) + (uint64_t)tid * sizeof(CUtensorMap)) : "memory");
   const size_t rix = (size_t)b * 2 * pl.tc_nt + 2 * tile + rank;  // this CTA's 128-row tile (partials of multi-chunk tiles)
   // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
   if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 1) return;      // not a contiguous-run tile
@@ -184,12 +186,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   const int nvb = CL / vkeys;                       // V stages per part
   const int GT = G1 + NQ * nvb;
 
-  // S stage g -> slice dk of d, r (0 = Q stage, else K stage), piece pc of the K stage, index gq of the pass's Q stage for dk
-  auto dec = [&](int g, int& dk, int& r, int& pc, int& gq, bool& lastk) {
-    if (g < GA) { dk = g / perA; r = g % perA; pc = r - 1; gq = dk * perA; lastk = r == perA - 1; }
-    else { const int h = g - GA; dk = h >> 1; r = h & 1; pc = 2; gq = GA + 2 * dk; lastk = r == 1; }
-  };
-
   if (warp == 0 || warp >= 10) {
     // ------------------------------------------------------------------ producers (both CTAs): stage g is issued by producer g % NPROD
     const int pw = warp == 0 ? 0 : warp - 9;
@@ -200,52 +196,61 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       for (int i = 1; i < nb; ++i) if (sm.box[i0 + i] != b0 + (uint32_t)(i * kBoxRows)) return false;
       return true;
     };
-    for (int g = pw; g < GT; g += NPROD) {
-      const int sl = g % NSX, use = g / NSX;
-      const uint32_t slot = ring + (uint32_t)sl * SLOTP;
-      const uint32_t fb_leader = map_to_rank(smem_u32(&sm.full[sl]), 0);     // both CTAs' copies complete on the leader's barrier
-      int dk = 0, r = 0, pc = 0, gq = 0; bool lastk = false;
-      int bytes;                                                             // bytes THIS CTA copies in the stage
-      if (g < G1) { dec(g, dk, r, pc, gq, lastk); bytes = r ? min(256, CL - pc * 256) * 64 : SLOTP; } else bytes = SLOTP;
-      if (lane == 0) {
-        if (use > 0 && !fail && !mbar_wait(&sm.empty[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
-        if (rank == 0) mbar_expect_tx(&sm.full[sl], 2 * bytes);               // bytes of both CTAs
-      }
-      __syncwarp();
-      if (g < G1) {
-        if (r == 0) {                                                        // Q: this CTA's 128 rows, one request
-          if (lane == 0) tma_box2(slot, &maps.q, dk * 64, b * rows_seq + row0, fb_leader);
-        } else {      // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
-          const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
-          const bool one = consecutive(i0, nb);                              // nb = 4 (128 rows) or 2 (64 rows)
-          if (one) {
-            if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-          } else if (lane < nb) {
-            const uint32_t bx = sm.box[i0 + lane];
-            tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+    // all stages are walked with counters (no divisions); this producer issues every NPROD-th one
+    const uint32_t full0 = map_to_rank(smem_u32(&sm.full[0]), 0);           // both CTAs' copies complete on the leader's barrier
+    int sl = 0, use = 0;                             // ring slot of stage g and how often it has been used before
+    int dk = 0, r = 0, per = perA, pc0 = -1;         // S stages: slice of d, position r within the slice (0 = Q, else piece pc0 + r)
+    int part = 0, kb = 0;                            // V stages
+    for (int g = 0; g < GT; ++g) {
+      const bool is_s = g < G1;
+      const int pc = pc0 + r;
+      if ((g & (NPROD - 1)) == pw) {
+        const uint32_t slot = ring + (uint32_t)sl * SLOTP;
+        const uint32_t fb_leader = full0 + (uint32_t)sl * 8u;
+        const int bytes = (is_s && r) ? min(256, CL - pc * 256) * 64 : SLOTP;  // bytes THIS CTA copies in the stage
+        if (lane == 0) {
+          if (use > 0 && !fail && !mbar_wait(&sm.empty[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
+          if (rank == 0) mbar_expect_tx(&sm.full[sl], 2 * bytes);               // bytes of both CTAs
+        }
+        __syncwarp();
+        if (is_s) {
+          if (r == 0) {                                                        // Q: this CTA's 128 rows, one request
+            if (lane == 0) tma_box2(slot, &maps.q, dk * 64, b * rows_seq + row0, fb_leader);
+          } else {      // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
+            const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
+            const bool one = consecutive(i0, nb);                              // nb = 4 (128 rows) or 2 (64 rows)
+            if (one) {
+              if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+            } else if (lane < nb) {
+              const uint32_t bx = sm.box[i0 + lane];
+              tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+            }
+          }
+        } else {
+          if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
+            const int i0 = kb * (64 / kBoxRows);
+            if (consecutive(i0, 2)) {
+              if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+            } else if (lane < 4) {
+              const int i = lane >> 1, j = lane & 1;
+              const uint32_t bx = sm.box[i0 + i];
+              tma_box2(slot + j * 8192 + i * BOXB, &maps.src[bx >> 30][0], (part * 4 + (int)rank * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+            }
+          } else {                  // 128 keys x this CTA's 64 dims: key boxes 0..3
+            const int i0 = kb * (128 / kBoxRows);
+            if (consecutive(i0, 4)) {
+              if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][2], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+            } else if (lane < 4) {
+              const uint32_t bx = sm.box[i0 + lane];
+              tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+            }
           }
         }
-      } else {
-        const int gv = g - G1, part = gv / nvb, kb = gv % nvb;
-        if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
-          const int i0 = kb * (64 / kBoxRows);
-          if (consecutive(i0, 2)) {
-            if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-          } else if (lane < 4) {
-            const int i = lane >> 1, j = lane & 1;
-            const uint32_t bx = sm.box[i0 + i];
-            tma_box2(slot + j * 8192 + i * BOXB, &maps.src[bx >> 30][0], (part * 4 + (int)rank * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
-          }
-        } else {                  // 128 keys x this CTA's 64 dims: key boxes 0..3
-          const int i0 = kb * (128 / kBoxRows);
-          if (consecutive(i0, 4)) {
-            if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][2], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-          } else if (lane < 4) {
-            const uint32_t bx = sm.box[i0 + lane];
-            tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
-          }
-        }
       }
+      if (++sl == NSX) { sl = 0; ++use; }
+      if (is_s) {
+        if (++r == per) { r = 0; if (++dk == 8) { dk = 0; per = 2; pc0 = 1; } }   // pass B: the Q stage, then piece 2
+      } else if (++kb == nvb) { kb = 0; ++part; }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -312,115 +317,172 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     const uint32_t tlane = tm + ((uint32_t)(q4 * 32) << 16);
     const uint32_t mybit = 1u << ((int)rank * (BM / s.H) + row / s.H);      // node of this row within the pair's plan tile
     const float scale2 = s.sm_scale * 1.4426950408889634f;
-    float m_run = -INFINITY, l_part = 0.f;           // reference max (log2 units); this thread's share of the row sum
+    float m_run = -INFINITY;                         // reference max of the row (log2 units)
+    float lp[4] = {0.f, 0.f, 0.f, 0.f};              // this thread's share of the row sum, four independent chains
 
-    for (int pc = 0; pc < npc; ++pc) {
-      if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
-      fence_after();
-      const int pkeys = min(256, CL - pc * 256);
-      const bool mine = hh * 128 < pkeys;            // this warp's 128-key block exists in the piece
-      const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128;   // S block (fp32 columns)
-      const int k0 = pc * 256 + hh * 128;                              // first key of the block within the chunk
-      // visibility of the block's keys for this lane's row, 32 keys per word (bit t = key c0 + t)
-      uint32_t vis[4];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint32_t mk = mine ? sm.kmask[k0 + c * 32 + lane] : 0u;
-        // lanes of a warp may belong to different nodes when H < 32: one ballot per node bit present in the warp
-        const uint32_t lo = __shfl_sync(0xffffffffu, mybit, 0), hi = __shfl_sync(0xffffffffu, mybit, 31);
+    // The softmax code works on slabs of 32 keys in short loops: the kernel passes through it once per piece, so long
+    // unrolled code would be fetched cold every time.
+    //
+    // Visibility of every slab for this lane's row, 32 keys per word (bit t = key t of the slab).  It does not depend on
+    // S: the words are computed while the S products run and parked in the (still unused) output staging area.
+    uint32_t* visw = reinterpret_cast<uint32_t*>(smem_raw + CTLB + NSX * SLOTP) + (warp - 2) * 32 + lane;   // [piece * 4 + slab][256 threads]
+    {
+      // lanes of a warp may belong to different nodes when H < 32: one ballot per node bit present in the warp
+      const uint32_t lo = __shfl_sync(0xffffffffu, mybit, 0), hi = __shfl_sync(0xffffffffu, mybit, 31);
+#pragma unroll 1
+      for (int i = 0; i < 4 * npc; ++i) {
+        const int pc = i >> 2, c = i & 3;
+        const bool mine = hh * 128 < min(256, CL - pc * 256);
+        const uint32_t mk = mine ? sm.kmask[pc * 256 + hh * 128 + c * 32 + lane] : 0u;
         uint32_t v = __ballot_sync(0xffffffffu, mk & mybit);
         if (lo != hi) {
           v = 0;
           for (uint32_t bit = lo; bit <= hi; bit <<= 1) { const uint32_t w = __ballot_sync(0xffffffffu, mk & bit); if (bit == mybit) v = w; }
         }
-        vis[c] = v;
+        visw[i * 256] = v;
       }
-      // the thread's 128 S values are read from TMEM once and stay in registers for both passes (max, then exp)
-      uint32_t sv[128];
-      float mx = -INFINITY;
-      if (mine) {
+    }
+    // masked maximum of one slab of S (fp32 columns [col, col + 32))
+    auto slab_max = [&](uint32_t col, uint32_t vis, float mx) {
+      uint32_t sv[32];
+      tmem_ld32(col, sv);
+      float mc[4] = {mx, -INFINITY, -INFINITY, -INFINITY};
+      if (vis == 0xffffffffu) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32_nowait(scol + c * 32, sv + c * 32);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int t = 0; t < 32; ++t) mc[t & 3] = fmaxf(mc[t & 3], __uint_as_float(sv[t]));
+      } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_regs_ready(sv + c * 32);
+        for (int t = 0; t < 32; ++t) if ((vis >> t) & 1u) mc[t & 3] = fmaxf(mc[t & 3], __uint_as_float(sv[t]));
+      }
+      return fmaxf(fmaxf(mc[0], mc[1]), fmaxf(mc[2], mc[3]));
+    };
+    // P of one slab: 32 S values -> 16 bf16 pairs (low half = even key) stored at P columns [pcol, pcol + 16); the row
+    // sum shares go to lp
+    auto slab_exp = [&](const uint32_t* sv, uint32_t vis, float moff, uint32_t pcol) {
+      uint32_t pk[16];
+      if (vis == 0xffffffffu) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (vis[c] == 0xffffffffu) {
+        for (int t = 0; t < 32; t += 2) {
+          const float p0 = ex2(fmaf(__uint_as_float(sv[t]), scale2, -moff));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[t + 1]), scale2, -moff));
+          lp[(t >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+          pk[t >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
+      } else {
 #pragma unroll
-            for (int t = 0; t < 32; ++t) mx = fmaxf(mx, __uint_as_float(sv[c * 32 + t]));
-          } else {
-#pragma unroll
-            for (int t = 0; t < 32; ++t) if ((vis[c] >> t) & 1u) mx = fmaxf(mx, __uint_as_float(sv[c * 32 + t]));
-          }
+        for (int t = 0; t < 32; t += 2) {
+          const float p0 = ((vis >> t) & 1u) ? ex2(fmaf(__uint_as_float(sv[t]), scale2, -moff)) : 0.f;
+          const float p1 = ((vis >> (t + 1)) & 1u) ? ex2(fmaf(__uint_as_float(sv[t + 1]), scale2, -moff)) : 0.f;
+          lp[(t >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+          pk[t >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
         }
       }
-      sm.xch[hh][row] = mx;
-      compute_sync();
-      const float m_piece = fmaxf(sm.xch[0][row], sm.xch[1][row]) * scale2;
-      // Keep one reference max per row.  A later piece may exceed it by up to RESCALE_GAP (weights up to 2^16 are
-      // harmless in bf16/fp32); beyond that the P written so far and the running sum are rescaled.
-      float factor = 1.f;
-      if (m_piece > m_run + RESCALE_GAP || m_run == -INFINITY) {
-        if (m_run != -INFINITY) factor = ex2(m_run - m_piece);
-        m_run = m_piece;
-      }
-      if (__any_sync(0xffffffffu, factor != 1.f)) {  // warp-uniform: tcgen05.ld/st are warp-collective
-        for (int pj = 0; pj < pc; ++pj) {
-          const uint32_t pcol = tlane + pj * 128 + hh * 64;
-#pragma unroll
-          for (int v = 0; v < 2; ++v) {
-            uint32_t r[32];
-            tmem_ld32(pcol + v * 32, r);
-#pragma unroll
-            for (int t = 0; t < 32; ++t) {
-              float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r[t]));
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(f.x * factor, f.y * factor);
-              r[t] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-            tmem_st16(pcol + v * 32, r);
-            tmem_st16(pcol + v * 32 + 16, r + 16);
-          }
-        }
-        l_part *= factor;
-      }
-      const float moff = (m_run == -INFINITY) ? 0.f : m_run;
-      if (mine) {                                    // P overwrites the S values pairwise: sv[0..63] then hold the packed bf16 pairs
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (vis[c] == 0xffffffffu) {
-#pragma unroll
-            for (int t = 0; t < 32; t += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(sv[c * 32 + t]), scale2, -moff));
-              const float p1 = ex2(fmaf(__uint_as_float(sv[c * 32 + t + 1]), scale2, -moff));
-              l_part += p0 + p1;
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);     // low half = even key
-              sv[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-          } else {
-#pragma unroll
-            for (int t = 0; t < 32; t += 2) {
-              const float p0 = ((vis[c] >> t) & 1u) ? ex2(fmaf(__uint_as_float(sv[c * 32 + t]), scale2, -moff)) : 0.f;
-              const float p1 = ((vis[c] >> (t + 1)) & 1u) ? ex2(fmaf(__uint_as_float(sv[c * 32 + t + 1]), scale2, -moff)) : 0.f;
-              l_part += p0 + p1;
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-              sv[(c * 32 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-          }
-        }
-      }
-      fence_before();
-      compute_sync();                                // both S blocks of the piece have been read by every warp
-      fence_after();
-      if (mine) {
-#pragma unroll
-        for (int v = 0; v < 4; ++v) tmem_st16(tlane + pc * 128 + hh * 64 + v * 16, sv + v * 16);
-      }
+      tmem_st16(pcol, pk);
+    };
+    auto p_stored = [&](int pc) {                    // this warp's P of piece pc is in TMEM: tell the leader's MMA warp
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[pc]), 0));   // this piece's P is in TMEM (tells the leader's MMA warp)
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[pc]), 0));
+    };
+    auto block_mine = [&](int pc) { return hh * 128 < min(256, CL - pc * 256); };
+
+    // Pass A: pieces 0 and 1 complete together and share one row maximum.  Pass B: piece 2 arrives later; the reference
+    // maximum is kept unless the piece exceeds it by more than RESCALE_GAP (weights up to 2^16 are harmless in
+    // bf16/fp32), else the P written so far and the sums are rescaled.
+    //
+    // Where P lands: piece pc -> columns [128 pc, 128 pc + 128), the warps with hh = 0 write the lower 64 (keys of their S
+    // block, the piece's first 128), the warps with hh = 1 the upper 64.  P of pieces 0 and 2 overlays the first half of the
+    // piece's own S: a warp with hh = 0 writes behind its own reads (slab c -> P columns 16 c.. below the 32 c.. it has
+    // read), but the warps with hh = 1 write over S slabs 2 and 3 of their hh = 0 neighbours, so those are read into
+    // registers first and a named barrier tells the neighbours.  P of piece 1 overlays S of piece 0, which every warp
+    // has finished with at the barrier between the pieces.
+#pragma unroll 1
+    for (int pass = 0; pass < (npc == 3 ? 2 : 1); ++pass) {
+      const int pcb = pass ? 2 : 0, pce = pass ? 3 : npA;
+#pragma unroll 1
+      for (int pc = pcb; pc < pce; ++pc)
+        if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
+      fence_after();
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int pc = pcb; pc < pce; ++pc) {
+        if (!block_mine(pc)) continue;
+        const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) mx = slab_max(scol + c * 32, visw[(pc * 4 + c) * 256], mx);
+      }
+      sm.xch[hh][row] = mx;
+      compute_sync();
+      const float m_pass = fmaxf(sm.xch[0][row], sm.xch[1][row]) * scale2;
+      float factor = 1.f;
+      if (m_pass > m_run + RESCALE_GAP || m_run == -INFINITY) {
+        if (m_run != -INFINITY) factor = ex2(m_run - m_pass);
+        m_run = m_pass;
+      }
+      if (pass && __any_sync(0xffffffffu, factor != 1.f)) {  // warp-uniform: tcgen05.ld/st are warp-collective
+#pragma unroll 1
+        for (int v = 0; v < 4; ++v) {
+          const uint32_t pcol = tlane + (v >> 1) * 128 + hh * 64 + (v & 1) * 32;
+          uint32_t r[32];
+          tmem_ld32(pcol, r);
+#pragma unroll
+          for (int t = 0; t < 32; ++t) {
+            float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r[t]));
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(f.x * factor, f.y * factor);
+            r[t] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          tmem_st16(pcol, r);
+          tmem_st16(pcol + 16, r + 16);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) lp[c] *= factor;
+      }
+      const float moff = (m_run == -INFINITY) ? 0.f : m_run;
+#pragma unroll 1
+      for (int pc = pcb; pc < pce; ++pc) {
+        if (pc != pcb) {       // P of piece 1 overlays S of piece 0: every warp has read it for the last time
+          fence_before();
+          compute_sync();
+          fence_after();
+        }
+        const bool mine = block_mine(pc);
+        const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128, pcol = tlane + pc * 128 + hh * 64;
+        const uint32_t* vw = visw + pc * 4 * 256;
+        uint32_t hold[64];
+        if (hh == 0) {
+          if (mine) {
+            tmem_ld32_nowait(scol + 64, hold);
+            tmem_ld32_nowait(scol + 96, hold + 32);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            tmem_regs_ready(hold);
+            tmem_regs_ready(hold + 32);
+          }
+          fence_before();
+          asm volatile("bar.arrive 2, 256;" ::: "memory");
+        } else {
+          asm volatile("bar.sync 2, 256;" ::: "memory");
+          fence_after();
+        }
+        if (mine) {
+          const int nstream = hh == 0 ? 2 : 4;
+#pragma unroll 1
+          for (int c = 0; c < nstream; ++c) {
+            uint32_t sv[32];
+            tmem_ld32(scol + c * 32, sv);
+            slab_exp(sv, vw[c * 256], moff, pcol + c * 16);
+          }
+          if (hh == 0) {
+            slab_exp(hold, vw[2 * 256], moff, pcol + 32);
+            slab_exp(hold + 32, vw[3 * 256], moff, pcol + 48);
+          }
+        }
+        p_stored(pc);
+      }
     }
+    const float l_part = (lp[0] + lp[1]) + (lp[2] + lp[3]);
     sm.xch[hh][row] = l_part;
     compute_sync();
     const float l_row = sm.xch[0][row] + sm.xch[1][row];
@@ -434,15 +496,25 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     for (int part = 0; part < NQ; ++part) {
       if (!fail && !mbar_wait(&sm.acc_ev[3 + part], 0)) fail = 1;
       fence_after();
-      for (int c0 = 0; c0 < cw; c0 += 64) {
-        uint32_t r0[32], r1[32];
-        tmem_ld32(tlane + OCOL + hh * cw + c0, r0);
-        tmem_ld32(tlane + OCOL + hh * cw + c0 + 32, r1);
-        if (c0 + 64 >= cw && part < NQ - 1) {         // last columns are in registers: the MMA may overwrite this part
-          fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[3 + part]), 0));
-        }
+      // the thread's columns of the part (128 or 64) go to registers at once, so that the MMA may overwrite the part
+      // while the values are normalised and stored
+      uint32_t ro[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) if (c * 32 < cw) tmem_ld32_nowait(tlane + OCOL + hh * cw + c * 32, ro + c * 32);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_regs_ready(ro + c * 32);
+      if (part < NQ - 1) {
+        fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&sm.cmp_ev[3 + part]), 0));
+      }
+#pragma unroll
+      for (int cg = 0; cg < 2; ++cg) {
+        const int c0 = cg * 64;
+        if (c0 >= cw) break;
+        const uint32_t* r0 = ro + cg * 64;
+        const uint32_t* r1 = ro + cg * 64 + 32;
         const int col = part * OW + hh * cw + c0;
         if (nch == 1 && full_tile) {
           // stage the 32 x 64 bf16 tile in the 128-byte swizzle pattern and store it with one TMA request
