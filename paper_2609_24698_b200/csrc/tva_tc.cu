@@ -40,9 +40,15 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
   const int32_t* selcnt = reinterpret_cast<const int32_t*>(ws + pl.off_selcnt) + (size_t)b * D;
   const int32_t* sel = reinterpret_cast<const int32_t*>(ws + pl.off_sel) + (size_t)b * D * s.topk;
-  const uint8_t* cdone = sc.csa_done + (size_t)b * D;
-  const uint8_t* hdone = sc.hca_done + (size_t)b * D;
+  // the done flags and the cache row offsets are fetched together with the tree scalars (one memory latency for all)
+  __shared__ uint8_t cdone[TSV_MAX_D], hdone[TSV_MAX_D];
+  __shared__ int64_t row0_sm[2];
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + D) cdone[threadIdx.x - 64] = sc.csa_done[(size_t)b * D + threadIdx.x - 64];
+  if (threadIdx.x >= 96 && threadIdx.x < 96 + D) hdone[threadIdx.x - 96] = sc.hca_done[(size_t)b * D + threadIdx.x - 96];
+  if (threadIdx.x == 40) row0_sm[0] = c.csa_row0[b];
+  if (threadIdx.x == 41) row0_sm[1] = c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  const int64_t csa_row0 = row0_sm[0], hca_row0 = row0_sm[1];
   if (threadIdx.x == 0) {
     int dn = 1;
     for (int nl = 0; nl < npt; ++nl) {
@@ -95,7 +101,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
         const int r = i / cpr, cc = i % cpr;
         const char* src = nullptr;
-        if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)c.hca_row0[b] + r) * rowb;
+        if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)hca_row0 + r) * rowb;
         else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
         else if (r < n_misc) {
           int ord = r - nh_in - tm.nn;
@@ -144,8 +150,8 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         }
         kb += nb * kBoxRows;
       };
-      emit(0, c.csa_row0[b], n_csa, 0);
-      if (tm.n_hca > kHcaMiscMax) emit(1, c.hca_row0[b], tm.n_hca, 1);
+      emit(0, csa_row0, n_csa, 0);
+      if (tm.n_hca > kHcaMiscMax) emit(1, hca_row0, tm.n_hca, 1);
       emit(2, (int64_t)b * s.window, min(tm.L, s.window), 2);
       emit(3, (int64_t)b * pl.tc_misc_rows, n_misc, 3);
       if (threadIdx.x == 0) { *nkeys = kb; *mode = 1; }
@@ -160,12 +166,12 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const uint32_t m = i < n_csa ? (dense ? validbits : cmask[i]) : 0u;
     int tot;
     const int pos = base + block_excl_scan_256(m != 0, wsum, tot);
-    if (m) { kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)c.csa_row0[b] + i) * rowb); kmask[pos] = (uint8_t)m; }
+    if (m) { kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)csa_row0 + i) * rowb); kmask[pos] = (uint8_t)m; }
     base += tot;
   }
   // committed HCA entries
   for (int i = threadIdx.x; i < tm.n_hca; i += blockDim.x) {
-    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + ((size_t)c.hca_row0[b] + i) * rowb); kmask[base + i] = (uint8_t)validbits;
+    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + ((size_t)hca_row0 + i) * rowb); kmask[base + i] = (uint8_t)validbits;
   }
   base += tm.n_hca;
   // committed window positions seen by at least one node of the tile
@@ -227,12 +233,17 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   const int n = s.B * pl.tc_nt;
   const volatile int32_t* nkeys = reinterpret_cast<const volatile int32_t*>(ws + pl.off_nkeys);
   int32_t* order = reinterpret_cast<int32_t*>(ws + pl.off_order);
+  __shared__ int32_t nk_sm[2048];                       // the counts are fetched once; the ranking reads them from shared memory
+  if (n <= 2048) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) nk_sm[i] = nkeys[i];
+    __syncthreads();
+  }
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     int rank = i;
-    if (n <= 4096) {                                    // rank = tiles with more keys (ties: lower index first)
-      const int ki = nkeys[i];
+    if (n <= 2048) {                                    // rank = tiles with more keys (ties: lower index first)
+      const int ki = nk_sm[i];
       rank = 0;
-      for (int j = 0; j < n; ++j) { const int kj = nkeys[j]; rank += (kj > ki) || (kj == ki && j < i); }
+      for (int j = 0; j < n; ++j) { const int kj = nk_sm[j]; rank += (kj > ki) || (kj == ki && j < i); }
     }
     order[rank] = i;
   }
@@ -595,7 +606,7 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
   TvaPlan p = p_in;
   p.tc_tma = tva_tc_pair_usable(c) ? 1 : 0;
   const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
-  if (plan_sm > 48 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
+  if (plan_sm > 32 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
     return TSV_ERR_CUDA;
   TSV_PREP(tc_plan_kernel);
   TSV_PREP(tc_attn_kernel);
