@@ -222,6 +222,8 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
   __shared__ int is_last;
+  if (threadIdx.x < 2)                                // finished-chunk counters of the tile's two 128-row halves
+    reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[((size_t)blockIdx.y * pl.tc_nt + blockIdx.x) * 2 + threadIdx.x] = 0;
   tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
   __threadfence();
   __syncthreads();
@@ -553,7 +555,8 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   const size_t tix = (size_t)b * pl.tc_nt + tile, rix = (size_t)b * 2 * pl.tc_nt + rt;
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   int nch, CL;
-  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] == 1) chunking_x(nk, nch, CL); else chunking(nk, nch, CL);
+  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] == 1) return;     // the paired kernel merges its own chunks
+  chunking(nk, nch, CL);
   if (nk <= 0 || nch <= 1) return;
   const int rows_seq = s.D * s.H, row0 = rt * BM;
   bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
@@ -617,14 +620,17 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
     const int r = launch_tva_tc_pair(s, p, c, nd, out, ws, status, st);
     if (r != TSV_OK) return r;
   }
-  if (!p.tc_tma || p.need_scores) {            // tiles with ranked selections (or no TMA): pointer-gather kernel
+  // The pointer-gather kernel serves tiles whose committed CSA run is longer than twice the selection size (and every
+  // tile when the caches do not allow TMA).  With capacities that rule such tiles out it is not launched, nor is the
+  // merge kernel: the paired kernel merges the chunks of its own tiles.
+  if (!p.tc_tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk)) {
     if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
     tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
-  }
-  if (p.tc_chmax > 1) {
-    tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
-    count_launch();
+    if (p.tc_chmax > 1) {
+      tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
+      count_launch();
+    }
   }
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }

@@ -40,7 +40,7 @@ struct Ctl {                               // control block at the start of dyna
   uint64_t cmp_ev[6];                      // compute warps -> MMA, one barrier per event, each used once:
                                            //   [pc] P of piece pc is in TMEM   [3 + p] part p of O has been read out
   uint32_t tmem_base;
-  int32_t pad;
+  int32_t merge_here;                      // set for the CTA that finished a multi-chunk tile last
   uint32_t box[NCX / kBoxRows];            // tensor map id << 30 | first row
   uint8_t kmask[NCX];
   float xch[2][BM];
@@ -571,6 +571,45 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
     }
     if (store_pending && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (nch > 1) {
+      // Tiles of several chunks: each chunk leaves its unnormalised part of O with (max, sum) per row; the CTA that
+      // finishes a 128-row tile last merges the parts (fixed order, so the result does not depend on who was last).
+      __threadfence();
+      compute_sync();
+      if (warp == 2 && lane == 0) {
+        int32_t* cnt = reinterpret_cast<int32_t*>(ws + pl.off_tcnt) + rix;
+        const int done = atomicAdd(cnt, 1);
+        sm.merge_here = done == nch - 1;
+      }
+      compute_sync();
+      if (sm.merge_here) {
+        __threadfence();
+        bf16* orow0 = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
+        const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + rix * pl.tc_chmax * BM * DH;
+        const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM;
+        for (int i = (warp - 2) * 32 + lane; i < BM * DH / 8; i += 256) {
+          const int r = i / (DH / 8), c8 = i % (DH / 8);
+          if (row0 + r >= rows_seq) continue;
+          float m = -INFINITY;
+          for (int ch = 0; ch < nch; ++ch) { const float2 ml = __ldcg(pml + ch * BM + r); if (ml.y > 0.f) m = fmaxf(m, ml.x); }
+          float l = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          for (int ch = 0; ch < nch; ++ch) {
+            const float2 ml = __ldcg(pml + ch * BM + r);
+            if (!(ml.y > 0.f)) continue;
+            const float w = exp2f(ml.x - m);
+            l = fmaf(ml.y, w, l);
+            const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + r) * DH + c8 * 8);
+            const float4 a = __ldcg(p4), bq = __ldcg(p4 + 1);
+            o[0] = fmaf(a.x, w, o[0]); o[1] = fmaf(a.y, w, o[1]); o[2] = fmaf(a.z, w, o[2]); o[3] = fmaf(a.w, w, o[3]);
+            o[4] = fmaf(bq.x, w, o[4]); o[5] = fmaf(bq.y, w, o[5]); o[6] = fmaf(bq.z, w, o[6]); o[7] = fmaf(bq.w, w, o[7]);
+          }
+          const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+          for (int t = 0; t < 8; ++t) o[t] *= inv;
+          st16(orow0 + (size_t)r * DH + c8 * 8, o);
+        }
+      }
+    }
   }
   if (fail) atomicOr(status + b, TSV_ST_INTERNAL);
   fence_before();
