@@ -67,7 +67,7 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
     p.off_box = off;   off = up256(off + tiles * (p.tc_maxk / 32) * 2 * sizeof(int32_t));
     p.off_mode = off;  off = up256(off + tiles * sizeof(int32_t));
     p.off_misc = off;  off = up256(off + (size_t)s.B * p.tc_misc_rows * s.d * 2);
-    p.off_order = off; off = up256(off + tiles * sizeof(int32_t));
+    p.off_order = off; off = up256(off + tiles * 4 * sizeof(int32_t));
     p.off_counter = off; off = up256(off + sizeof(uint32_t));
     p.off_tcnt = off;  off = up256(off + 2 * tiles * sizeof(int32_t));     // finished chunks per 128-row tile (paired kernel)
   }

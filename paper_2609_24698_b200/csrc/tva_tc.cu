@@ -234,7 +234,9 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   __threadfence();
   const int n = s.B * pl.tc_nt;
   const volatile int32_t* nkeys = reinterpret_cast<const volatile int32_t*>(ws + pl.off_nkeys);
-  int32_t* order = reinterpret_cast<int32_t*>(ws + pl.off_order);
+  const volatile int32_t* mode = reinterpret_cast<const volatile int32_t*>(ws + pl.off_mode);
+  int4* order = reinterpret_cast<int4*>(ws + pl.off_order);    // {tile index, mode, keys, -} per position: the paired kernel
+                                                               // learns all it needs about its tile from one load
   __shared__ int32_t nk_sm[2048];                       // the counts are fetched once; the ranking reads them from shared memory
   if (n <= 2048) {
     for (int i = threadIdx.x; i < n; i += blockDim.x) nk_sm[i] = nkeys[i];
@@ -242,12 +244,12 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   }
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     int rank = i;
+    const int ki = nkeys[i];
     if (n <= 2048) {                                    // rank = tiles with more keys (ties: lower index first)
-      const int ki = nk_sm[i];
       rank = 0;
       for (int j = 0; j < n; ++j) { const int kj = nk_sm[j]; rank += (kj > ki) || (kj == ki && j < i); }
     }
-    order[rank] = i;
+    order[rank] = make_int4(i, mode[i], ki, 0);
   }
   if (threadIdx.x == 0) *counter = 0;                   // ready for the next call on this workspace
 }

@@ -116,7 +116,8 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   // the two CTAs of a pair are neighbours in x; pairs take the (sequence, tile) items in the order the plan kernel left
   // (most keys first)
   const int chunk = blockIdx.y;
-  const int item = reinterpret_cast<const int32_t*>(ws + pl.off_order)[blockIdx.x >> 1];
+  const int4 rec = reinterpret_cast<const int4*>(ws + pl.off_order)[blockIdx.x >> 1];   // {tile index, mode, keys, -}: one load
+  const int item = rec.x;
   const int b = item / pl.tc_nt, tile = item % pl.tc_nt;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint32_t rank;
@@ -126,8 +127,8 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps) + (uint64_t)tid * sizeof(CUtensorMap)) : "memory");
   const size_t rix = (size_t)b * 2 * pl.tc_nt + 2 * tile + rank;  // this CTA's 128-row tile (partials of multi-chunk tiles)
   // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
-  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 1) return;      // not a contiguous-run tile
-  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
+  if (rec.y != 1) return;                                      // not a contiguous-run tile
+  const int nk = rec.z;
   const int rows_seq = s.D * s.H, row0 = tile * PR + (int)rank * BM;           // first of this CTA's rows within the sequence
   if (nk <= 0) {                                               // flagged sequence or padding-only tile: zeros
     if (chunk == 0) {

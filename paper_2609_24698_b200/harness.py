@@ -7,6 +7,7 @@ on one CUDA stream with no host synchronisation in between.
 """
 from __future__ import annotations
 
+import weakref
 from typing import Dict, List, Optional, Sequence
 
 import numpy as np
@@ -127,12 +128,14 @@ class VerifyEngine:
         self.accept_len = torch.zeros(B, **i32)
         self.accept_path = torch.zeros(B, D, **i32)
         self.bonus = torch.zeros(B, **i32)
-        self._packs: Dict[int, tsv.LayerPack] = {}
+        # pointer packs per input set; weak keys: an entry must die with its input set (an id() key could be reused by a
+        # later input set and hand accept_and_refresh the pointers of freed tensors)
+        self._packs = weakref.WeakKeyDictionary()
 
     def _pack(self, inp: InputSet) -> tsv.LayerPack:
-        p = self._packs.get(id(inp))
+        p = self._packs.get(inp)
         if p is None:
-            p = self._packs[id(inp)] = tsv.LayerPack(self.caches, inp.layers, self.scratch)
+            p = self._packs[inp] = tsv.LayerPack(self.caches, inp.layers, self.scratch)
         return p
 
     def launch_cycle(self, inp: InputSet, attention: bool = True, refresh: bool = True) -> None:

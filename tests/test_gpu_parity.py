@@ -60,7 +60,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
         tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path,
                                eng.bonus, eng.status)
         torch.cuda.synchronize()
-        assert int(eng.status.abs().sum()) == 0
+        assert int(eng.status.abs().sum()) == 0, f"cycle {cyc}: status flags {eng.status.cpu().tolist()}"
         pairs = [(l, b) for l in range(cfg.layers) for b in range(sh.B)] if out_pairs is None else list(out_pairs(cyc))
         g_alen, g_path, g_bonus = eng.accept_len.cpu().numpy(), eng.accept_path.cpu().numpy(), eng.bonus.cpu().numpy()
         scs = {}
