@@ -18,7 +18,7 @@ constexpr int THREADS = 256;
 constexpr int kHcaMiscMaxTc = 32;
 constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
 constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 14;   // tries between two looks at the clock (see mbar_wait; once a wait gives up, no later wait of the thread is attempted)
+constexpr uint32_t WAIT_LIMIT = 1u << 14;   // polls before a wait gives up (then no later wait of the thread is attempted)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -48,25 +48,16 @@ __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::aft
 // Bounded wait on an mbarrier phase; false if the limit ran out.  Each try suspends the warp in hardware for up to
 // SUSPEND_NS (it wakes as soon as the phase completes), so waiting warps do not compete for issue slots or for the
 // shared-memory pipe with the warps that feed the tensor core.
-// The limit is wall time (how long one try suspends is up to the hardware, so a count of tries bounds nothing useful):
-// after WAIT_LIMIT tries the global timer is consulted, and the wait gives up once WAIT_NS have passed since then.
 constexpr uint32_t SUSPEND_NS = 4000;
-constexpr unsigned long long WAIT_NS = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   const uint32_t a = smem_u32(bar);
-  unsigned long long t_start = 0;
-  for (;;) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-      uint32_t ok;
-      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                   : "=r"(ok) : "r"(a), "r"(parity), "r"(SUSPEND_NS) : "memory");
-      if (ok) return true;
-    }
-    unsigned long long now;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-    if (t_start == 0) t_start = now;
-    else if (now - t_start > WAIT_NS) return false;
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a), "r"(parity), "r"(SUSPEND_NS) : "memory");
+    if (ok) return true;
   }
+  return false;
 }
 
 __device__ __forceinline__ void cp16(uint32_t dst, const void* src, bool valid) {

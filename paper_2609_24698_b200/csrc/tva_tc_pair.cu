@@ -480,7 +480,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
             slab_exp(hold + 32, vw[3 * 256], moff, pcol + 48);
           }
         }
-        p_stored(pc);
+        // the MMA warp waits for the last piece only (and, with three pieces, for piece 1 before it overwrites that
+        // piece's S columns); the wait for the stores of a later piece covers the earlier ones
+        if (pc == npc - 1 || (npc == 3 && pc == 1)) p_stored(pc);
       }
     }
     const float l_part = (lp[0] + lp[1]) + (lp[2] + lp[3]);
