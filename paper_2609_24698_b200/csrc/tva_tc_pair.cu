@@ -30,12 +30,16 @@ constexpr int TTHREADS = 32 * (10 + NPROD - 1);   // warp 1: MMA issuer; warps 2
 constexpr int BOXB = kBoxRows * 128;       // bytes of one box: kBoxRows rows x 128 bytes
 constexpr float RESCALE_GAP = 16.f;        // log2 units a later piece's row max may exceed the running reference
 
-constexpr int NSX = 12;                    // ring slots; a 32 KiB area after the ring stages the output tiles
+constexpr int NSX = 12;                    // 16 KiB slots of the staging area; a 32 KiB area after it stages the output tiles
+constexpr int NQS = 8;                     // S phase: slots [0, 8) hold the Q slices (all of d, resident for every piece),
+constexpr int NKS = NSX - NQS;             //          slots [8, 12) are the ring of the K stages;
+                                           // V phase: all 12 slots form the ring of the V stages
 
 struct Ctl {                               // control block at the start of dynamic shared memory
-  uint64_t full[NSX];
-  uint64_t empty[NSX];
-  uint64_t acc_ev[7];                      // MMA -> compute warps, one barrier per event, each used once:
+  uint64_t fullQ[NQS];                     // Q slice dk has arrived (used once)
+  uint64_t fullK[NKS], emptyK[NKS];        // ring of the K stages
+  uint64_t fullV[NSX], emptyV[NSX];        // ring of the V stages (starts when the S products are complete)
+  uint64_t acc_ev[7];                      // MMA -> other warps, one barrier per event, each used once:
                                            //   [pc] S of piece pc is complete   [3 + p] part p of O is complete
   uint64_t cmp_ev[6];                      // compute warps -> MMA, one barrier per event, each used once:
                                            //   [pc] P of piece pc is in TMEM   [3 + p] part p of O has been read out
@@ -148,7 +152,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   int fail = (smem_u32(smem_raw) & 1023u) ? 1 : 0;             // the swizzled tiles need a 1024-byte aligned base
 
   if (tid == 0) {
-    for (int i = 0; i < NSX; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+    for (int i = 0; i < NQS; ++i) mbar_init(&sm.fullQ[i], 1);
+    for (int i = 0; i < NKS; ++i) { mbar_init(&sm.fullK[i], 1); mbar_init(&sm.emptyK[i], 1); }
+    for (int i = 0; i < NSX; ++i) { mbar_init(&sm.fullV[i], 1); mbar_init(&sm.emptyV[i], 1); }
     for (int i = 0; i < 7; ++i) mbar_init(&sm.acc_ev[i], 1);
     for (int i = 0; i < 6; ++i) mbar_init(&sm.cmp_ev[i], 16);   // 8 compute warps of each CTA
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -181,11 +187,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   const int OW = DH / NQ;                           // columns of one part
   const uint32_t OCOL = 512 - OW;
   const int vkeys = 16384 / OW;                     // keys per V stage: 64 or 128
-  const int npA = npc < 2 ? npc : 2, perA = 1 + npA;
-  const int GA = 8 * perA;
-  const int G1 = GA + (npc > 2 ? 16 : 0);
   const int nvb = CL / vkeys;                       // V stages per part
-  const int GT = G1 + NQ * nvb;
+  const int NKST = 8 * npc;                         // K stages: piece after piece, per piece the eight 64-wide slices of d
+  const int NVST = NQ * nvb;                        // V stages
 
   if (warp == 0 || warp >= 10) {
     // ------------------------------------------------------------------ producers (both CTAs): stage g is issued by producer g % NPROD
@@ -197,61 +201,79 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       for (int i = 1; i < nb; ++i) if (sm.box[i0 + i] != b0 + (uint32_t)(i * kBoxRows)) return false;
       return true;
     };
-    // all stages are walked with counters (no divisions); this producer issues every NPROD-th one
-    const uint32_t full0 = map_to_rank(smem_u32(&sm.full[0]), 0);           // both CTAs' copies complete on the leader's barrier
-    int sl = 0, use = 0;                             // ring slot of stage g and how often it has been used before
-    int dk = 0, r = 0, per = perA, pc0 = -1;         // S stages: slice of d, position r within the slice (0 = Q, else piece pc0 + r)
-    int part = 0, kb = 0;                            // V stages
-    for (int g = 0; g < GT; ++g) {
-      const bool is_s = g < G1;
-      const int pc = pc0 + r;
-      if ((g & (NPROD - 1)) == pw) {
+    // Q slices: producer 0.  K stage gk = 8 pc + dk: producer (gk + 1) & 1, so that the first K stage leaves at the same
+    // time as the first Q slice.  V stage gv: producer gv & 1.  Both CTAs' copies complete on the leader's barriers.
+    auto issue_q = [&](int dk) {
+      if (lane == 0) {
+        if (rank == 0) mbar_expect_tx(&sm.fullQ[dk], 2 * SLOTP);
+        tma_box2(ring + (uint32_t)dk * SLOTP, &maps.q, dk * 64, b * rows_seq + row0, map_to_rank(smem_u32(&sm.fullQ[dk]), 0));
+      }
+      __syncwarp();
+    };
+    auto issue_k = [&](int gk) {
+      const int pc = gk >> 3, dk = gk & 7, sl = gk & (NKS - 1), use = gk >> 2;
+      const uint32_t slot = ring + (uint32_t)(NQS + sl) * SLOTP;
+      const uint32_t fb_leader = map_to_rank(smem_u32(&sm.fullK[sl]), 0);
+      const int bytes = min(256, CL - pc * 256) * 64;                        // bytes THIS CTA copies in the stage
+      if (lane == 0) {
+        if (use > 0 && !fail && !mbar_wait(&sm.emptyK[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
+        if (rank == 0) mbar_expect_tx(&sm.fullK[sl], 2 * bytes);              // bytes of both CTAs
+      }
+      __syncwarp();
+      // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
+      const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
+      if (consecutive(i0, nb)) {                                             // nb = 4 (128 rows) or 2 (64 rows)
+        if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+      } else if (lane < nb) {
+        const uint32_t bx = sm.box[i0 + lane];
+        tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
+      }
+      __syncwarp();
+    };
+    static_assert(NKS == 4, "issue_k derives the slot use from gk >> 2");
+    if (pw == 0) {
+      for (int i = 0; i < 4; ++i) { issue_q(2 * i); issue_q(2 * i + 1); issue_k(2 * i + 1); }
+      for (int gk = 9; gk < NKST; gk += 2) issue_k(gk);
+    } else {
+      for (int gk = 0; gk < NKST; gk += 2) issue_k(gk);
+    }
+    // V stages reuse the whole staging area: they start when the last S product is complete (the softmax of the last
+    // piece is still to come, so the ring is full by the time the PV products start)
+    if (lane == 0 && !fail && !mbar_wait(&sm.acc_ev[npc - 1], 0)) fail = 1;
+    __syncwarp();
+    {
+      int part = 0, kb = pw;
+      while (kb >= nvb) { kb -= nvb; ++part; }
+      for (int gv = pw; gv < NVST; gv += NPROD) {
+        const int sl = gv % NSX, use = gv / NSX;
         const uint32_t slot = ring + (uint32_t)sl * SLOTP;
-        const uint32_t fb_leader = full0 + (uint32_t)sl * 8u;
-        const int bytes = (is_s && r) ? min(256, CL - pc * 256) * 64 : SLOTP;  // bytes THIS CTA copies in the stage
+        const uint32_t fb_leader = map_to_rank(smem_u32(&sm.fullV[sl]), 0);
         if (lane == 0) {
-          if (use > 0 && !fail && !mbar_wait(&sm.empty[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
-          if (rank == 0) mbar_expect_tx(&sm.full[sl], 2 * bytes);               // bytes of both CTAs
+          if (use > 0 && !fail && !mbar_wait(&sm.emptyV[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
+          if (rank == 0) mbar_expect_tx(&sm.fullV[sl], 2 * SLOTP);
         }
         __syncwarp();
-        if (is_s) {
-          if (r == 0) {                                                        // Q: this CTA's 128 rows, one request
-            if (lane == 0) tma_box2(slot, &maps.q, dk * 64, b * rows_seq + row0, fb_leader);
-          } else {      // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
-            const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
-            const bool one = consecutive(i0, nb);                              // nb = 4 (128 rows) or 2 (64 rows)
-            if (one) {
-              if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-            } else if (lane < nb) {
-              const uint32_t bx = sm.box[i0 + lane];
-              tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
-            }
+        if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
+          const int i0 = kb * (64 / kBoxRows);
+          if (consecutive(i0, 2)) {
+            if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+          } else if (lane < 4) {
+            const int i = lane >> 1, j = lane & 1;
+            const uint32_t bx = sm.box[i0 + i];
+            tma_box2(slot + j * 8192 + i * BOXB, &maps.src[bx >> 30][0], (part * 4 + (int)rank * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
           }
-        } else {
-          if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
-            const int i0 = kb * (64 / kBoxRows);
-            if (consecutive(i0, 2)) {
-              if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-            } else if (lane < 4) {
-              const int i = lane >> 1, j = lane & 1;
-              const uint32_t bx = sm.box[i0 + i];
-              tma_box2(slot + j * 8192 + i * BOXB, &maps.src[bx >> 30][0], (part * 4 + (int)rank * 2 + j) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
-            }
-          } else {                  // 128 keys x this CTA's 64 dims: key boxes 0..3
-            const int i0 = kb * (128 / kBoxRows);
-            if (consecutive(i0, 4)) {
-              if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][2], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
-            } else if (lane < 4) {
-              const uint32_t bx = sm.box[i0 + lane];
-              tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
-            }
+        } else {                  // 128 keys x this CTA's 64 dims: key boxes 0..3
+          const int i0 = kb * (128 / kBoxRows);
+          if (consecutive(i0, 4)) {
+            if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][2], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
+          } else if (lane < 4) {
+            const uint32_t bx = sm.box[i0 + lane];
+            tma_box2(slot + lane * BOXB, &maps.src[bx >> 30][0], (part * 2 + (int)rank) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader);
           }
         }
+        kb += NPROD;
+        while (kb >= nvb) { kb -= nvb; ++part; }
       }
-      if (++sl == NSX) { sl = 0; ++use; }
-      if (is_s) {
-        if (++r == per) { r = 0; if (++dk == 8) { dk = 0; per = 2; pc0 = 1; } }   // pass B: the Q stage, then piece 2
-      } else if (++kb == nvb) { kb = 0; ++part; }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -263,38 +285,30 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       // descriptors of a stage are the slot-0 descriptor plus a multiple of the slot size (the address field counts
       // 16-byte units and cannot overflow within the ring).
       const uint64_t dk0 = make_desc(ring, 16, 1024), dv0 = make_desc(ring, NQ == 2 ? 8192 : 16384, 1024);
-      int sl = 0; uint32_t ph = 0;                       // slot and parity of the next stage
-      auto wait_full = [&]() { if (!fail && !mbar_wait(&sm.full[sl], ph)) fail = 1; };
-      auto advance = [&]() { if (++sl == NSX) { sl = 0; ph ^= 1u; } };
-      // one pass over d for pieces [pc0, pc0 + np): per 64-wide slice the Q stage, then one K stage per piece
-      auto s_pass = [&](int pc0, int np) {
-        for (int dk = 0; dk < 8; ++dk) {
-          wait_full();
-          const int qsl = sl;
-          const uint64_t qd = dk0 + (uint64_t)(sl * (SLOTP >> 4));
-          advance();
-          for (int pc = pc0; pc < pc0 + np; ++pc) {
-            wait_full();
-            if (pc == 2 && dk == 0) need_ev(1);          // piece 2 reuses the S columns of piece 1
-            fence_after();
-            const uint64_t kd = dk0 + (uint64_t)(sl * (SLOTP >> 4));
-            const uint32_t scol = tm + (pc == 0 ? 0 : 256);
-            const uint32_t idesc = CL - pc * 256 >= 256 ? idesc_k256 : idesc_k128;
+      // S, piece after piece (the softmax of a piece runs while the tensor core works on the next one): per piece the
+      // eight slices of d, Q slice from its resident slot, K stage from the ring
+      int gk = 0;
+      for (int pc = 0; pc < npc; ++pc) {
+        if (pc == 2) need_ev(1);                         // piece 2 reuses the S columns of piece 1
+        const uint32_t scol = tm + (pc == 0 ? 0 : 256);
+        const uint32_t idesc = CL - pc * 256 >= 256 ? idesc_k256 : idesc_k128;
+        for (int dk = 0; dk < 8; ++dk, ++gk) {
+          const int sl = gk & (NKS - 1);
+          if (pc == 0 && !fail && !mbar_wait(&sm.fullQ[dk], 0)) fail = 1;
+          if (!fail && !mbar_wait(&sm.fullK[sl], (uint32_t)(gk >> 2) & 1u)) fail = 1;
+          fence_after();
+          const uint64_t qd = dk0 + (uint64_t)(dk * (SLOTP >> 4)), kd = dk0 + (uint64_t)((NQS + sl) * (SLOTP >> 4));
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) mma2_ss(scol, qd + 2 * ks, kd + 2 * ks, idesc, (dk | ks) != 0);
-            mma2_commit(&sm.empty[sl]);
-            advance();
-          }
-          mma2_commit(&sm.empty[qsl]);                  // the Q slice of this pass and dk is no longer needed
+          for (int ks = 0; ks < 4; ++ks) mma2_ss(scol, qd + 2 * ks, kd + 2 * ks, idesc, (dk | ks) != 0);
+          mma2_commit(&sm.emptyK[sl]);
         }
-        for (int pc = pc0; pc < pc0 + np; ++pc) mma2_commit(&sm.acc_ev[pc]);   // the S pieces of this pass are complete
-      };
-      s_pass(0, npA);
-      if (npc > 2) s_pass(2, 1);
+        mma2_commit(&sm.acc_ev[pc]);                     // S of the piece is complete
+      }
+      int sl = 0; uint32_t ph = 0;                       // slot and parity of the next V stage
       for (int part = 0; part < NQ; ++part) {
         need_ev(part == 0 ? npc - 1 : 3 + part - 1);     // all of P is in TMEM / the previous part of O has been read out
         for (int kb = 0; kb < nvb; ++kb) {
-          wait_full();
+          if (!fail && !mbar_wait(&sm.fullV[sl], ph)) fail = 1;
           fence_after();
           const uint64_t vd = dv0 + (uint64_t)(sl * (SLOTP >> 4));
           if (NQ == 2) {          // per CTA: 64 keys x 128 dims = two [64 x 64] tiles
@@ -304,8 +318,8 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) mma2_ts(tm + OCOL, tm + kb * 64 + ks * 8, vd + ks * (2048 >> 4), idesc_v, (kb | ks) != 0);
           }
-          mma2_commit(&sm.empty[sl]);
-          advance();
+          mma2_commit(&sm.emptyV[sl]);
+          if (++sl == NSX) { sl = 0; ph ^= 1u; }
         }
         mma2_commit(&sm.acc_ev[3 + part]);
       }
@@ -390,30 +404,27 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     };
     auto block_mine = [&](int pc) { return hh * 128 < min(256, CL - pc * 256); };
 
-    // Pass A: pieces 0 and 1 complete together and share one row maximum.  Pass B: piece 2 arrives later; the reference
-    // maximum is kept unless the piece exceeds it by more than RESCALE_GAP (weights up to 2^16 are harmless in
-    // bf16/fp32), else the P written so far and the sums are rescaled.
+    // The pieces arrive one after the other (the tensor core computes S of the next piece meanwhile).  The first piece sets
+    // the reference maximum of the row; a later piece keeps it unless it exceeds it by more than RESCALE_GAP (weights up
+    // to 2^16 are harmless in bf16/fp32), else the P written so far and the sums are rescaled.
     //
     // Where P lands: piece pc -> columns [128 pc, 128 pc + 128), the warps with hh = 0 write the lower 64 (keys of their S
     // block, the piece's first 128), the warps with hh = 1 the upper 64.  P of pieces 0 and 2 overlays the first half of the
     // piece's own S: a warp with hh = 0 writes behind its own reads (slab c -> P columns 16 c.. below the 32 c.. it has
     // read), but the warps with hh = 1 write over S slabs 2 and 3 of their hh = 0 neighbours, so those are read into
-    // registers first and a named barrier tells the neighbours.  P of piece 1 overlays S of piece 0, which every warp
-    // has finished with at the barrier between the pieces.
+    // registers first; a barrier of the eight warps follows.  P of piece 1 overlays S of piece 0, which every warp
+    // has finished with when it passes the barrier of piece 1's maximum exchange.
 #pragma unroll 1
-    for (int pass = 0; pass < (npc == 3 ? 2 : 1); ++pass) {
-      const int pcb = pass ? 2 : 0, pce = pass ? 3 : npA;
-#pragma unroll 1
-      for (int pc = pcb; pc < pce; ++pc)
-        if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
+    for (int pc = 0; pc < npc; ++pc) {
+      if (!fail && !mbar_wait(&sm.acc_ev[pc], 0)) fail = 1;
       fence_after();
+      const bool mine = block_mine(pc);
+      const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128, pcol = tlane + pc * 128 + hh * 64;
+      const uint32_t* vw = visw + pc * 4 * 256;
       float mx = -INFINITY;
+      if (mine) {
 #pragma unroll 1
-      for (int pc = pcb; pc < pce; ++pc) {
-        if (!block_mine(pc)) continue;
-        const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) mx = slab_max(scol + c * 32, visw[(pc * 4 + c) * 256], mx);
+        for (int c = 0; c < 4; ++c) mx = slab_max(scol + c * 32, vw[c * 256], mx);
       }
       sm.xch[hh][row] = mx;
       compute_sync();
@@ -423,35 +434,26 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         if (m_run != -INFINITY) factor = ex2(m_run - m_pass);
         m_run = m_pass;
       }
-      if (pass && __any_sync(0xffffffffu, factor != 1.f)) {  // warp-uniform: tcgen05.ld/st are warp-collective
+      if (pc && __any_sync(0xffffffffu, factor != 1.f)) {  // warp-uniform: tcgen05.ld/st are warp-collective
 #pragma unroll 1
-        for (int v = 0; v < 4; ++v) {
-          const uint32_t pcol = tlane + (v >> 1) * 128 + hh * 64 + (v & 1) * 32;
+        for (int v = 0; v < 2 * pc; ++v) {           // this thread's P columns of the earlier pieces
+          const uint32_t qcol = tlane + (v >> 1) * 128 + hh * 64 + (v & 1) * 32;
           uint32_t r[32];
-          tmem_ld32(pcol, r);
+          tmem_ld32(qcol, r);
 #pragma unroll
           for (int t = 0; t < 32; ++t) {
             float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r[t]));
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(f.x * factor, f.y * factor);
             r[t] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-          tmem_st16(pcol, r);
-          tmem_st16(pcol + 16, r + 16);
+          tmem_st16(qcol, r);
+          tmem_st16(qcol + 16, r + 16);
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) lp[c] *= factor;
       }
       const float moff = (m_run == -INFINITY) ? 0.f : m_run;
-#pragma unroll 1
-      for (int pc = pcb; pc < pce; ++pc) {
-        if (pc != pcb) {       // P of piece 1 overlays S of piece 0: every warp has read it for the last time
-          fence_before();
-          compute_sync();
-          fence_after();
-        }
-        const bool mine = block_mine(pc);
-        const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128, pcol = tlane + pc * 128 + hh * 64;
-        const uint32_t* vw = visw + pc * 4 * 256;
+      {
         uint32_t hold[64];
         if (hh == 0) {
           if (mine) {
@@ -462,11 +464,11 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
             tmem_regs_ready(hold + 32);
           }
           fence_before();
-          asm volatile("bar.arrive 2, 256;" ::: "memory");
-        } else {
-          asm volatile("bar.sync 2, 256;" ::: "memory");
-          fence_after();
         }
+        // all eight warps meet: the neighbours' slabs are in registers, and everybody has read the exchanged maxima (the
+        // exchange buffer is written again for the next piece)
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        if (hh) fence_after();
         if (mine) {
           const int nstream = hh == 0 ? 2 : 4;
 #pragma unroll 1
