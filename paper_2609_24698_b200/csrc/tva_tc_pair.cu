@@ -32,8 +32,9 @@ constexpr float RESCALE_GAP = 16.f;        // log2 units a later piece's row max
 
 constexpr int NSX = 12;                    // 16 KiB slots of the staging area; a 32 KiB area after it stages the output tiles
 constexpr int NQS = 8;                     // S phase: slots [0, 8) hold the Q slices (all of d, resident for every piece),
-constexpr int NKS = NSX - NQS;             //          slots [8, 12) are the ring of the K stages;
-                                           // V phase: all 12 slots form the ring of the V stages
+constexpr int NKS = NSX - NQS + 2;         //          slots [8, 14) are the ring of the K stages: the last two are the
+                                           //          output staging area, idle until the first part of O is read out;
+                                           // V phase: slots [0, 12) form the ring of the V stages
 
 struct Ctl {                               // control block at the start of dynamic shared memory
   uint64_t fullQ[NQS];                     // Q slice dk has arrived (used once)
@@ -211,7 +212,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       __syncwarp();
     };
     auto issue_k = [&](int gk) {
-      const int pc = gk >> 3, dk = gk & 7, sl = gk & (NKS - 1), use = gk >> 2;
+      const int pc = gk >> 3, dk = gk & 7, sl = gk % NKS, use = gk / NKS;
       const uint32_t slot = ring + (uint32_t)(NQS + sl) * SLOTP;
       const uint32_t fb_leader = map_to_rank(smem_u32(&sm.fullK[sl]), 0);
       const int bytes = min(256, CL - pc * 256) * 64;                        // bytes THIS CTA copies in the stage
@@ -230,7 +231,6 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       }
       __syncwarp();
     };
-    static_assert(NKS == 4, "issue_k derives the slot use from gk >> 2");
     if (pw == 0) {
       for (int i = 0; i < 4; ++i) { issue_q(2 * i); issue_q(2 * i + 1); issue_k(2 * i + 1); }
       for (int gk = 9; gk < NKST; gk += 2) issue_k(gk);
@@ -287,24 +287,25 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       const uint64_t dk0 = make_desc(ring, 16, 1024), dv0 = make_desc(ring, NQ == 2 ? 8192 : 16384, 1024);
       // S, piece after piece (the softmax of a piece runs while the tensor core works on the next one): per piece the
       // eight slices of d, Q slice from its resident slot, K stage from the ring
-      int gk = 0;
+      int sl = 0; uint32_t kph = 0;                      // slot and parity of the next K stage
       for (int pc = 0; pc < npc; ++pc) {
         if (pc == 2) need_ev(1);                         // piece 2 reuses the S columns of piece 1
         const uint32_t scol = tm + (pc == 0 ? 0 : 256);
         const uint32_t idesc = CL - pc * 256 >= 256 ? idesc_k256 : idesc_k128;
-        for (int dk = 0; dk < 8; ++dk, ++gk) {
-          const int sl = gk & (NKS - 1);
+        for (int dk = 0; dk < 8; ++dk) {
           if (pc == 0 && !fail && !mbar_wait(&sm.fullQ[dk], 0)) fail = 1;
-          if (!fail && !mbar_wait(&sm.fullK[sl], (uint32_t)(gk >> 2) & 1u)) fail = 1;
+          if (!fail && !mbar_wait(&sm.fullK[sl], kph)) fail = 1;
           fence_after();
           const uint64_t qd = dk0 + (uint64_t)(dk * (SLOTP >> 4)), kd = dk0 + (uint64_t)((NQS + sl) * (SLOTP >> 4));
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) mma2_ss(scol, qd + 2 * ks, kd + 2 * ks, idesc, (dk | ks) != 0);
           mma2_commit(&sm.emptyK[sl]);
+          if (++sl == NKS) { sl = 0; kph ^= 1u; }
         }
         mma2_commit(&sm.acc_ev[pc]);                     // S of the piece is complete
       }
-      int sl = 0; uint32_t ph = 0;                       // slot and parity of the next V stage
+      sl = 0;
+      uint32_t ph = 0;                                   // slot and parity of the next V stage
       for (int part = 0; part < NQ; ++part) {
         need_ev(part == 0 ? npc - 1 : 3 + part - 1);     // all of P is in TMEM / the previous part of O has been read out
         for (int kb = 0; kb < nvb; ++kb) {
@@ -338,25 +339,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     // The softmax code works on slabs of 32 keys in short loops: the kernel passes through it once per piece, so long
     // unrolled code would be fetched cold every time.
     //
-    // Visibility of every slab for this lane's row, 32 keys per word (bit t = key t of the slab).  It does not depend on
-    // S: the words are computed while the S products run and parked in the (still unused) output staging area.
-    uint32_t* visw = reinterpret_cast<uint32_t*>(smem_raw + CTLB + NSX * SLOTP) + (warp - 2) * 32 + lane;   // [piece * 4 + slab][256 threads]
-    {
-      // lanes of a warp may belong to different nodes when H < 32: one ballot per node bit present in the warp
-      const uint32_t lo = __shfl_sync(0xffffffffu, mybit, 0), hi = __shfl_sync(0xffffffffu, mybit, 31);
-#pragma unroll 1
-      for (int i = 0; i < 4 * npc; ++i) {
-        const int pc = i >> 2, c = i & 3;
-        const bool mine = hh * 128 < min(256, CL - pc * 256);
-        const uint32_t mk = mine ? sm.kmask[pc * 256 + hh * 128 + c * 32 + lane] : 0u;
-        uint32_t v = __ballot_sync(0xffffffffu, mk & mybit);
-        if (lo != hi) {
-          v = 0;
-          for (uint32_t bit = lo; bit <= hi; bit <<= 1) { const uint32_t w = __ballot_sync(0xffffffffu, mk & bit); if (bit == mybit) v = w; }
-        }
-        visw[i * 256] = v;
-      }
-    }
+    // Visibility of a slab for this warp's rows, 32 keys per word (bit t = key t of the slab).  The 32 rows of a warp
+    // belong to one node (H >= 32 on this path), so one ballot over the keys' node masks gives the word.
+    auto slab_vis = [&](int pc, int c) { return __ballot_sync(0xffffffffu, sm.kmask[pc * 256 + hh * 128 + c * 32 + lane] & mybit); };
     // masked maximum of one slab of S (fp32 columns [col, col + 32))
     auto slab_max = [&](uint32_t col, uint32_t vis, float mx) {
       uint32_t sv[32];
@@ -420,11 +405,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       fence_after();
       const bool mine = block_mine(pc);
       const uint32_t scol = tlane + (pc == 0 ? 0 : 256) + hh * 128, pcol = tlane + pc * 128 + hh * 64;
-      const uint32_t* vw = visw + pc * 4 * 256;
       float mx = -INFINITY;
       if (mine) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) mx = slab_max(scol + c * 32, vw[c * 256], mx);
+        for (int c = 0; c < 4; ++c) mx = slab_max(scol + c * 32, slab_vis(pc, c), mx);
       }
       sm.xch[hh][row] = mx;
       compute_sync();
@@ -475,11 +459,11 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
           for (int c = 0; c < nstream; ++c) {
             uint32_t sv[32];
             tmem_ld32(scol + c * 32, sv);
-            slab_exp(sv, vw[c * 256], moff, pcol + c * 16);
+            slab_exp(sv, slab_vis(pc, c), moff, pcol + c * 16);
           }
           if (hh == 0) {
-            slab_exp(hold, vw[2 * 256], moff, pcol + 32);
-            slab_exp(hold + 32, vw[3 * 256], moff, pcol + 48);
+            slab_exp(hold, slab_vis(pc, 2), moff, pcol + 32);
+            slab_exp(hold + 32, slab_vis(pc, 3), moff, pcol + 48);
           }
         }
         // the MMA warp waits for the last piece only (and, with three pieces, for piece 1 before it overwrites that
