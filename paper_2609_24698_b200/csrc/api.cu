@@ -36,6 +36,7 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   const int64_t pref = s.max_L / s.m_csa;
   p.cand_cap = (int32_t)(pref + s.D);
   p.need_scores = p.cand_cap > s.topk;
+  p.idx_fused = p.need_scores && p.cand_cap <= kIdxFusedMax && s.HI <= 8 && (size_t)s.HI * s.di * sizeof(float) <= 32768;
   const int64_t ksel = p.cand_cap < s.topk ? p.cand_cap : s.topk;
   p.keys_max = (int32_t)(ksel + s.max_L / s.m_hca + s.D + s.window + s.D);
   const int hgroups = (s.H + 15) / 16;

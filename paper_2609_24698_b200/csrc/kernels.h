@@ -34,6 +34,8 @@ struct AarLayers {
 struct TvaPlan {
   int32_t cand_cap;      // max CSA candidates per node (committed + in-tree)
   int32_t need_scores;   // cand_cap > topk: some node may have to rank its candidates
+  int32_t idx_fused;     // ranked nodes score their committed entries inside topk_kernel (short candidate lists: the
+                         // separate scoring kernel, which exits at once for every sequence that needs no ranking, is not launched)
   int32_t keys_max;      // max keys one node can attend to
   int32_t ks;            // keys per split (CUDA-core path)
   int32_t nsplit;        // max splits per node
@@ -54,6 +56,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
 
+constexpr int kIdxFusedMax = 2048;   // candidate capacity up to which topk_kernel computes the indexer scores itself
 constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs are padded to a multiple of it
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);

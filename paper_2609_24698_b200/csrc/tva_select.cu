@@ -157,6 +157,40 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       if (lane == 0) extra[i] = tot;
     }
   }
+  if (pl.idx_fused) {
+    // short candidate lists: the committed entries are scored here as well (same formula as idx_score_kernel: thread per
+    // entry, the node's indexer queries in shared memory), into the score array the radix passes read
+    extern __shared__ float iq_sm[];                  // [HI][di]
+    const int HI = s.HI, di = s.di;
+    constexpr int V = Vec<T>::N;
+    const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * HI * di;
+    for (int i = threadIdx.x; i < HI * di; i += blockDim.x) iq_sm[i] = to_f(iq[i]);
+    __syncthreads();
+    const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
+    float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+    for (int e = threadIdx.x; e < n_csa; e += blockDim.x) {
+      float acc[8];
+#pragma unroll
+      for (int h = 0; h < 8; ++h) acc[h] = 0.f;
+      for (int cidx = 0; cidx < di / V; ++cidx) {
+        float kk[V];
+        ld16(ik0 + (size_t)e * di + cidx * V, kk);
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          if (h < HI) {
+            const float* qv = iq_sm + h * di + cidx * V;
+#pragma unroll
+            for (int t = 0; t < V; ++t) acc[h] = fmaf(qv[t], kk[t], acc[h]);
+          }
+        }
+      }
+      float tot = 0.f;
+#pragma unroll
+      for (int h = 0; h < 8; ++h)
+        if (h < HI) tot = fmaf(nd.iw[((size_t)b * D + n) * HI + h], fmaxf(acc[h], 0.f), tot);
+      sw[e] = tot;
+    }
+  }
   if (threadIdx.x == 0) { sh_prefix = 0; sh_remaining = k; }
   __syncthreads();
   const float* scores = reinterpret_cast<const float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
@@ -216,7 +250,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
 int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st) {
   const bool bf = s.dtype == TSV_BF16;
-  if (p.need_scores) {
+  if (p.need_scores && !p.idx_fused) {
     const int pref_cap = (int)(s.max_L / s.m_csa);
     dim3 grid((pref_cap + 255) / 256, s.B, s.D <= 8 ? s.D : 8);        // z: slabs of nodes, so a ranked sequence is scored by many CTAs
     const size_t sm = (size_t)32 * s.di * sizeof(float);
@@ -236,8 +270,9 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   dim3 g2(s.D, s.B);
   TSV_PREP(topk_kernel<bf16>);
   TSV_PREP(topk_kernel<float>);
-  if (bf) topk_kernel<bf16><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
-  else topk_kernel<float><<<g2, 256, 0, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
+  const size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;   // the node's indexer queries
+  if (bf) topk_kernel<bf16><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
+  else topk_kernel<float><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }
