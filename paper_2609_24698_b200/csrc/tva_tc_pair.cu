@@ -5,13 +5,13 @@
 // 128 of them in its own tensor memory.  The two SMs execute every MMA together (M = 256): the B operand
 // -- the staged key rows -- is split between the two shared memories, so each SM fetches only HALF of
 // the K tile (S = Q K^T: half of the keys) and half of the V tile (O = P K: half of the columns of d).
-// That halves the bytes each SM pulls from L2, which is what bounds this kernel.
-//   warp 0     producer: TMA boxes (cp.async.bulk.tensor, 128-byte swizzle) into a ring of 16 KiB slots; the
-//              copies of BOTH CTAs complete on the mbarrier of the leader (rank 0) CTA
-//   warp 1     MMA issuer (leader CTA only): tcgen05.mma.cta_group::2, slot release and accumulator
-//              events by tcgen05.commit multicast to both CTAs
-//   warps 2-9  softmax on the CTA's own S rows (TMEM), P written back to TMEM, epilogue of O through
-//              swizzled shared-memory tiles and TMA stores; events to the leader's MMA warp by remote arrive
+// That halves the bytes each SM pulls from L2.
+//   warps 0, 10  producers: TMA boxes (cp.async.bulk.tensor, 128-byte swizzle) into 16 KiB slots; the copies of BOTH
+//                CTAs complete on the mbarriers of the leader (rank 0) CTA
+//   warp 1       MMA issuer (leader CTA only): tcgen05.mma.cta_group::2, slot release and accumulator
+//                events by tcgen05.commit multicast to both CTAs
+//   warps 2-9    softmax on the CTA's own S rows (TMEM), P written back to TMEM, epilogue of O through
+//                swizzled shared-memory tiles and TMA stores; events to the leader's MMA warp by remote arrive
 // Stage stream, TMEM column plan, running-max rule and chunking are those described at the kernel.
 #include <cuda.h>
 #include <stdio.h>
@@ -25,7 +25,7 @@ namespace pair {
 
 using namespace tc;
 
-constexpr int NPROD = 2;                    // producer warps: warp 0 and warps 10.., stage g belongs to producer g % NPROD
+constexpr int NPROD = 2;                    // producer warps: warp 0 and warp 10
 constexpr int TTHREADS = 32 * (10 + NPROD - 1);   // warp 1: MMA issuer; warps 2-9: softmax and epilogue
 constexpr int BOXB = kBoxRows * 128;       // bytes of one box: kBoxRows rows x 128 bytes
 constexpr float RESCALE_GAP = 16.f;        // log2 units a later piece's row max may exceed the running reference
@@ -109,10 +109,10 @@ constexpr uint32_t OOB_BOX = 0x3FFFFF00u;   // map 0, a row beyond every tensor:
 }  // namespace pair
 
 // Per CTA (rank r of the pair), for a chunk of CL keys (pieces of 256 keys, the last may hold 128):
-//   S stages: pass A = pieces 0 and 1, pass B = piece 2; per pass and 64-wide slice dk of d:
-//       [Q: this CTA's 128 rows x 64 dims]  then per piece  [K: this CTA's half of the piece's keys x 64 dims]
-//   V stages: CL <= 512: per half of d, per 64 keys:  [64 keys x this CTA's 128 of the half's 256 dims]
-//             else       per quarter of d, per 128 keys: [128 keys x this CTA's 64 of the quarter's 128 dims]
+//   Q slices:  per 64-wide slice dk of d  [this CTA's 128 rows x 64 dims], fetched once, resident for all pieces
+//   K stages:  piece after piece, per slice dk  [this CTA's half of the piece's keys x 64 dims]
+//   V stages (after the last S product): CL <= 512: per half of d, per 64 keys:  [64 keys x this CTA's 128 of the half's 256 dims]
+//                                        else       per quarter of d, per 128 keys: [128 keys x this CTA's 64 of the quarter's 128 dims]
 __global__ void __launch_bounds__(pair::TTHREADS, 1)
 tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s,
                     const TvaPlan pl, void* __restrict__ out_, char* __restrict__ ws, int32_t* __restrict__ status) {
