@@ -49,6 +49,36 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   if (threadIdx.x == 41) row0_sm[1] = c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
   const int64_t csa_row0 = row0_sm[0], hca_row0 = row0_sm[1];
+  if (blockIdx.x >= (unsigned)pl.tc_nt) {
+    // The extra CTA of the sequence (grid x = tiles + 1): rows that are small and scattered (few HCA entries, tree nodes,
+    // entries closed inside the tree) are packed into one contiguous per-sequence buffer so that TMA boxes can fetch
+    // them.  Kept off the tile CTAs: the copy is a chain of its own (addresses, loads, stores).
+    if (tm.status || !pl.tc_tma) return;
+    const size_t rowb = (size_t)s.d * 2;
+    const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
+    int ncd = 0, nhd = 0;
+    for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
+    const int n_misc = nh_in + tm.nn + ncd + nhd;
+    uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
+    const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows, cpr = (int)(rowb / 16);
+    for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
+      const int r = i / cpr, cc = i % cpr;
+      const char* src = nullptr;
+      if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)hca_row0 + r) * rowb;
+      else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
+      else if (r < n_misc) {
+        int ord = r - nh_in - tm.nn;
+        const bool isc = ord < ncd;
+        if (!isc) ord -= ncd;
+        const uint8_t* dn = isc ? cdone : hdone;
+        int a = 0;
+        for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
+        src = (const char*)(isc ? sc.new_csa_kv : sc.new_hca_kv) + ((size_t)b * D + a) * rowb;
+      }
+      dst[i] = src ? reinterpret_cast<const uint4*>(src)[cc] : make_uint4(0, 0, 0, 0);
+    }
+    return;
+  }
   if (threadIdx.x == 0) {
     int dn = 1;
     for (int nl = 0; nl < npt; ++nl) {
@@ -89,32 +119,11 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     return false;
   };
   if (pl.tc_tma) {
-    // rows that are small and scattered (few HCA entries, tree nodes, entries closed inside the tree) are packed
-    // into one contiguous per-sequence buffer so that TMA boxes can fetch them: written by the CTA of tile 0
+    // the packed per-sequence rows (written by the sequence's extra CTA): few HCA entries, tree nodes, entries closed in the tree
     const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
     int ncd = 0, nhd = 0;
     for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
     const int n_misc = nh_in + tm.nn + ncd + nhd;
-    if (tile == 0) {
-      uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
-      const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows, cpr = (int)(rowb / 16);
-      for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
-        const int r = i / cpr, cc = i % cpr;
-        const char* src = nullptr;
-        if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)hca_row0 + r) * rowb;
-        else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
-        else if (r < n_misc) {
-          int ord = r - nh_in - tm.nn;
-          const bool isc = ord < ncd;
-          if (!isc) ord -= ncd;
-          const uint8_t* dn = isc ? cdone : hdone;
-          int a = 0;
-          for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
-          src = (const char*)(isc ? sc.new_csa_kv : sc.new_hca_kv) + ((size_t)b * D + a) * rowb;
-        }
-        dst[i] = src ? reinterpret_cast<const uint4*>(src)[cc] : make_uint4(0, 0, 0, 0);
-      }
-    }
     // Ranked nodes still take the contiguous-run path while the run is at most twice the selection size: all committed
     // entries are staged and the unselected ones are masked per node.
     if (dense || n_csa <= 2 * s.topk) {
@@ -222,7 +231,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
   __shared__ int is_last;
-  if (threadIdx.x < 2)                                // finished-chunk counters of the tile's two 128-row halves
+  if (threadIdx.x < 2 && blockIdx.x < (unsigned)pl.tc_nt)   // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[((size_t)blockIdx.y * pl.tc_nt + blockIdx.x) * 2 + threadIdx.x] = 0;
   tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
   __threadfence();
@@ -616,7 +625,7 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
   TSV_PREP(tc_plan_kernel);
   TSV_PREP(tc_attn_kernel);
   TSV_PREP(tc_combine_kernel);
-  tc_plan_kernel<<<dim3(p.tc_nt, s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);
+  tc_plan_kernel<<<dim3(p.tc_nt + (p.tc_tma ? 1 : 0), s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);   // x: tiles (+ the packing CTA)
   count_launch();
   if (p.tc_tma) {
     const int r = launch_tva_tc_pair(s, p, c, nd, out, ws, status, st);
