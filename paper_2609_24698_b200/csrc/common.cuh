@@ -89,7 +89,7 @@ __device__ inline void build_tree_meta(TreeMeta& tm, const tsv_shape& s, int32_t
 }
 
 // Cooperative front end of build_tree_meta: the first threads of the CTA fetch the parent array and the per-sequence
-// scalars in parallel (one memory latency instead of a chain of dependent loads), then thread 0 derives the tree facts.
+// scalars in parallel (one memory latency instead of a chain of dependent loads), then warp 0 derives the tree facts.
 // Must be called by all threads of the CTA (contains two barriers); needs blockDim.x >= 64.
 struct TreeStage { int32_t parent[TSV_MAX_D]; int32_t scal[4]; };
 __device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, const tsv_shape& s, const int32_t* L_b, const int32_t* parent_b,
@@ -101,7 +101,32 @@ __device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, cons
   if (t == 34 && csa_cap_b) st.scal[2] = *csa_cap_b;
   if (t == 35 && hca_cap_b) st.scal[3] = *hca_cap_b;
   __syncthreads();
-  if (t == 0) build_tree_meta(tm, s, st.scal[0], st.parent, st.scal[1], csa_cap_b ? &st.scal[2] : nullptr, hca_cap_b ? &st.scal[3] : nullptr);
+  if (t < 32) {
+    // Same facts as build_tree_meta, lane n deriving node n: ancestors by walking up the staged parent array (a valid
+    // array has parent < node, so the walk ends within D steps).  With any invalid entry the sequence is flagged and
+    // every kernel skips it, so the facts of the other nodes need not match the serial routine then.
+    int L = st.scal[0], nn = st.scal[1], stt = 0;
+    if (nn < 1 || nn > s.D) { stt |= TSV_ST_NODES; nn = 0; }
+    if (L < 0 || (int64_t)L + s.D > s.max_L) { stt |= TSV_ST_LENGTH; L = 0; }
+    const int n = t;
+    const int p = (n < nn) ? st.parent[n] : -1;
+    const bool bad = (n < nn) && (n == 0 ? p != -1 : (p < 0 || p >= n));
+    if (__any_sync(0xffffffffu, bad)) stt |= TSV_ST_PARENT;
+    uint32_t anc = 0;
+    int depth = 0;
+    if (n < nn && !bad) {
+      anc = 1u << n;
+      int cur = p;
+      for (int it = 0; it < TSV_MAX_D && cur >= 0 && cur < n; ++it) { anc |= 1u << cur; ++depth; cur = st.parent[cur]; }
+    }
+    tm.depth[n] = depth; tm.parent[n] = (n < nn && !bad && n > 0) ? p : -1; tm.anc[n] = anc;
+    if (t == 0) {
+      if (csa_cap_b && (L + s.D) / s.m_csa > st.scal[2]) stt |= TSV_ST_CSA_CAP;
+      if (hca_cap_b && (L + s.D) / s.m_hca > st.scal[3]) stt |= TSV_ST_HCA_CAP;
+      tm.L = L; tm.nn = nn; tm.status = stt;
+      tm.n_csa = L / s.m_csa; tm.n_hca = L / s.m_hca;
+    }
+  }
   __syncthreads();
 }
 

@@ -61,8 +61,10 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
     const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows, cpr = (int)(rowb / 16);
-    for (int i = threadIdx.x; i < rows_out * cpr; i += blockDim.x) {
-      const int r = i / cpr, cc = i % cpr;
+    // warp per row, eight rows of a warp in flight: the source of a row is worked out once, all loads of the batch are
+    // issued before the first store
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    auto row_src = [&](int r) -> const uint4* {
       const char* src = nullptr;
       if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)hca_row0 + r) * rowb;
       else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
@@ -75,22 +77,43 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
         src = (const char*)(isc ? sc.new_csa_kv : sc.new_hca_kv) + ((size_t)b * D + a) * rowb;
       }
-      dst[i] = src ? reinterpret_cast<const uint4*>(src)[cc] : make_uint4(0, 0, 0, 0);
+      return reinterpret_cast<const uint4*>(src);
+    };
+    if (cpr == 64) {                                   // d = 512 in bf16: two 16-byte pieces of a row per lane
+      for (int r0 = w; r0 < rows_out; r0 += 8 * nw) {
+        uint4 v[8][2];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int r = r0 + k * nw;
+          const uint4* src = r < rows_out ? row_src(r) : nullptr;
+          v[k][0] = src ? __ldg(src + lane) : make_uint4(0, 0, 0, 0);
+          v[k][1] = src ? __ldg(src + 32 + lane) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int r = r0 + k * nw;
+          if (r < rows_out) { dst[(size_t)r * 64 + lane] = v[k][0]; dst[(size_t)r * 64 + 32 + lane] = v[k][1]; }
+        }
+      }
+    } else {
+      for (int r = w; r < rows_out; r += nw) {
+        const uint4* src = row_src(r);
+        for (int cc = lane; cc < cpr; cc += 32) dst[(size_t)r * cpr + cc] = src ? src[cc] : make_uint4(0, 0, 0, 0);
+      }
     }
     return;
   }
-  if (threadIdx.x == 0) {
-    int dn = 1;
-    for (int nl = 0; nl < npt; ++nl) {
-      const int n = n0 + nl;
-      int extra = 0;
-      if (n < tm.nn)
-        for (int j = 0; j < n; ++j) if (((tm.anc[n] >> j) & 1u) && cdone[j]) ++extra;
-      n_cand[nl] = tm.n_csa + extra;
-      if (n < tm.nn && n_cand[nl] > s.topk) dn = 0;
-      win_lo[nl] = max(0, tm.L + tm.depth[n < tm.nn ? n : 0] - s.window + 1);
+  if (threadIdx.x < 32) {                              // lane nl: candidates and window start of node n0 + nl
+    const int lane = threadIdx.x, n = n0 + lane;
+    const uint32_t cmaskbits = __ballot_sync(0xffffffffu, lane < D && cdone[lane]);   // nodes that close a CSA block
+    const bool real = lane < npt && n < tm.nn;
+    const int nc = tm.n_csa + (real ? __popc(tm.anc[n] & ((1u << n) - 1u) & cmaskbits) : 0);   // + blocks closed at strict ancestors
+    if (lane < npt) {
+      n_cand[lane] = nc;
+      win_lo[lane] = max(0, tm.L + tm.depth[real ? n : 0] - s.window + 1);
     }
-    dense = dn;
+    const uint32_t over = __ballot_sync(0xffffffffu, real && nc > s.topk);
+    if (lane == 0) dense = over == 0;
   }
   __syncthreads();
   int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
