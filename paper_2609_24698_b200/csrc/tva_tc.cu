@@ -151,41 +151,48 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     // entries are staged and the unselected ones are masked per node.
     if (dense || n_csa <= 2 * s.topk) {
       int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
-      int kb = 0;
-      auto emit = [&](int map, int64_t start, int count, int seg) {
-        const int nb = (count + kBoxRows - 1) / kBoxRows;
-        for (int i = threadIdx.x; i < nb; i += blockDim.x) box[kb / kBoxRows + i] = make_int2(map, (int)(start + kBoxRows * i));
-        for (int i = threadIdx.x; i < nb * kBoxRows; i += blockDim.x) {
-          uint32_t m = 0;
-          if (i < count) {
-            if (seg == 0) m = dense ? validbits : cmask[i];
-            else if (seg == 1) m = validbits;
-            else if (seg == 2) {
-              const int pos = tm.L - 1 - ((tm.L - 1 - i) % s.window);
-              for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
-            } else if (i < nh_in) m = validbits;
-            else if (i < nh_in + tm.nn) {
-              const int j = i - nh_in;
-              for (int nl = 0; nl < nvalid; ++nl) if ((tm.anc[n0 + nl] >> j) & 1u) m |= 1u << nl;
-            } else {
-              int ord = i - nh_in - tm.nn;
-              const bool isc = ord < ncd;
-              if (!isc) ord -= ncd;
-              const uint8_t* dn = isc ? cdone : hdone;
-              int a = 0;
-              for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
-              for (int nl = 0; nl < nvalid; ++nl)
-                if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && (!isc || newc_selected(nl, a))) m |= 1u << nl;
-            }
+      // four runs, each padded to whole boxes: committed CSA entries, HCA entries (when too many for the packed rows),
+      // the window ring, the packed rows.  One pass over all keys: a thread finds the run of its key by comparison, so
+      // the runs' (short, latency-bound) mask computations overlap instead of following each other.
+      const int cnt[4] = {n_csa, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, min(tm.L, s.window), n_misc};
+      const int64_t start[4] = {csa_row0, hca_row0, (int64_t)b * s.window, (int64_t)b * pl.tc_misc_rows};
+      int k0[5];                                       // first key of each run
+      k0[0] = 0;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) k0[g + 1] = k0[g] + (cnt[g] + kBoxRows - 1) / kBoxRows * kBoxRows;
+      const int kb = k0[4];
+      for (int bi = threadIdx.x; bi < kb / kBoxRows; bi += blockDim.x) {
+        const int k = bi * kBoxRows;
+        const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
+        box[bi] = make_int2(g, (int)(start[g] + (k - k0[g])));
+      }
+      for (int k = threadIdx.x; k < kb; k += blockDim.x) {
+        const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
+        const int i = k - k0[g];
+        uint32_t m = 0;
+        if (i < cnt[g]) {
+          if (g == 0) m = dense ? validbits : cmask[i];
+          else if (g == 1) m = validbits;
+          else if (g == 2) {
+            const int pos = tm.L - 1 - ((tm.L - 1 - i) % s.window);
+            for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
+          } else if (i < nh_in) m = validbits;
+          else if (i < nh_in + tm.nn) {
+            const int j = i - nh_in;
+            for (int nl = 0; nl < nvalid; ++nl) if ((tm.anc[n0 + nl] >> j) & 1u) m |= 1u << nl;
+          } else {
+            int ord = i - nh_in - tm.nn;
+            const bool isc = ord < ncd;
+            if (!isc) ord -= ncd;
+            const uint8_t* dn = isc ? cdone : hdone;
+            int a = 0;
+            for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
+            for (int nl = 0; nl < nvalid; ++nl)
+              if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && (!isc || newc_selected(nl, a))) m |= 1u << nl;
           }
-          kmask[kb + i] = (uint8_t)m;
         }
-        kb += nb * kBoxRows;
-      };
-      emit(0, csa_row0, n_csa, 0);
-      if (tm.n_hca > kHcaMiscMax) emit(1, hca_row0, tm.n_hca, 1);
-      emit(2, (int64_t)b * s.window, min(tm.L, s.window), 2);
-      emit(3, (int64_t)b * pl.tc_misc_rows, n_misc, 3);
+        kmask[k] = (uint8_t)m;
+      }
       if (threadIdx.x == 0) { *nkeys = kb; *mode = 1; }
       return;
     }
