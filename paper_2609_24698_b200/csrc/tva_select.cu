@@ -104,6 +104,16 @@ __device__ __forceinline__ uint32_t order_key(float f) {       // larger float -
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// 16 raw bytes of storage elements widened to fp32 (the tag argument selects the storage type)
+__device__ __forceinline__ void unpack16(const uint4& v, float* o, const float*) {
+  o[0] = __uint_as_float(v.x); o[1] = __uint_as_float(v.y); o[2] = __uint_as_float(v.z); o[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void unpack16(const uint4& v, float* o, const bf16*) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(w[i] << 16); o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
@@ -172,15 +182,26 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       float acc[8];
 #pragma unroll
       for (int h = 0; h < 8; ++h) acc[h] = 0.f;
-      for (int cidx = 0; cidx < di / V; ++cidx) {
-        float kk[V];
-        ld16(ik0 + (size_t)e * di + cidx * V, kk);
+      // the key row is fetched 8 x 16 bytes at a time, all loads of a batch in flight before the first use (few CTAs
+      // rank, so a thread cannot count on other warps to hide its load latency)
+      for (int c0 = 0; c0 < di / V; c0 += 8) {
+        uint4 raw[8];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          if (h < HI) {
-            const float* qv = iq_sm + h * di + cidx * V;
+        for (int u = 0; u < 8; ++u)
+          raw[u] = (c0 + u < di / V) ? __ldg(reinterpret_cast<const uint4*>(ik0 + (size_t)e * di + (c0 + u) * V)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int t = 0; t < V; ++t) acc[h] = fmaf(qv[t], kk[t], acc[h]);
+        for (int u = 0; u < 8; ++u) {
+          if (c0 + u < di / V) {
+            float kk[V];
+            unpack16(raw[u], kk, (const T*)nullptr);
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+              if (h < HI) {
+                const float* qv = iq_sm + h * di + (c0 + u) * V;
+#pragma unroll
+                for (int t = 0; t < V; ++t) acc[h] = fmaf(qv[t], kk[t], acc[h]);
+              }
+            }
           }
         }
       }
@@ -194,16 +215,36 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   if (threadIdx.x == 0) { sh_prefix = 0; sh_remaining = k; }
   __syncthreads();
   const float* scores = reinterpret_cast<const float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
-  auto key_of = [&](int i) { return order_key(i < n_csa ? scores[i] : extra[i - n_csa]); };
+  // order-preserving keys; lists of up to 9 x 256 candidates keep them in registers for the five passes below (candidate
+  // i = threadIdx.x + 256 j is key j of its thread), longer lists read the scores again
+  constexpr int KREG = 9;
+  const bool in_regs = n_cand <= KREG * 256;
+  uint32_t kreg[KREG];
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < KREG; ++j) {
+      const int i = threadIdx.x + 256 * j;
+      kreg[j] = i < n_cand ? order_key(i < n_csa ? __ldcg(scores + i) : extra[i - n_csa]) : 0u;
+    }
+  }
+  auto key_of = [&](int i) { return order_key(i < n_csa ? __ldcg(scores + i) : extra[i - n_csa]); };
   uint32_t mask = 0;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     hist[threadIdx.x] = 0;
     __syncthreads();
     const uint32_t prefix = sh_prefix;
-    for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
-      const uint32_t key = key_of(i);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    if (in_regs) {
+#pragma unroll
+      for (int j = 0; j < KREG; ++j) {
+        const uint32_t key = kreg[j];
+        if (threadIdx.x + 256 * j < n_cand && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      }
+    } else {
+      for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
+        const uint32_t key = key_of(i);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      }
     }
     __syncthreads();
     if (threadIdx.x < 32) {                           // warp 0 finds the bin holding the rem-th largest key: lane l owns bins 255-8l .. 248-8l
@@ -229,10 +270,15 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   const uint32_t thr = sh_prefix;       // key of the k-th largest score
   const int r = sh_remaining;           // how many of the scores equal to it are taken (lowest indices)
   int eq_base = 0, out_base = 0;
-  for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
+  for (int i0 = 0, j0 = 0; i0 < n_cand; i0 += blockDim.x, ++j0) {
     const int i = i0 + threadIdx.x;
     uint32_t key = 0;
-    if (i < n_cand) key = key_of(i);
+    if (i < n_cand) {
+      if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < KREG; ++j) if (j == j0) key = kreg[j];
+      } else key = key_of(i);
+    }
     const int eq = (i < n_cand) && key == thr, gt = (i < n_cand) && key > thr;
     int tot_eq, tot_take;
     const int eq_rank = eq_base + block_excl_scan_256(eq, wsum, tot_eq);
