@@ -178,6 +178,49 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     __syncthreads();
     const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
     float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+    if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
+      // Rows of 256 bytes (the benchmark's indexer width): eight lanes share an entry, each holding its 32-byte slice of
+      // the node's queries in registers for all entries; four entries of a group are in flight (few CTAs rank and global
+      // latency is long, so the number of dependent load rounds per thread is what counts: 4 here), and the per-head
+      // dot products are completed by three shuffles.
+      constexpr int EL = 2 * V;                        // row elements per lane
+      const int grp = threadIdx.x >> 3, gl = threadIdx.x & 7;
+      float q[4][EL], iwreg[4];
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        iwreg[h] = h < HI ? nd.iw[((size_t)b * D + n) * HI + h] : 0.f;
+#pragma unroll
+        for (int j = 0; j < EL; ++j) q[h][j] = h < HI ? iq_sm[h * di + gl * EL + j] : 0.f;
+      }
+      for (int base = 0; base < n_csa; base += 128) {  // uniform trip count: the shuffles below need the whole warp
+        uint4 raw[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = base + grp + 32 * u;
+          const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)(e < n_csa ? e : 0) * di) + gl * 2;
+          raw[u][0] = __ldg(rowp); raw[u][1] = __ldg(rowp + 1);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          float kk[EL];
+          unpack16(raw[u][0], kk, (const T*)nullptr);
+          unpack16(raw[u][1], kk + V, (const T*)nullptr);
+          float tot = 0.f;
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            float pp = 0.f;
+#pragma unroll
+            for (int j = 0; j < EL; ++j) pp = fmaf(q[h][j], kk[j], pp);
+            pp += __shfl_xor_sync(0xffffffffu, pp, 1);
+            pp += __shfl_xor_sync(0xffffffffu, pp, 2);
+            pp += __shfl_xor_sync(0xffffffffu, pp, 4);
+            tot = fmaf(iwreg[h], fmaxf(pp, 0.f), tot);
+          }
+          const int e = base + grp + 32 * u;
+          if (gl == 0 && e < n_csa) sw[e] = tot;
+        }
+      }
+    } else
     for (int e = threadIdx.x; e < n_csa; e += blockDim.x) {
       float acc[8];
 #pragma unroll
