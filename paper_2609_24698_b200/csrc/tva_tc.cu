@@ -122,24 +122,45 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   const uint32_t validbits = (1u << nvalid) - 1u;
   const int n_csa = tm.n_csa;
   const size_t rowb = (size_t)s.d * 2;
+  // Ranked nodes: node bits per committed CSA entry (cmask) and, per node, which blocks closed inside the tree are in
+  // its selection (bit = block index - n_csa).  One pass over the selections of all the tile's nodes: the loads of a
+  // batch are issued together (the tile CTA of a ranked sequence is on the critical path of the whole stage).
+  __shared__ uint32_t newc_bits[8];
   if (!dense) {
-    for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] = 0;
+    uint32_t* cm32 = reinterpret_cast<uint32_t*>(cmask);
+    for (int i = threadIdx.x; i < (n_csa + 3) / 4; i += blockDim.x) cm32[i] = 0;
+    if (threadIdx.x < 8) newc_bits[threadIdx.x] = 0;
     __syncthreads();
-    for (int nl = 0; nl < nvalid; ++nl) {
-      const int n = n0 + nl, cnt = selcnt[n];
-      if (n_cand[nl] <= s.topk) { for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)(1u << nl); }
-      else for (int j = threadIdx.x; j < cnt; j += blockDim.x) { const int idx = sel[(size_t)n * s.topk + j]; if (idx < n_csa) cmask[idx] |= (uint8_t)(1u << nl); }
+    uint32_t allbits = 0;                              // nodes that take every committed entry
+    for (int nl = 0; nl < nvalid; ++nl) if (n_cand[nl] <= s.topk) allbits |= 1u << nl;
+    const int total = nvalid * s.topk;
+    for (int x0 = 0; x0 < total; x0 += 8 * blockDim.x) {
+      int idx[8], nls[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int x = x0 + u * blockDim.x + threadIdx.x;
+        const int nl = x < total ? x / s.topk : 0, jj = x - nl * s.topk;
+        nls[u] = nl;
+        idx[u] = (x < total && n_cand[nl] > s.topk) ? __ldcg(sel + (size_t)(n0 + nl) * s.topk + jj) : -1;   // unused slots hold -1
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (idx[u] < 0) continue;
+        if (idx[u] < n_csa) atomicOr(cm32 + (idx[u] >> 2), (1u << nls[u]) << (8 * (idx[u] & 3)));
+        else if (idx[u] - n_csa < 32) atomicOr(&newc_bits[nls[u]], 1u << (idx[u] - n_csa));
+      }
+    }
+    __syncthreads();
+    if (allbits) {
+      for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)allbits;
       __syncthreads();
     }
   }
   // is the entry closed at node a (a strict ancestor of node n0 + nl) among that node's selected CSA entries?
   auto newc_selected = [&](int nl, int a) {
     if (n_cand[nl] <= s.topk) return true;
-    const int n = n0 + nl, blk = (tm.L + tm.depth[a]) / s.m_csa, cnt = selcnt[n];
-    const int32_t* sl = sel + (size_t)n * s.topk;
-    int lo_ = 0, hi_ = cnt - 1;
-    while (lo_ <= hi_) { const int mid = (lo_ + hi_) >> 1; const int v = sl[mid]; if (v == blk) return true; if (v < blk) lo_ = mid + 1; else hi_ = mid - 1; }
-    return false;
+    const int dblk = (tm.L + tm.depth[a]) / s.m_csa - n_csa;
+    return dblk >= 0 && dblk < 32 && ((newc_bits[nl] >> dblk) & 1u);
   };
   if (pl.tc_tma) {
     // the packed per-sequence rows (written by the sequence's extra CTA): few HCA entries, tree nodes, entries closed in the tree
@@ -649,7 +670,7 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
   TvaPlan p = p_in;
   p.tc_tma = tva_tc_pair_usable(c) ? 1 : 0;
-  const size_t plan_sm = p.need_scores ? (size_t)p.cand_cap : 0;
+  const size_t plan_sm = p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) : 0;   // node bits per entry, cleared by words
   if (plan_sm > 32 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
     return TSV_ERR_CUDA;
   TSV_PREP(tc_plan_kernel);
