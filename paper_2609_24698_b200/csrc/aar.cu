@@ -14,37 +14,49 @@ __global__ void __launch_bounds__(32) aar_walk_kernel(const tsv_shape s, const A
                                                       const int32_t* __restrict__ target, int32_t* __restrict__ accept_len,
                                                       int32_t* __restrict__ accept_path, int32_t* __restrict__ bonus,
                                                       int32_t* __restrict__ status, const int do_walk) {
-  __shared__ TreeMeta tm;
-  if (threadIdx.x != 0) return;
-  const int b = blockIdx.x, D = s.D;
+  // One warp per sequence.  Lane l checks layer l's length and capacities (the same checks as build_tree_meta), lane n
+  // checks node n's parent; the greedy walk runs on ballots: lane c holds node c's parent and draft token.
+  const int b = blockIdx.x, D = s.D, lane = threadIdx.x;
   int st = 0;
-  for (int l = 0; l < ls.n; ++l) {
-    build_tree_meta(tm, s, ls.l[l].c.L[b], parent + (size_t)b * D, n_nodes[b], ls.l[l].c.csa_cap + b, ls.l[l].c.hca_cap + b);
-    st |= tm.status;
+  int nn = n_nodes[b];
+  if (nn < 1 || nn > D) { st |= TSV_ST_NODES; nn = 0; }
+  for (int l = lane; l < ls.n; l += 32) {
+    int L = ls.l[l].c.L[b];
+    if (L < 0 || (int64_t)L + D > s.max_L) { st |= TSV_ST_LENGTH; L = 0; }
+    if ((L + D) / s.m_csa > ls.l[l].c.csa_cap[b]) st |= TSV_ST_CSA_CAP;
+    if ((L + D) / s.m_hca > ls.l[l].c.hca_cap[b]) st |= TSV_ST_HCA_CAP;
   }
-  if (st) atomicOr(status + b, st);
+  const int par = lane < nn ? parent[(size_t)b * D + lane] : -1;
+  if (lane < nn && (lane == 0 ? par != -1 : (par < 0 || par >= lane))) st |= TSV_ST_PARENT;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) st |= __shfl_xor_sync(0xffffffffu, st, o);
+  if (lane == 0 && st) atomicOr(status + b, st);
   if (!do_walk) return;
-  st |= status[b];
+  st |= status[b];                                     // flags raised earlier in the cycle (every lane reads the same word)
+  st = __shfl_sync(0xffffffffu, st, 0);
   int len = 0, bt = -1;
   if (!st) {
-    const int32_t* dr = draft + (size_t)b * D;
-    const int32_t* tg = target + (size_t)b * D;
+    const int dr = lane < nn ? draft[(size_t)b * D + lane] : 0;
+    const int tg = lane < nn ? target[(size_t)b * D + lane] : 0;
     int cur = 0;
-    accept_path[(size_t)b * D + len++] = 0;
+    if (lane == 0) accept_path[(size_t)b * D] = 0;
+    len = 1;
     for (;;) {
-      int nxt = -1;
-      const int want = tg[cur];
-      for (int c = cur + 1; c < tm.nn; ++c)
-        if (tm.parent[c] == cur && dr[c] == want) { nxt = c; break; }
-      if (nxt < 0) break;
-      accept_path[(size_t)b * D + len++] = nxt;
+      const int want = __shfl_sync(0xffffffffu, tg, cur);
+      const uint32_t match = __ballot_sync(0xffffffffu, lane > cur && lane < nn && par == cur && dr == want);
+      if (!match) break;
+      const int nxt = __ffs(match) - 1;                // the first matching child in node order
+      if (lane == 0) accept_path[(size_t)b * D + len] = nxt;
+      ++len;
       cur = nxt;
     }
-    bt = tg[cur];
+    bt = __shfl_sync(0xffffffffu, tg, cur);
   }
-  for (int i = len; i < D; ++i) accept_path[(size_t)b * D + i] = -1;
-  accept_len[b] = len;
-  bonus[b] = bt;
+  if (lane == 0) {
+    for (int i = len; i < D; ++i) accept_path[(size_t)b * D + i] = -1;
+    accept_len[b] = len;
+    bonus[b] = bt;
+  }
 }
 
 __device__ __forceinline__ void copy_row16(void* dst, const void* src, int bytes, int tid, int nthr) {
