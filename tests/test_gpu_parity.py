@@ -222,6 +222,15 @@ def test_budget_and_batch_sweep(D, B):
     lockstep(cfg, cycles=2)
 
 
+def test_ranked_short_candidate_lists_bf16():
+    """Benchmark head shape with a small top-k: every node ranks its candidates, the lists are short enough to be scored
+    inside the selection kernel (256-byte indexer rows), and the committed runs lie on both sides of 2 x topk, so ranked
+    tiles take the contiguous-run path with per-node masks as well as the pointer-gather path."""
+    cfg = synth.Config("ranked_short", 71, synth.Shape("bf16", 6, 8, 64, 512, 4, 128, 4, 128, 128, 128),
+                       L_min=300, L_max=1400, seed=9)
+    lockstep(cfg, cycles=2)
+
+
 # ------------------------------------------------------------------------------------------------ status / error paths
 def test_device_detected_errors_commit_nothing():
     from paper_2609_24698_b200 import binding as tsv, harness as hz
