@@ -43,7 +43,7 @@ struct TvaPlan {
   // tensor-core path (bf16, d = 512): row tiles per sequence, key-list capacity per tile, max chunks per tile
   int32_t tc, tc_nt, tc_maxk, tc_chmax;
   int32_t tc_tma, tc_misc_rows;      // contiguous-run tiles go through TMA; rows of the per-sequence packed buffer
-  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_counter, off_tcnt;
+  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt, off_pos;
 };
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
 

@@ -126,11 +126,44 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   __shared__ int wsum[9];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
+  if (blockIdx.x == (unsigned)s.D) {
+    // Extra CTA column (only with the tensor-core attention path): CTA (D, 0) ranks the 256-row tiles of all sequences by
+    // the number of keys they will stage, most first, so that the paired attention kernel starts the long tiles first
+    // and the short ones fill the tail.  The counts follow from lengths, node counts and done flags alone (for tiles on
+    // the contiguous-run path they are exact; for pointer-gather tiles an estimate: only the order depends on them), so
+    // the ranking is ready before the plan kernel runs and each plan CTA can leave its record at its final position.
+    if (blockIdx.y != 0) return;
+    __shared__ int32_t nk_est[2048];
+    const int D = s.D, nt = pl.tc_nt, ntile = s.B * nt, npt = 256 / s.H;
+    int32_t* pos = reinterpret_cast<int32_t*>(ws + pl.off_pos);
+    if (ntile > 2048) { for (int i = threadIdx.x; i < ntile; i += blockDim.x) pos[i] = i; return; }
+    auto r32 = [](int x) { return (x + kBoxRows - 1) / kBoxRows * kBoxRows; };
+    for (int i = threadIdx.x; i < ntile; i += blockDim.x) {
+      const int b = i / nt, tile = i - b * nt;
+      const int L = c.L[b], nn = nd.n_nodes[b];
+      int est = 0;
+      if (L >= 0 && (int64_t)L + D <= s.max_L && nn >= 1 && nn <= D && tile * npt < nn) {
+        int ncd = 0, nhd = 0;
+        for (int j = 0; j < nn; ++j) { ncd += sc.csa_done[(size_t)b * D + j] != 0; nhd += sc.hca_done[(size_t)b * D + j] != 0; }
+        const int n_csa = L / s.m_csa, n_hca = L / s.m_hca, nh_in = n_hca <= kHcaMiscMax ? n_hca : 0, win = min(L, s.window);
+        if (n_csa <= 2 * s.topk) est = r32(n_csa) + (n_hca > kHcaMiscMax ? r32(n_hca) : 0) + r32(win) + r32(nh_in + nn + ncd + nhd);
+        else est = min(n_csa, npt * s.topk) + n_hca + win + 3 * nn;
+      }
+      nk_est[i] = est;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < ntile; i += blockDim.x) {
+      const int ki = nk_est[i];
+      int rank = 0;
+      for (int j = 0; j < ntile; ++j) { const int kj = nk_est[j]; rank += (kj > ki) || (kj == ki && j < i); }
+      pos[i] = rank;
+    }
+    return;
+  }
   const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk;
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
-  if (pl.tc && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *reinterpret_cast<unsigned int*>(ws + pl.off_counter) = 0u;   // the plan kernel's finished-CTA counter
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
   if (threadIdx.x == 0) {
     if (tm.status && n == 0) atomicOr(status + b, tm.status);
@@ -356,7 +389,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
       count_launch();
     }
   }
-  dim3 g2(s.D, s.B);
+  dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
   TSV_PREP(topk_kernel<bf16>);
   TSV_PREP(topk_kernel<float>);
   const size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;   // the node's indexer queries

@@ -275,43 +275,24 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   }
 }
 
-// Plan of every (sequence, 256-row tile).  The CTA that finishes last also orders the tiles by decreasing key count:
-// the paired attention kernel takes tiles in that order, so the long ones start first and the short ones fill the tail
-// (the grid is less than two waves of CTA pairs, and tile lengths differ by an order of magnitude).
+// Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the scheduling
+// position the selection kernel computed for it (most keys first): the paired attention kernel takes the tiles in that
+// order and learns all it needs about its tile from one load.
 __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
-  __shared__ int is_last;
-  if (threadIdx.x < 2 && blockIdx.x < (unsigned)pl.tc_nt)   // finished-chunk counters of the tile's two 128-row halves
-    reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[((size_t)blockIdx.y * pl.tc_nt + blockIdx.x) * 2 + threadIdx.x] = 0;
+  const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
+  const size_t tix = (size_t)blockIdx.y * pl.tc_nt + blockIdx.x;
+  int pos = (int)tix;                                 // fetched now, used at the end
+  if (tile_cta && threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // (with TSV_FLAG_SKIP_SELECT: the previous call's)
+  if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
+    reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
   tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
-  __threadfence();
-  __syncthreads();
-  unsigned int* counter = reinterpret_cast<unsigned int*>(ws + pl.off_counter);
-  if (threadIdx.x == 0) is_last = atomicAdd(counter, 1u) == gridDim.x * gridDim.y - 1;
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  const int n = s.B * pl.tc_nt;
-  const volatile int32_t* nkeys = reinterpret_cast<const volatile int32_t*>(ws + pl.off_nkeys);
-  const volatile int32_t* mode = reinterpret_cast<const volatile int32_t*>(ws + pl.off_mode);
-  int4* order = reinterpret_cast<int4*>(ws + pl.off_order);    // {tile index, mode, keys, -} per position: the paired kernel
-                                                               // learns all it needs about its tile from one load
-  __shared__ int32_t nk_sm[2048];                       // the counts are fetched once; the ranking reads them from shared memory
-  if (n <= 2048) {
-    for (int i = threadIdx.x; i < n; i += blockDim.x) nk_sm[i] = nkeys[i];
-    __syncthreads();
+  if (tile_cta && threadIdx.x == 0) {                 // thread 0 wrote the tile's key count and mode itself
+    if (pos < 0 || pos >= s.B * pl.tc_nt) pos = (int)tix;
+    reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
+        make_int4((int)tix, reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix], reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix], 0);
   }
-  for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    int rank = i;
-    const int ki = nkeys[i];
-    if (n <= 2048) {                                    // rank = tiles with more keys (ties: lower index first)
-      rank = 0;
-      for (int j = 0; j < n; ++j) { const int kj = nk_sm[j]; rank += (kj > ki) || (kj == ki && j < i); }
-    }
-    order[rank] = make_int4(i, mode[i], ki, 0);
-  }
-  if (threadIdx.x == 0) *counter = 0;                   // ready for the next call on this workspace
 }
 
 // ------------------------------------------------------------------------------------------------ attention
