@@ -10,7 +10,8 @@
 //                    mode 1 (every node selects all CSA candidates, or the CSA slab is at most 2 x topk rows): contiguous
 //                    runs {CSA slab, HCA slab, window ring, packed misc rows} as 32-row TMA boxes + node masks;
 //                    mode 0 (selection far from dense): row pointers of the union of the nodes' selections + masks.
-//                    The last CTA to finish orders the tiles by key count for the paired kernel.
+//                    Each tile CTA leaves its record {tile, mode, keys} at the scheduling position the selection kernel
+//                    computed (most keys first); an extra CTA per sequence packs the small scattered rows.
 //   tc_attn_kernel   mode-0 tiles, one CTA per 128 rows and chunk of <= 512 keys:
 //       phase 1  S[128 x CL] = Q K^T      tcgen05.mma kind::f16, A = Q slice (smem, K-major), B = 256 key rows x 64 dims
 //       phase 2  exact softmax of the chunk on the fp32 S read with tcgen05.ld; P (bf16) written back over S (tcgen05.st)
@@ -18,7 +19,7 @@
 //     Operand tiles stream through a ring of seven 32 KiB slots filled with 16-byte cp.async copies written in the
 //     128-byte swizzle pattern (any row from any source array, zero fill for padding), four stages ahead of the MMA
 //     issue; slots are released by tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
-//   tc_combine_kernel merges the chunks of tiles that needed more than one (fixed order), per 128 rows.
+//   tc_combine_kernel merges the chunks of mode-0 tiles that needed more than one (fixed order), per 128 rows.
 #include "tc_common.cuh"
 
 namespace tsv {
