@@ -576,26 +576,64 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         bf16* orow0 = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
         const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + rix * pl.tc_chmax * BM * DH;
         const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM;
-        for (int i = (warp - 2) * 32 + lane; i < BM * DH / 8; i += 256) {
-          const int r = i / (DH / 8), c8 = i % (DH / 8);
-          if (row0 + r >= rows_seq) continue;
-          float m = -INFINITY;
-          for (int ch = 0; ch < nch; ++ch) { const float2 ml = __ldcg(pml + ch * BM + r); if (ml.y > 0.f) m = fmaxf(m, ml.x); }
-          float l = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          for (int ch = 0; ch < nch; ++ch) {
-            const float2 ml = __ldcg(pml + ch * BM + r);
-            if (!(ml.y > 0.f)) continue;
-            const float w = exp2f(ml.x - m);
-            l = fmaf(ml.y, w, l);
-            const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + r) * DH + c8 * 8);
-            const float4 a = __ldcg(p4), bq = __ldcg(p4 + 1);
-            o[0] = fmaf(a.x, w, o[0]); o[1] = fmaf(a.y, w, o[1]); o[2] = fmaf(a.z, w, o[2]); o[3] = fmaf(a.w, w, o[3]);
-            o[4] = fmaf(bq.x, w, o[4]); o[5] = fmaf(bq.y, w, o[5]); o[6] = fmaf(bq.z, w, o[6]); o[7] = fmaf(bq.w, w, o[7]);
-          }
-          const float inv = l > 0.f ? 1.f / l : 0.f;
+        // One CTA merges a whole 128-row tile, so global latency has to be covered inside the thread: a warp takes 16 rows
+        // (w, w + 8, ...), first the rows' reference maxima and sums (lane j < 16 for row w + 8 j, one round of loads), then
+        // four rows at a time with all their loads of a chunk pair in flight; a lane owns columns 4 (l + 32 k) .. + 3.
+        const int w = warp - 2;
+        float m_row = -INFINITY, inv_row = 0.f;
+        if (lane < 16) {
+          const int r = w + 8 * lane;
+          float l = 0.f;
+          for (int ch = 0; ch < nch; ++ch) { const float2 ml = __ldcg(pml + ch * BM + r); if (ml.y > 0.f) m_row = fmaxf(m_row, ml.x); }
+          for (int ch = 0; ch < nch; ++ch) { const float2 ml = __ldcg(pml + ch * BM + r); if (ml.y > 0.f) l = fmaf(ml.y, exp2f(ml.x - m_row), l); }
+          inv_row = l > 0.f ? 1.f / l : 0.f;
+        }
+#pragma unroll 1
+        for (int step = 0; step < 4; ++step) {
+          float4 acc[4][4];
+          float mj[4], invj[4];
 #pragma unroll
-          for (int t = 0; t < 8; ++t) o[t] *= inv;
-          st16(orow0 + (size_t)r * DH + c8 * 8, o);
+          for (int jx = 0; jx < 4; ++jx) {
+            mj[jx] = __shfl_sync(0xffffffffu, m_row, 4 * step + jx);
+            invj[jx] = __shfl_sync(0xffffffffu, inv_row, 4 * step + jx);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc[jx][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll 2
+          for (int ch = 0; ch < nch; ++ch) {
+            float2 ml[4];
+            float4 v[4][4];
+#pragma unroll
+            for (int jx = 0; jx < 4; ++jx) {
+              const int r = w + 8 * (4 * step + jx);
+              ml[jx] = __ldcg(pml + ch * BM + r);
+              const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + r) * DH);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) v[jx][k] = __ldcg(p4 + lane + 32 * k);
+            }
+#pragma unroll
+            for (int jx = 0; jx < 4; ++jx) {
+              const float wgt = ml[jx].y > 0.f ? exp2f(ml[jx].x - mj[jx]) : 0.f;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                acc[jx][k].x = fmaf(v[jx][k].x, wgt, acc[jx][k].x); acc[jx][k].y = fmaf(v[jx][k].y, wgt, acc[jx][k].y);
+                acc[jx][k].z = fmaf(v[jx][k].z, wgt, acc[jx][k].z); acc[jx][k].w = fmaf(v[jx][k].w, wgt, acc[jx][k].w);
+              }
+            }
+          }
+#pragma unroll
+          for (int jx = 0; jx < 4; ++jx) {
+            const int r = w + 8 * (4 * step + jx);
+            if (row0 + r >= rows_seq) continue;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[jx][k].x * invj[jx], acc[jx][k].y * invj[jx]);
+              const __nv_bfloat162 hi = __floats2bfloat162_rn(acc[jx][k].z * invj[jx], acc[jx][k].w * invj[jx]);
+              uint2 o2;
+              o2.x = *reinterpret_cast<const uint32_t*>(&lo); o2.y = *reinterpret_cast<const uint32_t*>(&hi);
+              *reinterpret_cast<uint2*>(orow0 + (size_t)r * DH + 4 * (lane + 32 * k)) = o2;
+            }
+          }
         }
       }
     }
