@@ -317,9 +317,15 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
         if (threadIdx.x + 256 * j < n_cand && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
       }
     } else {
-      for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
-        const uint32_t key = key_of(i);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      // long lists: eight scores of a thread in flight per round (a node's list is scanned by one CTA, so the loads'
+      // latency has to be covered inside the thread)
+      for (int i0 = threadIdx.x; i0 < n_cand; i0 += 8 * 256) {
+        uint32_t kk[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { const int i = i0 + 256 * u; kk[u] = i < n_cand ? key_of(i) : 0u; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (i0 + 256 * u < n_cand && (kk[u] & mask) == prefix) atomicAdd(&hist[(kk[u] >> shift) & 255u], 1);
       }
     }
     __syncthreads();
@@ -345,6 +351,52 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   }
   const uint32_t thr = sh_prefix;       // key of the k-th largest score
   const int r = sh_remaining;           // how many of the scores equal to it are taken (lowest indices)
+  if (!in_regs) {
+    // Long lists: warp w owns a contiguous share of the candidates and walks it twice, eight 32-candidate steps of loads
+    // in flight per round: first counting the keys above and equal to the threshold, then (after one exchange of the
+    // warps' counts) writing the selected indices in ascending order at positions found with ballots.
+    __shared__ int wgt[8], weq[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int share = ((n_cand + 7) / 8 + 31) & ~31;
+    const int beg = w * share, end = min(n_cand, beg + share);
+    int cg = 0, ce = 0;
+    for (int i0 = beg; i0 < end; i0 += 256) {
+      uint32_t kk[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int i = i0 + 32 * u + lane; kk[u] = i < end ? key_of(i) : 0u; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const bool in = i0 + 32 * u + lane < end; cg += in && kk[u] > thr; ce += in && kk[u] == thr; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
+    if (lane == 0) { wgt[w] = cg; weq[w] = ce; }
+    __syncthreads();
+    int eq_base = 0, out_base = 0;
+    for (int x = 0; x < w; ++x) { eq_base += weq[x]; out_base += wgt[x]; }
+    out_base += min(r, eq_base);                       // of the equal keys before this share, the first r are taken
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int i0 = beg; i0 < end; i0 += 256) {
+      uint32_t kk[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int i = i0 + 32 * u + lane; kk[u] = i < end ? key_of(i) : 0u; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + 32 * u + lane;
+        const bool in = i < end, eq = in && kk[u] == thr, gt = in && kk[u] > thr;
+        const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
+        const bool take = gt || (eq && eq_base + __popc(eqm & lt) < r);
+        const uint32_t tkm = __ballot_sync(0xffffffffu, take);
+        if (take) {
+          const int pos = out_base + __popc(tkm & lt);
+          const int v = i < n_csa ? i : pe.newc_blk[i - n_csa];
+          sel[pos] = v; if (usr) usr[pos] = v;
+        }
+        eq_base += __popc(eqm); out_base += __popc(tkm);
+      }
+    }
+    if (threadIdx.x == 0) *selcnt = k;
+    return;
+  }
   int eq_base = 0, out_base = 0;
   for (int i0 = 0, j0 = 0; i0 < n_cand; i0 += blockDim.x, ++j0) {
     const int i = i0 + threadIdx.x;
