@@ -114,6 +114,75 @@ __device__ __forceinline__ void unpack16(const uint4& v, float* o, const bf16*) 
   for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(w[i] << 16); o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
 }
 
+// Indexer scores for long candidate lists with 256-byte key rows (the benchmark's indexer width), one node per CTA in z:
+// eight lanes share an entry, each holding its 32-byte slice of the node's queries in registers, so the inner product runs
+// from registers (the thread-per-entry kernel above reads a query value from shared memory for every multiply-add and is
+// bound by that); a CTA covers kRows256PerCta entries (the set-up of a CTA is amortised over them), four entries of a
+// lane group in flight.  grid (ceil(entries / kRows256PerCta), B, D).
+constexpr int kRows256PerCta = 2048;
+template <typename T>
+__global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                                const tsv_scratch sc, char* __restrict__ ws) {
+  __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
+  const int b = blockIdx.y, n = blockIdx.z, D = s.D, di = s.di, HI = s.HI;
+  constexpr int V = Vec<T>::N, EL = 2 * V;
+  {   // cheap exit: even with every ancestor closing a block, no node of this sequence has more than topk candidates
+    const int L0 = c.L[b];
+    if (L0 < 0 || L0 / s.m_csa + D <= s.topk || (int)(blockIdx.x * kRows256PerCta) >= L0 / s.m_csa) return;
+  }
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, nullptr, nullptr);
+  if (tm.status || n >= tm.nn || (int)(blockIdx.x * kRows256PerCta) >= tm.n_csa) return;
+  {   // does this node rank?  candidates = committed entries + blocks closed at its strict ancestors
+    int extra = 0;
+    for (int j = 0; j < n; ++j) if (((tm.anc[n] >> j) & 1u) && sc.csa_done[(size_t)b * D + j]) ++extra;
+    if (tm.n_csa + extra <= s.topk) return;
+  }
+  const int grp = threadIdx.x >> 3, gl = threadIdx.x & 7;
+  const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * HI * di;
+  float q[4][EL], iwreg[4];
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    iwreg[h] = h < HI ? nd.iw[((size_t)b * D + n) * HI + h] : 0.f;
+    float t0[V], t1[V];
+    if (h < HI) { ld16(iq + h * di + gl * EL, t0); ld16(iq + h * di + gl * EL + V, t1); }
+#pragma unroll
+    for (int j = 0; j < V; ++j) { q[h][j] = h < HI ? t0[j] : 0.f; q[h][V + j] = h < HI ? t1[j] : 0.f; }
+  }
+  const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
+  float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+  const int n_csa = tm.n_csa, e_base = blockIdx.x * kRows256PerCta, e_end = min(n_csa, e_base + kRows256PerCta);
+#pragma unroll 1
+  for (int base = e_base; base < e_end; base += 128) {          // uniform trip count: the shuffles need the whole warp
+    uint4 raw[4][2];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = base + grp + 32 * u;
+      const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)(e < n_csa ? e : 0) * di) + gl * 2;
+      raw[u][0] = __ldg(rowp); raw[u][1] = __ldg(rowp + 1);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float kk[EL];
+      unpack16(raw[u][0], kk, (const T*)nullptr);
+      unpack16(raw[u][1], kk + V, (const T*)nullptr);
+      float tot = 0.f;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        float pp = 0.f;
+#pragma unroll
+        for (int j = 0; j < EL; ++j) pp = fmaf(q[h][j], kk[j], pp);
+        pp += __shfl_xor_sync(0xffffffffu, pp, 1);
+        pp += __shfl_xor_sync(0xffffffffu, pp, 2);
+        pp += __shfl_xor_sync(0xffffffffu, pp, 4);
+        tot = fmaf(iwreg[h], fmaxf(pp, 0.f), tot);
+      }
+      const int e = base + grp + 32 * u;
+      if (gl == 0 && e < n_csa) sw[e] = tot;
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
@@ -428,7 +497,12 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
     const int pref_cap = (int)(s.max_L / s.m_csa);
     dim3 grid((pref_cap + 255) / 256, s.B, s.D <= 8 ? s.D : 8);        // z: slabs of nodes, so a ranked sequence is scored by many CTAs
     const size_t sm = (size_t)32 * s.di * sizeof(float);
-    if (grid.x > 0) {
+    if (grid.x > 0 && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) {
+      const dim3 g8((pref_cap + kRows256PerCta - 1) / kRows256PerCta, s.B, s.D);   // one node per CTA: queries in registers
+      if (bf) { TSV_PREP(idx_score_rows256_kernel<bf16>); idx_score_rows256_kernel<bf16><<<g8, 256, 0, st>>>(s, p, c, nd, sc, ws); }
+      else { TSV_PREP(idx_score_rows256_kernel<float>); idx_score_rows256_kernel<float><<<g8, 256, 0, st>>>(s, p, c, nd, sc, ws); }
+      count_launch();
+    } else if (grid.x > 0) {
       if (bf) {
         cudaFuncSetAttribute(idx_score_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
         TSV_PREP(idx_score_kernel<bf16>);
