@@ -606,26 +606,48 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
   const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + rix * pl.tc_chmax * BM * DH;
   const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM;
-  for (int i = threadIdx.x; i < BM * DH / 8; i += blockDim.x) {
-    const int row = i / (DH / 8), c8 = i % (DH / 8);
-    if (row0 + row >= rows_seq) continue;
-    float m = -INFINITY;
-    for (int ch = 0; ch < nch; ++ch) { const float2 ml = pml[ch * BM + row]; if (ml.y > 0.f) m = fmaxf(m, ml.x); }
-    float l = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int ch = 0; ch < nch; ++ch) {
-      const float2 ml = pml[ch * BM + row];
-      if (!(ml.y > 0.f)) continue;
-      const float w = exp2f(ml.x - m);
-      l = fmaf(ml.y, w, l);
-      const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + row) * DH + c8 * 8);
-      const float4 a = p4[0], bq = p4[1];
-      o[0] = fmaf(a.x, w, o[0]); o[1] = fmaf(a.y, w, o[1]); o[2] = fmaf(a.z, w, o[2]); o[3] = fmaf(a.w, w, o[3]);
-      o[4] = fmaf(bq.x, w, o[4]); o[5] = fmaf(bq.y, w, o[5]); o[6] = fmaf(bq.z, w, o[6]); o[7] = fmaf(bq.w, w, o[7]);
-    }
-    const float inv = l > 0.f ? 1.f / l : 0.f;
+  // grid z splits the tile's 128 rows into groups of 8: a warp merges one row, a lane owns columns 4 (l + 32 k) .. + 3.
+  // The chunks are accumulated in order (the result does not depend on the launch shape), four chunks' loads in flight.
+  const int lane = threadIdx.x & 31, row = blockIdx.z * 8 + (threadIdx.x >> 5);
+  if (row >= BM || row0 + row >= rows_seq) return;
+  float m = -INFINITY;
+  for (int ch = lane; ch < nch; ch += 32) { const float2 ml = pml[ch * BM + row]; if (ml.y > 0.f) m = fmaxf(m, ml.x); }
 #pragma unroll
-    for (int t = 0; t < 8; ++t) o[t] *= inv;
-    st16(out + (size_t)row * DH + c8 * 8, o);
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float l = 0.f;
+  float4 acc[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c0 = 0; c0 < nch; c0 += 4) {
+    float2 ml[4];
+    float4 v[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int ch = c0 + u < nch ? c0 + u : nch - 1;
+      ml[u] = pml[ch * BM + row];
+      const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + row) * DH);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) v[u][k] = p4[lane + 32 * k];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (c0 + u >= nch || !(ml[u].y > 0.f)) continue;
+      const float w = exp2f(ml[u].x - m);
+      l = fmaf(ml[u].y, w, l);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        acc[k].x = fmaf(v[u][k].x, w, acc[k].x); acc[k].y = fmaf(v[u][k].y, w, acc[k].y);
+        acc[k].z = fmaf(v[u][k].z, w, acc[k].z); acc[k].w = fmaf(v[u][k].w, w, acc[k].w);
+      }
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k].x * inv, acc[k].y * inv), hi = __floats2bfloat162_rn(acc[k].z * inv, acc[k].w * inv);
+    uint2 o2;
+    o2.x = *reinterpret_cast<const uint32_t*>(&lo); o2.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + (size_t)row * DH + 4 * (lane + 32 * k)) = o2;
   }
 }
 
@@ -672,7 +694,7 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, c
     tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
     if (p.tc_chmax > 1) {
-      tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B), 256, 0, st>>>(s, p, out, ws);
+      tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);   // z: groups of 8 rows
       count_launch();
     }
   }
