@@ -222,6 +222,15 @@ def test_budget_and_batch_sweep(D, B):
     lockstep(cfg, cycles=2)
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_long_candidate_lists_generic_scoring(dtype):
+    """More than 2048 candidates per node with indexer rows that are not 256 bytes wide: the thread-per-entry scoring
+    kernel and both key paths of the per-node selection (up to 2304 candidates: keys in registers; beyond: re-read)."""
+    cfg = synth.small_config(name="long_lists", dtype=dtype, B=3, D=6, H=4, d=16, m_csa=2, topk=24, HI=2, di=8, m_hca=32,
+                             window=16, L_min=4200, L_max=5200, layers=1, seed=77, cfg_id=72)
+    lockstep(cfg, cycles=2)
+
+
 def test_ranked_short_candidate_lists_bf16():
     """Benchmark head shape with a small top-k: every node ranks its candidates, the lists are short enough to be scored
     inside the selection kernel (256-byte indexer rows), and the committed runs lie on both sides of 2 x topk, so ranked
