@@ -221,14 +221,35 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   }
   if (threadIdx.x == 0) *mode = 0;
   // committed CSA entries, in index order
+  // warp w owns a contiguous share of the entries: count its selected ones, exchange the counts once, then write the
+  // pointers in index order at positions found with ballots (no block-wide scan per 256 entries: runs are up to 32768 long)
   int base = 0;
-  for (int i0 = 0; i0 < n_csa; i0 += blockDim.x) {
-    const int i = i0 + threadIdx.x;
-    const uint32_t m = i < n_csa ? (dense ? validbits : cmask[i]) : 0u;
-    int tot;
-    const int pos = base + block_excl_scan_256(m != 0, wsum, tot);
-    if (m) { kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)csa_row0 + i) * rowb); kmask[pos] = (uint8_t)m; }
-    base += tot;
+  {
+    __shared__ int wcnt[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int share = ((n_csa + 7) / 8 + 31) & ~31;
+    const int beg = min(n_csa, w * share), end = min(n_csa, beg + share);
+    auto mask_of = [&](int i) -> uint32_t { return i < end ? (dense ? validbits : (uint32_t)cmask[i]) : 0u; };
+    int cnt = 0;
+    for (int i0 = beg; i0 < end; i0 += 32) cnt += mask_of(i0 + lane) != 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0) wcnt[w] = cnt;
+    __syncthreads();
+    int pos0 = 0, total = 0;
+    for (int x = 0; x < 8; ++x) { if (x < w) pos0 += wcnt[x]; total += wcnt[x]; }
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int i0 = beg; i0 < end; i0 += 32) {
+      const int i = i0 + lane;
+      const uint32_t m = mask_of(i);
+      const uint32_t sel_m = __ballot_sync(0xffffffffu, m != 0);
+      if (m) {
+        const int pos = pos0 + __popc(sel_m & lt);
+        kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)csa_row0 + i) * rowb); kmask[pos] = (uint8_t)m;
+      }
+      pos0 += __popc(sel_m);
+    }
+    base = total;
   }
   // committed HCA entries
   for (int i = threadIdx.x; i < tm.n_hca; i += blockDim.x) {
