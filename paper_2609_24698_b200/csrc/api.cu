@@ -35,6 +35,7 @@ static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   const int64_t pref = s.max_L / s.m_csa;
   p.cand_cap = (int32_t)(pref + s.D);
+  p.score_ld = (p.cand_cap + 3) & ~3;
   p.need_scores = p.cand_cap > s.topk;
   p.idx_fused = p.need_scores && p.cand_cap <= kIdxFusedMax && s.HI <= 8 && (size_t)s.HI * s.di * sizeof(float) <= 32768;
   const int64_t ksel = p.cand_cap < s.topk ? p.cand_cap : s.topk;
@@ -51,7 +52,7 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   size_t off = 0;
   p.off_selcnt = off; off = up256(off + (size_t)s.B * s.D * sizeof(int32_t));
   p.off_sel = off;    off = up256(off + (size_t)s.B * s.D * s.topk * sizeof(int32_t));
-  p.off_scores = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.cand_cap * sizeof(float));
+  p.off_scores = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.score_ld * sizeof(float));
   p.off_po = off;     if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * s.d * sizeof(float));
   p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
   p.tc = tva_tc_eligible(s);

@@ -33,6 +33,7 @@ struct AarLayers {
 // Workspace carve-up of tree_verify_attn (byte offsets from a 256-byte aligned base).
 struct TvaPlan {
   int32_t cand_cap;      // max CSA candidates per node (committed + in-tree)
+  int32_t score_ld;      // floats per node row of the score array: cand_cap rounded up to 4 (16-byte rows)
   int32_t need_scores;   // cand_cap > topk: some node may have to rank its candidates
   int32_t idx_fused;     // ranked nodes score their committed entries inside topk_kernel (short candidate lists: the
                          // separate scoring kernel, which exits at once for every sequence that needs no ranking, is not launched)

@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   const bool live = e < tm.n_csa;
   const T* ikrow = reinterpret_cast<const T*>(c.csa_ik) + ((size_t)c.csa_row0[b] + (live ? e : 0)) * di;
-  float* scores = reinterpret_cast<float*>(ws + pl.off_scores) + (size_t)b * D * pl.cand_cap;
+  float* scores = reinterpret_cast<float*>(ws + pl.off_scores) + (size_t)b * D * pl.score_ld;
   constexpr int V = Vec<T>::N;
   const int npg = min(32 / HI, (D + (int)gridDim.z - 1) / (int)gridDim.z);   // nodes per group; blockIdx.z owns a slab of nodes
   const int nz0 = blockIdx.z * ((D + (int)gridDim.z - 1) / (int)gridDim.z), nz1 = min(tm.nn, nz0 + (D + (int)gridDim.z - 1) / (int)gridDim.z);
@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
         for (int j = 0; j < 32; ++j) {
           if (j / HI == g && j < G) sc_ = fmaf(nd.iw[((size_t)b * D + n0 + g) * HI + (j % HI)], fmaxf(acc[j], 0.f), sc_);
         }
-        scores[(size_t)(n0 + g) * pl.cand_cap + e] = sc_;
+        scores[(size_t)(n0 + g) * pl.score_ld + e] = sc_;
       }
     }
   }
@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
     for (int j = 0; j < V; ++j) { q[h][j] = h < HI ? t0[j] : 0.f; q[h][V + j] = h < HI ? t1[j] : 0.f; }
   }
   const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
-  float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+  float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
   const int n_csa = tm.n_csa, e_base = blockIdx.x * kRows256PerCta, e_end = min(n_csa, e_base + kRows256PerCta);
 #pragma unroll 1
   for (int base = e_base; base < e_end; base += 128) {          // uniform trip count: the shuffles need the whole warp
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     for (int i = threadIdx.x; i < HI * di; i += blockDim.x) iq_sm[i] = to_f(iq[i]);
     __syncthreads();
     const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
-    float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+    float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
     if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
       // Rows of 256 bytes (the benchmark's indexer width): eight lanes share an entry, each holding its 32-byte slice of
       // the node's queries in registers for all entries; four entries of a group are in flight (few CTAs rank and global
@@ -359,7 +359,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   }
   if (threadIdx.x == 0) { sh_prefix = 0; sh_remaining = k; }
   __syncthreads();
-  const float* scores = reinterpret_cast<const float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.cand_cap;
+  const float* scores = reinterpret_cast<const float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
   // order-preserving keys; lists of up to 9 x 256 candidates keep them in registers for the five passes below (candidate
   // i = threadIdx.x + 256 j is key j of its thread), longer lists read the scores again
   constexpr int KREG = 9;
@@ -373,6 +373,51 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     }
   }
   auto key_of = [&](int i) { return order_key(i < n_csa ? __ldcg(scores + i) : extra[i - n_csa]); };
+  // Long lists are scanned in rounds: per round a thread takes eight groups of four consecutive candidates (groups g0,
+  // g0 + gstride, ...; key 4u + j is candidate 4 (g0 + gstride u) + j; a round of all threads covers 4 ground candidates
+  // from i_lo on).  A node's list is scanned by one CTA, so latency has to be covered inside the thread: the eight
+  // 16-byte loads of a round are issued unconditionally (group index clamped to the row; rows are padded to whole
+  // groups) and before anything that branches, and the next round's loads are issued before the current round's keys are
+  // used.  `full` (uniform over the threads that share i_lo, i_hi) says that every candidate of the round is a committed
+  // entry below i_hi, so that the body needs no range checks.
+  auto scan32 = [&](int first_g, int gstride, int ground, int i_lo, int i_hi, auto&& body) {
+    const float4* s4 = reinterpret_cast<const float4*>(scores);
+    const int gmax = pl.score_ld / 4 - 1;
+    const int nround = i_hi > i_lo ? (i_hi - i_lo + 4 * ground - 1) / (4 * ground) : 0;
+    const int i_full = min(i_hi, n_csa);
+    float4 va[8], vb[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) va[u] = __ldg(s4 + min(first_g + gstride * u, gmax));
+    for (int rd = 0; rd < nround; ++rd) {
+      const int g0 = first_g + rd * ground;
+      if (rd + 1 < nround) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) vb[u] = __ldg(s4 + min(g0 + ground + gstride * u, gmax));
+      }
+      const bool full = i_lo + (rd + 1) * 4 * ground <= i_full;
+      uint32_t kk[32];
+      if (full) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          kk[4 * u] = order_key(va[u].x); kk[4 * u + 1] = order_key(va[u].y);
+          kk[4 * u + 2] = order_key(va[u].z); kk[4 * u + 3] = order_key(va[u].w);
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float f[4] = {va[u].x, va[u].y, va[u].z, va[u].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int i = 4 * (g0 + gstride * u) + j;
+            kk[4 * u + j] = i < i_hi ? order_key(i < n_csa ? f[j] : extra[i - n_csa]) : 0u;
+          }
+        }
+      }
+      body(kk, g0, full);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) va[u] = vb[u];
+    }
+  };
   uint32_t mask = 0;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
@@ -386,16 +431,12 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
         if (threadIdx.x + 256 * j < n_cand && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
       }
     } else {
-      // long lists: eight scores of a thread in flight per round (a node's list is scanned by one CTA, so the loads'
-      // latency has to be covered inside the thread)
-      for (int i0 = threadIdx.x; i0 < n_cand; i0 += 8 * 256) {
-        uint32_t kk[8];
+      scan32(threadIdx.x, 256, 2048, 0, n_cand, [&](const uint32_t (&kk)[32], int g0, bool full) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { const int i = i0 + 256 * u; kk[u] = i < n_cand ? key_of(i) : 0u; }
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-          if (i0 + 256 * u < n_cand && (kk[u] & mask) == prefix) atomicAdd(&hist[(kk[u] >> shift) & 255u], 1);
-      }
+        for (int q = 0; q < 32; ++q)
+          if ((full || 4 * (g0 + 256 * (q >> 2)) + (q & 3) < n_cand) && (kk[q] & mask) == prefix)
+            atomicAdd(&hist[(kk[q] >> shift) & 255u], 1);
+      });
     }
     __syncthreads();
     if (threadIdx.x < 32) {                           // warp 0 finds the bin holding the rem-th largest key: lane l owns bins 255-8l .. 248-8l
@@ -421,21 +462,22 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   const uint32_t thr = sh_prefix;       // key of the k-th largest score
   const int r = sh_remaining;           // how many of the scores equal to it are taken (lowest indices)
   if (!in_regs) {
-    // Long lists: warp w owns a contiguous share of the candidates and walks it twice, eight 32-candidate steps of loads
-    // in flight per round: first counting the keys above and equal to the threshold, then (after one exchange of the
-    // warps' counts) writing the selected indices in ascending order at positions found with ballots.
+    // Long lists: warp w owns a contiguous share of the candidates (whole 128-candidate steps: a lane holds four
+    // consecutive candidates of a step) and walks it twice, eight steps per round: first counting the
+    // keys above and equal to the threshold, then (after one exchange of the warps' counts) writing the selected indices
+    // in ascending order at positions found with ballots.
     __shared__ int wgt[8], weq[8];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int share = ((n_cand + 7) / 8 + 31) & ~31;
+    const int share = ((n_cand + 7) / 8 + 127) & ~127;
     const int beg = w * share, end = min(n_cand, beg + share);
     int cg = 0, ce = 0;
-    for (int i0 = beg; i0 < end; i0 += 256) {
-      uint32_t kk[8];
+    scan32(beg / 4 + lane, 32, 256, beg, end, [&](const uint32_t (&kk)[32], int g0, bool full) {
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + 32 * u + lane; kk[u] = i < end ? key_of(i) : 0u; }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) { const bool in = i0 + 32 * u + lane < end; cg += in && kk[u] > thr; ce += in && kk[u] == thr; }
-    }
+      for (int q = 0; q < 32; ++q) {
+        const bool in = full || 4 * (g0 + 32 * (q >> 2)) + (q & 3) < end;
+        cg += in && kk[q] > thr; ce += in && kk[q] == thr;
+      }
+    });
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
     if (lane == 0) { wgt[w] = cg; weq[w] = ce; }
@@ -444,25 +486,38 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     for (int x = 0; x < w; ++x) { eq_base += weq[x]; out_base += wgt[x]; }
     out_base += min(r, eq_base);                       // of the equal keys before this share, the first r are taken
     const uint32_t lt = (1u << lane) - 1u;
-    for (int i0 = beg; i0 < end; i0 += 256) {
-      uint32_t kk[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + 32 * u + lane; kk[u] = i < end ? key_of(i) : 0u; }
+    scan32(beg / 4 + lane, 32, 256, beg, end, [&](const uint32_t (&kk)[32], int g0, bool full) {
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const int i = i0 + 32 * u + lane;
-        const bool in = i < end, eq = in && kk[u] == thr, gt = in && kk[u] > thr;
-        const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
-        const bool take = gt || (eq && eq_base + __popc(eqm & lt) < r);
-        const uint32_t tkm = __ballot_sync(0xffffffffu, take);
-        if (take) {
-          const int pos = out_base + __popc(tkm & lt);
-          const int v = i < n_csa ? i : pe.newc_blk[i - n_csa];
-          sel[pos] = v; if (usr) usr[pos] = v;
+        const int ib = 4 * (g0 + 32 * u);              // this lane's four candidates of the step
+        bool eq[4], take[4];
+        uint32_t eqm[4], tkm[4];
+        int run = eq_base, neq = 0, ntk = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          eq[j] = (full || ib + j < end) && kk[4 * u + j] == thr;
+          eqm[j] = __ballot_sync(0xffffffffu, eq[j]);
+          run += __popc(eqm[j] & lt); neq += __popc(eqm[j]);
         }
-        eq_base += __popc(eqm); out_base += __popc(tkm);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          take[j] = ((full || ib + j < end) && kk[4 * u + j] > thr) || (eq[j] && run < r);
+          run += eq[j];
+          tkm[j] = __ballot_sync(0xffffffffu, take[j]);
+        }
+        int pos = out_base;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { pos += __popc(tkm[j] & lt); ntk += __popc(tkm[j]); }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (take[j]) {
+            const int i = ib + j, v = i < n_csa ? i : pe.newc_blk[i - n_csa];
+            sel[pos] = v; if (usr) usr[pos] = v;
+            ++pos;
+          }
+        eq_base += neq; out_base += ntk;
       }
-    }
+    });
     if (threadIdx.x == 0) *selcnt = k;
     return;
   }
