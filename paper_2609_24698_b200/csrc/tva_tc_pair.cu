@@ -94,6 +94,9 @@ __device__ __forceinline__ uint32_t make_idesc2(int N, int b_mn_major) {      //
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// the two halves of the pair-wide barrier, for work that does not depend on the peer in between
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Tensor maps of one call: every source array with boxes of 32, 64 and 128 rows (64 columns, 128-byte swizzle), so that
@@ -164,6 +167,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  // Pair-wide barrier, first half: this CTA's barriers exist and its tensor memory is allocated (thread 0 and warp 0 arrive
+  // after doing that).  The plan's boxes and key masks are read while the peer gets there; the wait follows below.
+  __syncwarp();
+  cluster_arrive();
   {
     const int2* box_g = reinterpret_cast<const int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
     const uint8_t* kmask_g = reinterpret_cast<const uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
@@ -176,7 +183,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   }
   fence_before();
   __syncthreads();
-  cluster_sync_all();                                            // barriers of both CTAs exist before anyone signals them
+  cluster_wait();                                                // barriers of both CTAs exist before anyone signals them
   fence_after();
   const uint32_t tm = sm.tmem_base;
 
