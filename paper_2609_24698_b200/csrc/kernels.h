@@ -52,6 +52,10 @@ int launch_bsb(const tsv_shape& s, const tsv_cache& c, const tsv_nodes& nd, cons
 int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const int32_t* parent, const int32_t* n_nodes,
                const int32_t* draft, const int32_t* target, int32_t* accept_len, int32_t* accept_path,
                int32_t* bonus, int32_t* status, cudaStream_t st);
+// indexer scores of all nodes of a sequence as one small GEMM per tile of entries (bf16, 128-wide indexer rows, D * HI <= 32)
+bool idx_score_tc_applies(const tsv_shape& s);
+void launch_idx_score_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, char* ws,
+                         int32_t* status, cudaStream_t st);
 int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,

@@ -552,7 +552,9 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
     const int pref_cap = (int)(s.max_L / s.m_csa);
     dim3 grid((pref_cap + 255) / 256, s.B, s.D <= 8 ? s.D : 8);        // z: slabs of nodes, so a ranked sequence is scored by many CTAs
     const size_t sm = (size_t)32 * s.di * sizeof(float);
-    if (grid.x > 0 && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) {
+    if (grid.x > 0 && idx_score_tc_applies(s)) {
+      launch_idx_score_tc(s, p, c, nd, sc, ws, status, st);             // all nodes of a sequence at once, on the tensor core
+    } else if (grid.x > 0 && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) {
       const dim3 g8((pref_cap + kRows256PerCta - 1) / kRows256PerCta, s.B, s.D);   // one node per CTA: queries in registers
       if (bf) { TSV_PREP(idx_score_rows256_kernel<bf16>); idx_score_rows256_kernel<bf16><<<g8, 256, 0, st>>>(s, p, c, nd, sc, ws); }
       else { TSV_PREP(idx_score_rows256_kernel<float>); idx_score_rows256_kernel<float><<<g8, 256, 0, st>>>(s, p, c, nd, sc, ws); }
