@@ -5,10 +5,11 @@
 // For one sequence the inner products of ALL nodes and heads with a tile of entries are one small GEMM:
 //   [128 entries x 128 dims] x [128 dims x (D * HI <= 32) query rows]  ->  tcgen05.mma, M = 128, N = 32, K = 128, fp32 in TMEM.
 // An entry row is therefore read once per sequence instead of once per node.  A CTA walks kTilesPerCta tiles of 128
-// entries: the tile rows arrive by 16-byte cp.async into two 128-byte-swizzled K-major buffers (the next tile's copies are
-// issued before the previous tile's accumulator is read), thread 0 issues the eight MMAs of a tile, and the four warps
-// read the accumulator (lane = entry, column = node * HI + head), apply relu and the head weights and store one fp32
-// score per ranked node.  Several CTAs share an SM (73 KiB of shared memory, 64 TMEM columns each).
+// entries: the tile rows arrive by 16-byte cp.async into two 128-byte-swizzled K-major buffers (two tiles in flight: the
+// copies of tile t + 2 are issued as soon as the product of tile t is complete), thread 0 issues the eight MMAs of a
+// tile, and the four warps read the accumulator (lane = entry, column = node * HI + head), apply relu and the head
+// weights and store one fp32 score per ranked node.  Several CTAs share an SM (73 KiB of shared memory, 64 TMEM columns
+// each).
 #include "tc_common.cuh"
 
 namespace tsv {
@@ -98,6 +99,7 @@ __global__ void __launch_bounds__(kItThreads) idx_score_tc_kernel(const tsv_shap
     cp_commit();
   };
   load_tile(0);                                           // one group with the query rows
+  if (nt > 1) load_tile(1); else cp_commit();             // two tiles in flight from here on
   fence_before();
   __syncthreads();
   fence_after();
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(kItThreads) idx_score_tc_kernel(const tsv_shap
   };
 
   for (int t = 0; t < nt; ++t) {
-    cp_wait<0>();                                         // tile t (and the query rows) have landed: this thread's copies
+    cp_wait<1>();                                         // tile t (and the query rows) have landed: this thread's copies
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     fence_before();
     __syncthreads();                                      // everyone's copies; the accumulator buffer of tile t - 2 has been read
@@ -138,18 +140,13 @@ __global__ void __launch_bounds__(kItThreads) idx_score_tc_kernel(const tsv_shap
                  make_desc(bq + j * (kItN * 128) + ks * 32, 16, 1024), idesc, (j | ks) != 0);
       mma_commit(&sm.mma_bar[t & 1]);
     }
-    if (t >= 1) {                                         // tile t - 1 is complete: its buffer is free for tile t + 1
-      if (!fail && !mbar_wait(&sm.mma_bar[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u)) fail = 1;
-      fail = __any_sync(0xffffffffu, fail);               // warp-uniform: the accumulator loads are warp-collective
-      fence_after();
-    }
-    if (t + 1 < nt) load_tile(t + 1);
-    if (t >= 1 && !fail) epilogue(t - 1);
+    if (!fail && !mbar_wait(&sm.mma_bar[t & 1], (uint32_t)(t >> 1) & 1u)) fail = 1;
+    fail = __any_sync(0xffffffffu, fail);                 // warp-uniform: the accumulator loads are warp-collective
+    fence_after();
+    if (t + 2 < nt) load_tile(t + 2); else cp_commit();   // the tile's buffer is free again; one group per iteration either way
+    if (!fail) epilogue(t);
   }
-  if (!fail && !mbar_wait(&sm.mma_bar[(nt - 1) & 1], (uint32_t)((nt - 1) >> 1) & 1u)) fail = 1;
-  fail = __any_sync(0xffffffffu, fail);
-  fence_after();
-  if (!fail) epilogue(nt - 1);
+  cp_wait<0>();
   if (fail && lane == 0) atomicOr(status + b, TSV_ST_INTERNAL);
   fence_before();
   __syncthreads();
