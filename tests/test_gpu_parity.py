@@ -231,6 +231,16 @@ def test_long_candidate_lists_generic_scoring(dtype):
     lockstep(cfg, cycles=2)
 
 
+@pytest.mark.parametrize("D,HI", [(4, 8), (6, 2), (7, 1), (8, 4)])
+def test_long_candidate_lists_tensor_core_scoring(D, HI):
+    """More than 2048 candidates per node with 128-wide bf16 indexer rows: the scores of all nodes and heads come from
+    the tcgen05 scoring kernel (every head count it is built for; ragged last tiles, sequences on both sides of the
+    2304-candidate switch of the selection's key paths)."""
+    cfg = synth.small_config(name=f"long_lists_tc_d{D}_hi{HI}", dtype="bf16", B=3, D=D, H=4, d=16, m_csa=2, topk=24, HI=HI,
+                             di=128, m_hca=32, window=16, L_min=4200, L_max=5200, layers=1, seed=78 + HI, cfg_id=73)
+    lockstep(cfg, cycles=2)
+
+
 def test_ranked_short_candidate_lists_bf16():
     """Benchmark head shape with a small top-k: every node ranks its candidates, the lists are short enough to be scored
     inside the selection kernel (256-byte indexer rows), and the committed runs lie on both sides of 2 x topk, so ranked
