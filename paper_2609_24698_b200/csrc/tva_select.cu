@@ -183,6 +183,9 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
   }
 }
 
+// staging area of the rows a ranking CTA scores itself (256-byte indexer rows, padded in shared memory)
+constexpr int kStageRows = 128, kStagePitch = 272;   // two buffers of kStageRows rows
+
 template <typename T>
 __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
@@ -272,7 +275,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   if (pl.idx_fused) {
     // short candidate lists: the committed entries are scored here as well (same formula as idx_score_kernel: thread per
     // entry, the node's indexer queries in shared memory), into the score array the radix passes read
-    extern __shared__ float iq_sm[];                  // [HI][di]
+    extern __shared__ __align__(16) float iq_sm[];    // [HI][di], then the staged rows
     const int HI = s.HI, di = s.di;
     constexpr int V = Vec<T>::N;
     const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * HI * di;
@@ -281,10 +284,12 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
     float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
     if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
-      // Rows of 256 bytes (the benchmark's indexer width): eight lanes share an entry, each holding its 32-byte slice of
-      // the node's queries in registers for all entries; four entries of a group are in flight (few CTAs rank and global
-      // latency is long, so the number of dependent load rounds per thread is what counts: 4 here), and the per-head
-      // dot products are completed by three shuffles.
+      // Rows of 256 bytes (the benchmark's indexer width).  Few CTAs rank and each is a chain of its own, so what counts
+      // is how many bytes the CTA keeps in flight: the rows are staged in shared memory by 16-byte asynchronous copies,
+      // kStageRows rows per round in two buffers, the copies of the next round under the arithmetic of the current one.  Eight lanes
+      // then share an entry, lane l holding bytes [16 l, 16 l + 16) of both 128-byte halves of the node's queries in
+      // registers; the per-head dot products are completed by three shuffles.  Rows are padded by 16 bytes in shared
+      // memory so that the four entries a warp reads at a time fall into different banks.
       constexpr int EL = 2 * V;                        // row elements per lane
       const int grp = threadIdx.x >> 3, gl = threadIdx.x & 7;
       float q[4][EL], iwreg[4];
@@ -292,21 +297,39 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       for (int h = 0; h < 4; ++h) {
         iwreg[h] = h < HI ? nd.iw[((size_t)b * D + n) * HI + h] : 0.f;
 #pragma unroll
-        for (int j = 0; j < EL; ++j) q[h][j] = h < HI ? iq_sm[h * di + gl * EL + j] : 0.f;
+        for (int j = 0; j < EL; ++j) q[h][j] = h < HI ? iq_sm[h * di + (j < V ? gl * V + j : di / 2 + gl * V + (j - V))] : 0.f;
       }
-      for (int base = 0; base < n_csa; base += 128) {  // uniform trip count: the shuffles below need the whole warp
-        uint4 raw[4][2];
+      unsigned char* stage = reinterpret_cast<unsigned char*>(iq_sm + HI * di);
+      const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+      const char* ikb = reinterpret_cast<const char*>(ik0);
+      auto issue = [&](int rd) {                         // rows [rd kStageRows, ..) into buffer rd & 1; one group per call
+        const int base = rd * kStageRows, nrow = min(kStageRows, n_csa - base);
+        const uint32_t dst = stage_s + (uint32_t)(rd & 1) * (kStageRows * kStagePitch);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int e = base + grp + 32 * u;
-          const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)(e < n_csa ? e : 0) * di) + gl * 2;
-          raw[u][0] = __ldg(rowp); raw[u][1] = __ldg(rowp + 1);
+        for (int i = 0; i < kStageRows * 16 / 256; ++i) {
+          const int idx = threadIdx.x + 256 * i, row = idx >> 4, c16 = idx & 15;
+          if (row < nrow)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kStagePitch + c16 * 16),
+                         "l"(ikb + (size_t)(base + row) * 256 + c16 * 16) : "memory");
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      };
+      const int nrd = (n_csa + kStageRows - 1) / kStageRows;
+      issue(0);
+      for (int rd = 0; rd < nrd; ++rd) {                 // uniform trip count: barriers and shuffles below
+        if (rd + 1 < nrd) issue(rd + 1); else asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // round rd has landed (this thread's copies)
+        __syncthreads();
+        const int base = rd * kStageRows, nrow = min(kStageRows, n_csa - base);
+        const unsigned char* buf = stage + (size_t)(rd & 1) * (kStageRows * kStagePitch);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int r0 = 0; r0 < kStageRows; r0 += 32) {
+          const int row = r0 + grp;
+          const unsigned char* rp = buf + (row < nrow ? row : 0) * kStagePitch + gl * 16;
+          const uint4 lo = *reinterpret_cast<const uint4*>(rp), hi = *reinterpret_cast<const uint4*>(rp + 128);
           float kk[EL];
-          unpack16(raw[u][0], kk, (const T*)nullptr);
-          unpack16(raw[u][1], kk + V, (const T*)nullptr);
+          unpack16(lo, kk, (const T*)nullptr);
+          unpack16(hi, kk + V, (const T*)nullptr);
           float tot = 0.f;
 #pragma unroll
           for (int h = 0; h < 4; ++h) {
@@ -318,10 +341,11 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
             pp += __shfl_xor_sync(0xffffffffu, pp, 4);
             tot = fmaf(iwreg[h], fmaxf(pp, 0.f), tot);
           }
-          const int e = base + grp + 32 * u;
-          if (gl == 0 && e < n_csa) sw[e] = tot;
+          if (gl == 0 && row < nrow) sw[base + row] = tot;
         }
+        __syncthreads();                                 // the buffer is refilled two rounds on
       }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else
     for (int e = threadIdx.x; e < n_csa; e += blockDim.x) {
       float acc[8];
@@ -575,7 +599,12 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
   TSV_PREP(topk_kernel<bf16>);
   TSV_PREP(topk_kernel<float>);
-  const size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;   // the node's indexer queries
+  size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...
+  if (p.idx_fused && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) sm2 += (size_t)2 * kStageRows * kStagePitch;   // ... and the staged rows (two buffers)
+  if (sm2 > 48 * 1024) {
+    if (bf) cudaFuncSetAttribute(topk_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+    else cudaFuncSetAttribute(topk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+  }
   if (bf) topk_kernel<bf16><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
   else topk_kernel<float><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
   count_launch();
