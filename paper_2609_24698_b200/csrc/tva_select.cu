@@ -284,12 +284,11 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
     float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
     if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
-      // Rows of 256 bytes (the benchmark's indexer width).  Few CTAs rank and each is a chain of its own, so what counts
-      // is how many bytes the CTA keeps in flight: the rows are staged in shared memory by 16-byte asynchronous copies,
-      // kStageRows rows per round in two buffers, the copies of the next round under the arithmetic of the current one.  Eight lanes
-      // then share an entry, lane l holding bytes [16 l, 16 l + 16) of both 128-byte halves of the node's queries in
-      // registers; the per-head dot products are completed by three shuffles.  Rows are padded by 16 bytes in shared
-      // memory so that the four entries a warp reads at a time fall into different banks.
+      // Rows of 256 bytes (the benchmark's indexer width).  Few CTAs rank and each is a chain of its own, so load latency
+      // and arithmetic must not follow each other: the rows are staged in shared memory by 16-byte asynchronous copies,
+      // kStageRows rows per round in two buffers, the copies of the next round under the arithmetic of the current one.
+      // Eight lanes share an entry, lane l holding bytes [16 l, 16 l + 16) of both 128-byte halves of the node's
+      // queries in registers; the per-head dot products are completed by three shuffles.
       constexpr int EL = 2 * V;                        // row elements per lane
       const int grp = threadIdx.x >> 3, gl = threadIdx.x & 7;
       float q[4][EL], iwreg[4];
