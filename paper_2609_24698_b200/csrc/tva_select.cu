@@ -272,6 +272,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       if (lane == 0) extra[i] = tot;
     }
   }
+  const float* score_sm = nullptr;                    // scores of the committed entries in shared memory (set below), else in the workspace
   if (pl.idx_fused) {
     // short candidate lists: the committed entries are scored here as well (same formula as idx_score_kernel: thread per
     // entry, the node's indexer queries in shared memory), into the score array the radix passes read
@@ -299,6 +300,11 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
         for (int j = 0; j < EL; ++j) q[h][j] = h < HI ? iq_sm[h * di + (j < V ? gl * V + j : di / 2 + gl * V + (j - V))] : 0.f;
       }
       unsigned char* stage = reinterpret_cast<unsigned char*>(iq_sm + HI * di);
+      // the scores stay in shared memory: such a list has at most kIdxFusedMax + D candidates, which the radix passes
+      // below keep in registers, so nothing else reads them (written to and read back from global memory they cost a
+      // round trip of the chain)
+      float* ssm = reinterpret_cast<float*>(stage + 2 * kStageRows * kStagePitch);
+      score_sm = ssm;
       const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
       const char* ikb = reinterpret_cast<const char*>(ik0);
       auto issue = [&](int rd) {                         // rows [rd kStageRows, ..) into buffer rd & 1; one group per call
@@ -340,7 +346,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
             pp += __shfl_xor_sync(0xffffffffu, pp, 4);
             tot = fmaf(iwreg[h], fmaxf(pp, 0.f), tot);
           }
-          if (gl == 0 && row < nrow) sw[base + row] = tot;
+          if (gl == 0 && row < nrow) ssm[base + row] = tot;
         }
         __syncthreads();                                 // the buffer is refilled two rounds on
       }
@@ -386,13 +392,14 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   // order-preserving keys; lists of up to 9 x 256 candidates keep them in registers for the five passes below (candidate
   // i = threadIdx.x + 256 j is key j of its thread), longer lists read the scores again
   constexpr int KREG = 9;
+  static_assert(kIdxFusedMax + TSV_MAX_D <= KREG * 256, "lists scored in shared memory must fit the in-register key path");
   const bool in_regs = n_cand <= KREG * 256;
   uint32_t kreg[KREG];
   if (in_regs) {
 #pragma unroll
     for (int j = 0; j < KREG; ++j) {
       const int i = threadIdx.x + 256 * j;
-      kreg[j] = i < n_cand ? order_key(i < n_csa ? __ldcg(scores + i) : extra[i - n_csa]) : 0u;
+      kreg[j] = i < n_cand ? order_key(i < n_csa ? (score_sm ? score_sm[i] : __ldcg(scores + i)) : extra[i - n_csa]) : 0u;
     }
   }
   auto key_of = [&](int i) { return order_key(i < n_csa ? __ldcg(scores + i) : extra[i - n_csa]); };
@@ -599,7 +606,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   TSV_PREP(topk_kernel<bf16>);
   TSV_PREP(topk_kernel<float>);
   size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...
-  if (p.idx_fused && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) sm2 += (size_t)2 * kStageRows * kStagePitch;   // ... and the staged rows (two buffers)
+  if (p.idx_fused && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) sm2 += (size_t)2 * kStageRows * kStagePitch + (size_t)kIdxFusedMax * sizeof(float);   // ... the staged rows (two buffers), the scores
   if (sm2 > 48 * 1024) {
     if (bf) cudaFuncSetAttribute(topk_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
     else cudaFuncSetAttribute(topk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
