@@ -23,16 +23,30 @@ def _np(t):
 
 
 def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None, check_recompress=False,
-             parent_fn=None, return_engine=False):
+             parent_fn=None, return_engine=False, plant=None, graph=False, recompress_pairs=None, on_cycle=None,
+             per_row=False, incremental_caches=False):
     """Advance oracle and device cycle by cycle from the same prefix; compare everything each cycle.
-    out_pairs: None = compare attention outputs of every (layer, seq); else callable cycle -> iterable of pairs."""
+    out_pairs: None = compare attention outputs of every (layer, seq); else callable cycle -> iterable of pairs.
+    plant: callable(states, lengths) editing the oracle's prefix states in place before they are uploaded.
+    graph: the device cycle is ONE CUDA graph captured over a fixed input slot and replayed every cycle (the way the
+           benchmark runs it); the inputs of a cycle are copied into the slot before the replay.
+    check_recompress: True = every cycle, "final" = after the last cycle; recompress_pairs: callable cycle -> pairs
+           checked against recompression from scratch (None = all pairs).
+    on_cycle: callable(cycle, engine, states) for extra bookkeeping.
+    incremental_caches: per cycle compare only the cache rows appended in that cycle (plus lengths, window, open-block
+           states); all rows are compared after the last cycle and every tenth cycle.
+    per_row: also require every (node, head) output row to be within the tolerance of ITS OWN max magnitude (for inputs
+           where a few rows are far larger than the rest, so that the tensor-wide bound would say little about the others)."""
     from paper_2609_24698_b200 import binding as tsv, harness as hz
     sh = cfg.shape
     lengths = synth.prefix_lengths(cfg) if lengths is None else np.asarray(lengths)
     states = oracle_states(cfg, lengths)
+    if plant is not None:
+        plant(states, lengths)
     committed = None
     if check_recompress:
-        committed = [[dict(synth.prefix_tokens(cfg, l, b, int(lengths[b]))) for b in range(sh.B)] for l in range(cfg.layers)]
+        committed = [[{k: [v] for k, v in synth.prefix_tokens(cfg, l, b, int(lengths[b])).items()} for b in range(sh.B)]
+                     for l in range(cfg.layers)]                 # per tensor: list of pieces, joined when checked
     ccap, hcap = hz.capacities(sh, lengths, cycles * sh.D)
     max_L = int(lengths.max()) + (cycles + 1) * sh.D
     eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=True)
@@ -41,6 +55,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
             hz.fill_cache(eng.caches[l], sh, b, int(lengths[b]), state_arrays(states[l][b]))
     tol = TOL[sh.dtype]
     worst = 0.0
+    slot = graph_obj = None
     for cyc in range(cycles):
         nodes = [synth.node_inputs(cfg, l, cyc) for l in range(cfg.layers)]
         parent, n_nodes = synth.trees(cfg, cyc)
@@ -50,17 +65,33 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
             n_nodes = n_nodes_fn(cyc, n_nodes)
         draft, target = synth.tokens(cfg, cyc, parent, n_nodes)
         inp = hz.InputSet.from_numpy(sh, nodes, parent, n_nodes, draft, target)
-        before = eng.snapshot()
-        eng.launch_cycle(inp, refresh=False)
-        torch.cuda.synchronize()
-        # isolation: the first two calls leave every persistent byte unchanged
-        for c0, c1 in zip(before, eng.caches):
-            for name in tsv.CACHE_TENSORS:
-                assert torch.equal(getattr(c0, name), getattr(c1, name)), f"{name} changed before acceptance"
-        tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path,
-                               eng.bonus, eng.status)
-        torch.cuda.synchronize()
+        if graph:
+            if slot is None:
+                slot = hz.InputSet.empty(sh, cfg.layers)
+                for d_, s_ in zip(slot.tensors(), inp.tensors()):
+                    d_.copy_(s_)
+                snap = eng.snapshot()
+                eng.launch_cycle(slot)                     # eager warm-up on the same inputs, then back to the prefix
+                torch.cuda.synchronize()
+                eng.restore(snap)
+                graph_obj = eng.capture(slot)
+            for d_, s_ in zip(slot.tensors(), inp.tensors()):
+                d_.copy_(s_)
+            graph_obj.replay()
+            torch.cuda.synchronize()
+        else:
+            before = eng.snapshot()
+            eng.launch_cycle(inp, refresh=False)
+            torch.cuda.synchronize()
+            # isolation: the first two calls leave every persistent byte unchanged
+            for c0, c1 in zip(before, eng.caches):
+                for name in tsv.CACHE_TENSORS:
+                    assert torch.equal(getattr(c0, name), getattr(c1, name)), f"{name} changed before acceptance"
+            tsv.accept_and_refresh(eng.cshape, eng._pack(inp), inp.draft, inp.target, eng.accept_len, eng.accept_path,
+                                   eng.bonus, eng.status)
+            torch.cuda.synchronize()
         assert int(eng.status.abs().sum()) == 0, f"cycle {cyc}: status flags {eng.status.cpu().tolist()}"
+        prev_L = [[S.L for S in states[l]] for l in range(cfg.layers)]
         pairs = [(l, b) for l in range(cfg.layers) for b in range(sh.B)] if out_pairs is None else list(out_pairs(cyc))
         g_alen, g_path, g_bonus = eng.accept_len.cpu().numpy(), eng.accept_path.cpu().numpy(), eng.bonus.cpu().numpy()
         scs = {}
@@ -90,6 +121,12 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
             if not same:       # inside the tie band: evaluate the oracle with the device's selection
                 ref_out, _ = O.tree_verify_attn(states[l][b], sh, nb, parent[b], nn, scs[(l, b)], forced_sel=[g_idx[n] for n in range(nn)])
             e = rel_err(_np(eng.out[l][b]), ref_out)
+            if per_row:
+                g_out = _np(eng.out[l][b])
+                for n in range(nn):
+                    for h in range(sh.H):
+                        er = rel_err(g_out[n, h], ref_out[n, h])
+                        assert er <= tol, f"cycle {cyc} layer {l} seq {b} node {n} head {h}: row error {er:.3e} > {tol}"
             worst = max(worst, e)
             assert e <= tol, f"cycle {cyc} layer {l} seq {b}: attention output error {e:.3e} > {tol}"
             assert not _np(eng.out[l][b])[nn:].any()
@@ -102,23 +139,47 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
                 O.refresh(states[l][b], sh, per_seq(nodes[l], b), scs[(l, b)], path)
                 if committed is not None:
                     for k in committed[l][b]:
-                        committed[l][b][k] = np.concatenate([committed[l][b][k], nodes[l][k][b][path]], 0)
-        compare_caches(eng, states, sh, tol, committed if (check_recompress is True or cyc == cycles - 1) else None)
+                        committed[l][b][k].append(nodes[l][k][b][path])
+        rp = None if recompress_pairs is None else set(recompress_pairs(cyc))
+        full = not incremental_caches or cyc == cycles - 1 or cyc % 10 == 9
+        compare_caches(eng, states, sh, tol, committed if (check_recompress is True or cyc == cycles - 1) else None,
+                       None if cyc == cycles - 1 else rp, None if full else prev_L)
+        if on_cycle is not None:
+            on_cycle(cyc, eng, states)
     return (worst, eng, states) if return_engine else worst
 
 
-def compare_caches(eng, states, sh, tol, committed=None):
+def compare_caches(eng, states, sh, tol, committed=None, recompress_pairs=None, prev_L=None):
+    """Device caches against the oracle states.  prev_L[l][b] (committed lengths before this cycle): compare only the
+    entries appended since then (full-size runs; a later full comparison covers the untouched rows)."""
     for l, cache in enumerate(eng.caches):
         Ls = cache.L.cpu().numpy()
         r0c, r0h = cache.csa_row0.cpu().numpy(), cache.hca_row0.cpu().numpy()
-        ckv, cik, hkv, win = _np(cache.csa_kv), _np(cache.csa_ik), _np(cache.hca_kv), _np(cache.win_kv)
+        win = _np(cache.win_kv)
         f = {k: _np(getattr(cache, k)) for k in ("csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")}
+        lo_c = [0 if prev_L is None else prev_L[l][b] // sh.m_csa for b in range(sh.B)]
+        lo_h = [0 if prev_L is None else prev_L[l][b] // sh.m_hca for b in range(sh.B)]
+        if prev_L is None:
+            ckv, cik, hkv = _np(cache.csa_kv), _np(cache.csa_ik), _np(cache.hca_kv)
+            row_c = lambda b, i: r0c[b] + i
+            row_h = lambda b, i: r0h[b] + i
+        else:                                                                     # gather only the appended rows
+            ic = [int(r0c[b]) + i for b, S in enumerate(states[l]) for i in range(lo_c[b], S.L // sh.m_csa)]
+            ih = [int(r0h[b]) + i for b, S in enumerate(states[l]) for i in range(lo_h[b], S.L // sh.m_hca)]
+            tc_ = torch.tensor(ic, dtype=torch.long, device=cache.csa_kv.device)
+            th_ = torch.tensor(ih, dtype=torch.long, device=cache.csa_kv.device)
+            ckv, cik, hkv = _np(cache.csa_kv[tc_]), _np(cache.csa_ik[tc_]), _np(cache.hca_kv[th_])
+            pc_, ph_ = {r: j for j, r in enumerate(ic)}, {r: j for j, r in enumerate(ih)}
+            row_c = lambda b, i: pc_[int(r0c[b]) + i]
+            row_h = lambda b, i: ph_[int(r0h[b]) + i]
         for b, S in enumerate(states[l]):
             assert int(Ls[b]) == S.L                                            # committed length: exact
             n_csa, n_hca = S.L // sh.m_csa, S.L // sh.m_hca
             assert S.csa_kv.shape[0] == n_csa and S.hca_kv.shape[0] == n_hca      # entry indices: exact
-            assert rel_err(ckv[r0c[b]:r0c[b] + n_csa], S.csa_kv) <= tol and rel_err(cik[r0c[b]:r0c[b] + n_csa], S.csa_ik) <= tol
-            assert rel_err(hkv[r0h[b]:r0h[b] + n_hca], S.hca_kv) <= tol
+            rc = [row_c(b, i) for i in range(lo_c[b], n_csa)]
+            rh = [row_h(b, i) for i in range(lo_h[b], n_hca)]
+            assert rel_err(ckv[rc], S.csa_kv[lo_c[b]:]) <= tol and rel_err(cik[rc], S.csa_ik[lo_c[b]:]) <= tol
+            assert rel_err(hkv[rh], S.hca_kv[lo_h[b]:]) <= tol
             assert np.array_equal(win[b], S.win)                                 # token-level KV: copies, exact
             assert f["csa_mx"][b] == S.csa_part.mx and f["hca_mx"][b] == S.hca_part.mx
             assert abs(f["csa_s"][b] - S.csa_part.s) <= TOL_STATE * max(1.0, S.csa_part.s)
@@ -126,8 +187,8 @@ def compare_caches(eng, states, sh, tol, committed=None):
             assert rel_err(f["csa_acc_kv"][b], S.csa_part.acc[0]) <= TOL_STATE or not S.csa_part.acc[0].any()
             assert rel_err(f["csa_acc_ik"][b], S.csa_part.acc[1]) <= TOL_STATE or not S.csa_part.acc[1].any()
             assert rel_err(f["hca_acc_kv"][b], S.hca_part.acc[0]) <= TOL_STATE or not S.hca_part.acc[0].any()
-            if committed is not None:                                            # oracle state == recompression from scratch
-                states_close(S, O.recompress_from_scratch(sh, committed[l][b]), tol=1e-9)
+            if committed is not None and (recompress_pairs is None or (l, b) in recompress_pairs):   # oracle state == recompression from scratch
+                states_close(S, O.recompress_from_scratch(sh, {k: np.concatenate(v, 0) for k, v in committed[l][b].items()}), tol=1e-9)
 
 
 # ------------------------------------------------------------------------------------------------ small shapes, every edge
@@ -196,22 +257,55 @@ def test_cfg3_peaked():
     lockstep(cfg, cycles=2)
 
 
-def test_cfg4_full_size_stack_lockstep():
-    """8 layers x 64 sequences, the launch configuration the benchmark times.  Every cycle: branch states,
-    acceptance, committed caches of ALL (layer, sequence) pairs; attention outputs of all pairs on cycle 0 and of
-    a rotating sample later; recompression-from-scratch check of every pair after the last cycle."""
+def test_cfg4_full_size_stack_50_cycles():
+    """8 layers x 64 sequences, the launch configuration the benchmark times, 50 verify cycles back to back.  Every
+    cycle: branch states and closed entries, acceptance, committed lengths, appended cache rows, window and open-block
+    states of ALL 512 (layer, sequence) pairs; the refreshed state of a rotating sample of 48 pairs (all pairs after
+    the last cycle) against recompression of the committed tokens from scratch; attention outputs of all pairs on the
+    first and the last cycle (by then several sequences have more than top-k candidates and rank) and of a rotating
+    sample of 16 pairs plus the longest sequence in between."""
     cfg = synth.CONFIGS["cfg4"]
+    sh = cfg.shape
     rng = np.random.default_rng(4)
+    longest = int(np.argmax(synth.prefix_lengths(cfg)))
+    everyone = [(l, b) for l in range(cfg.layers) for b in range(sh.B)]
     def pairs(cyc):
-        if cyc == 0:
-            return [(l, b) for l in range(cfg.layers) for b in range(cfg.shape.B)]
-        return [(int(rng.integers(0, cfg.layers)), int(rng.integers(0, cfg.shape.B))) for _ in range(24)]
-    lockstep(cfg, cycles=5, out_pairs=pairs, check_recompress="final")
+        if cyc in (0, cfg.cycles - 1):
+            return everyone
+        return [(int(rng.integers(0, cfg.layers)), int(rng.integers(0, sh.B))) for _ in range(16)] + [(cyc % cfg.layers, longest)]
+    def rpairs(cyc):
+        return [(int(rng.integers(0, cfg.layers)), int(rng.integers(0, sh.B))) for _ in range(48)]
+    ranked = []
+    def watch(cyc, eng, states):
+        ranked.append(sum(S.L // sh.m_csa > sh.topk for S in states[0]))
+    lockstep(cfg, cycles=cfg.cycles, out_pairs=pairs, check_recompress=True, recompress_pairs=rpairs, incremental_caches=True,
+             on_cycle=watch)
+    assert cfg.cycles == 50 and ranked[-1] >= 2, "the run is meant to end with sequences past top-k candidates"
 
 
-def test_cfg5_long_context():
-    """131072-token prefixes, top-k 2048 of 32768 candidates: ranked selection, split key lists, combine."""
-    lockstep(synth.CONFIGS["cfg5"], cycles=3, check_recompress="final")
+def test_cfg5_long_context_100_cycles():
+    """131072-token prefixes, top-k 2048 of 32768 candidates, 100 verify-accept-refresh cycles: branch states,
+    acceptance and caches every cycle; attention outputs and selections on cycles 0, 1, 2, then every 16th and the
+    last; recompression from scratch after the last cycle.  The bytes the method must read per cycle are tracked
+    from the evolving lengths and selections (they may only grow with the prefix)."""
+    cfg = synth.CONFIGS["cfg5"]
+    sh = cfg.shape
+    everyone = [(0, b) for b in range(sh.B)]
+    track = []
+    def watch(cyc, eng, states):
+        es = 2
+        per_cycle = 0
+        idx = eng.topk_idx[0].cpu().numpy()
+        for b, S in enumerate(states[0]):
+            union = np.unique(idx[b][idx[b] >= 0]).size
+            n_csa_before = (S.L - int(eng.accept_len[b])) // sh.m_csa
+            per_cycle += (n_csa_before * sh.di + (union + S.hca_kv.shape[0] + sh.window + sh.D) * sh.d) * es
+        track.append(per_cycle)
+    lockstep(cfg, cycles=cfg.cycles, out_pairs=lambda c: everyone if (c < 3 or c % 16 == 0 or c == cfg.cycles - 1) else [],
+             check_recompress="final", incremental_caches=True, on_cycle=watch)
+    assert cfg.cycles == 100 and len(track) == 100
+    # indexer keys of all 32768+ entries and the union of the nodes' selections dominate: tens of MB, slowly growing
+    assert 40e6 < track[0] < 120e6 and track[-1] >= track[0] - 8e6
 
 
 @pytest.mark.parametrize("D,B", [(5, 1), (6, 2), (7, 64), (8, 4)])
@@ -249,6 +343,91 @@ def test_ranked_short_candidate_lists_bf16():
                        L_min=300, L_max=1400, seed=9)
     lockstep(cfg, cycles=2)
 
+
+
+# ------------------------------------------------------------------------------------------------ tensor-core path, peaked softmax
+BENCH_HEADS = dict(H=64, d=512, m_csa=4, HI=4, di=128, m_hca=128, window=128)
+
+
+def _plant_peaks(cfg, gap_nats=14.0):
+    """Returns a `plant` hook: into late window rows of every sequence it writes c * q/|q| of chosen (node, head) queries of
+    cycle 0, c such that this key's logit lies `gap_nats` above the (near-zero) logits of all other keys.  The window run
+    comes after the CSA run in a tile's key list, so these keys fall into the second or third 256-key piece of a chunk
+    (or into a later chunk): the row's running maximum jumps by more than the kernel's rescale threshold there.
+      position L-1    <- query of (node 3, head 5): visible to every node
+      position L-126  <- query of (deepest node, head 7): visible to depths <= 1 only, i.e. MASKED for the row it matches
+      position L-125  <- query of (root, head 9): visible to depths <= 2"""
+    sh = cfg.shape
+    def hook(states, lengths):
+        parent, n_nodes = synth.trees(cfg, 0)
+        for l in range(cfg.layers):
+            nodes = synth.node_inputs(cfg, l, 0)
+            for b, S in enumerate(states[l]):
+                depth = O.tree_depth(parent[b], int(n_nodes[b]))
+                deep = int(np.argmax(depth))
+                assert depth[deep] >= 2
+                for pos, (n, h) in ((S.L - 1, (3, 5)), (S.L - 126, (deep, 7)), (S.L - 125, (0, 9))):
+                    q = nodes["q"][b, n, h].astype(np.float64)
+                    c = gap_nats / (sh.scale * np.linalg.norm(q))
+                    S.win[pos % sh.window] = synth.quantize(c * q / np.linalg.norm(q), sh.dtype).astype(np.float64)
+    return hook
+
+
+def test_tc_planted_peaks_reach_rescale_and_merge_paths():
+    """Benchmark head shape.  Sequence lengths put the planted window keys into: the second piece of a single-chunk
+    tile (1200), the third piece (2040), a later chunk of a multi-chunk tile on the contiguous-run path (3500:
+    n_csa <= 2 topk), and a later chunk of the pointer-gather kernel (5000: n_csa > 2 topk)."""
+    cfg = synth.Config("tc_peaks", 81, synth.Shape("bf16", 5, 8, topk=512, **BENCH_HEADS), L_min=1, L_max=1, seed=3)
+    lockstep(cfg, cycles=1, lengths=[1200, 2040, 1660, 3500, 5000], plant=_plant_peaks(cfg), per_row=True)
+
+
+def test_tc_planted_peaks_ranked_tiles():
+    """Same planted keys with a small top-k, so that every node ranks: masked-run tiles (n_csa <= 2 topk) and
+    pointer-gather tiles, single- and multi-chunk."""
+    cfg = synth.Config("tc_peaks_ranked", 82, synth.Shape("bf16", 4, 8, topk=256, **BENCH_HEADS), L_min=1, L_max=1, seed=4)
+    lockstep(cfg, cycles=1, lengths=[1500, 2040, 2600, 4400], plant=_plant_peaks(cfg, gap_nats=16.0), per_row=True)
+
+
+def test_tc_peaked_scale100():
+    """sm_scale = 100 on the d = 512 path: logits are O(+-5) everywhere, so one wrongly masked or dropped key moves an
+    output row by far more than the tolerance.  Lengths cover single-chunk, multi-chunk and pointer-gather tiles."""
+    cfg = synth.Config("tc_scale100", 83, synth.Shape("bf16", 6, 8, topk=512, sm_scale=100.0, **BENCH_HEADS), L_min=1, L_max=1, seed=5)
+    lockstep(cfg, cycles=2, lengths=[300, 900, 1400, 2047, 3300, 4700], per_row=True)
+
+
+@pytest.mark.parametrize("H,D,B", [(32, 16, 3), (128, 8, 3), (64, 12, 3), (64, 16, 2), (32, 5, 2)])
+def test_tc_other_head_counts_and_budgets(H, D, B):
+    """The tensor-core path takes H in {32, 64, 128} and budgets up to 32 nodes: 8, 4 or 2 nodes per 256-row tile, up to
+    four tiles per sequence, partial last tiles; blocks closing inside the deeper trees."""
+    sh = synth.Shape("bf16", B, D, H, 512, 4, 512, 4, 128, 128, 128, sm_scale=8.0)
+    cfg = synth.Config(f"tc_h{H}_d{D}", 84, sh, L_min=250, L_max=2300, seed=H + D)
+    lockstep(cfg, cycles=2, per_row=True)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_budgets_beyond_eight_cuda_core_path(dtype):
+    """D = 12 and D = 16 on the CUDA-core path (d = 64): deeper trees close several CSA and HCA blocks inside the tree."""
+    for D in (12, 16):
+        cfg = synth.small_config(name=f"simt_d{D}", dtype=dtype, B=3, D=D, H=6, d=64, m_csa=2, topk=12, HI=2, di=16, m_hca=5,
+                                 window=20, L_min=30, L_max=200, layers=1, seed=90 + D, cfg_id=85, sm_scale=3.0)
+        lockstep(cfg, cycles=3, check_recompress=True)
+
+
+# ------------------------------------------------------------------------------------------------ the cycle as the benchmark runs it
+def test_graph_replayed_cycles_match_oracle_and_eager():
+    """One CUDA graph captured over a fixed input slot and replayed for four cycles (fresh inputs copied into the slot each
+    time), 2 layers on the benchmark head shape: branch states, outputs, selections, acceptance and refreshed caches
+    against the oracle every cycle; then bit-equality of outputs, selections, acceptance and caches with an engine that
+    ran the same four cycles eagerly."""
+    cfg = synth.Config("graph_cycle", 86, synth.Shape("bf16", 6, 8, topk=512, **BENCH_HEADS), layers=2, L_min=200, L_max=2600, seed=6)
+    _, eng_g, _ = lockstep(cfg, cycles=4, graph=True, return_engine=True, check_recompress=True)
+    _, eng_e, _ = lockstep(cfg, cycles=4, return_engine=True)
+    from paper_2609_24698_b200 import binding as tsv
+    for l in range(cfg.layers):
+        assert torch.equal(eng_g.out[l], eng_e.out[l]) and torch.equal(eng_g.topk_idx[l], eng_e.topk_idx[l])
+        for name in tsv.CACHE_TENSORS:
+            assert torch.equal(getattr(eng_g.caches[l], name), getattr(eng_e.caches[l], name)), name
+    assert torch.equal(eng_g.accept_path, eng_e.accept_path) and torch.equal(eng_g.accept_len, eng_e.accept_len)
 
 # ------------------------------------------------------------------------------------------------ status / error paths
 def test_device_detected_errors_commit_nothing():
