@@ -27,9 +27,15 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one tc_attn_pair_kernel launch on one layer of the bench workload
-# (ncu capture summarised in profiles/ncu_tc_attn_pair_kernel_cfg4.md): 65.41 MB read + 4.85 MB written.
-NCU_ATTN_TRAFFIC_BYTES = 70_262_784
+# Measured DRAM traffic (ncu: dram__bytes_read.sum + dram__bytes_write.sum), per workload: the dominant kernel of the
+# attention stage with the bytes of ONE of its launches (one layer), and, where captured, the sum over all kernels of one
+# verify cycle.  The captures are summarised under profiles/; workloads without a capture report null.
+NCU_DRAM = {
+    "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 70_262_784, "cycle_bytes": None},   # 65.41 MB read + 4.85 MB written
+}
+ATTN_KERNEL = {"cfg1": "attn_simt_kernel (fp32 CUDA-core path)", "cfg2": "tc_attn_pair_kernel", "cfg2_chain": "tc_attn_pair_kernel",
+               "cfg3": "tc_attn_pair_kernel + tc_attn_kernel (pointer gather) + tc_combine_kernel", "cfg4": "tc_attn_pair_kernel",
+               "cfg5": "tc_attn_kernel (pointer gather) + tc_combine_kernel"}
 
 
 def peaks():
@@ -87,8 +93,8 @@ def oracle_sample(cfg, n_layers_sample: int, n_seq_sample: int, steps: int, warm
     n_seq_sample sequences x n_layers_sample layers of the same seeded inputs, one verify cycle per step.
     Returns verified tokens/s scaled to the full layer count, and a description of the sample."""
     from oracle import tsv_oracle as O
-    from paper_2609_24698_b200 import synth
-    from paper_2609_24698_b200.workload import direct_arrays
+    from paper_2609_24698_b200 import synth      # (synth only: the CUDA library is not loaded into the oracle's process)
+    direct_arrays = synth.direct_arrays
     sh = cfg.shape
     lengths = synth.prefix_lengths(cfg)
 
@@ -106,7 +112,7 @@ def oracle_sample(cfg, n_layers_sample: int, n_seq_sample: int, steps: int, warm
         return st
 
     states = fresh_states()
-    times = []
+    times, cpu_times = [], []
     n_sets = min(3, warmup + steps)
     node_sets = [[{k: v[:n_seq_sample] for k, v in synth.node_inputs(cfg, l, c).items()} for l in range(n_layers_sample)]
                  for c in range(n_sets)]
@@ -115,18 +121,16 @@ def oracle_sample(cfg, n_layers_sample: int, n_seq_sample: int, steps: int, warm
         nodes = node_sets[c]
         parent, n_nodes = synth.trees(cfg, c)
         draft, target = synth.tokens(cfg, c, parent, n_nodes)
-        t0 = time.perf_counter()
+        t0, c0 = time.perf_counter(), time.process_time()
         O.verify_cycle(states, sh, nodes, parent[:n_seq_sample], n_nodes[:n_seq_sample], draft[:n_seq_sample], target[:n_seq_sample])
-        dt = time.perf_counter() - t0
+        dt, dc = time.perf_counter() - t0, time.process_time() - c0
         if it >= warmup:
-            times.append(dt)
+            times.append(dt); cpu_times.append(dc)
     t_cycle_full_layers = float(np.mean(times)) * cfg.layers / n_layers_sample
     tok_s = n_seq_sample * sh.D / t_cycle_full_layers
-    try:
-        import threadpoolctl
-        cores = max([p["num_threads"] for p in threadpoolctl.threadpool_info()] + [1])
-    except Exception:
-        cores = os.cpu_count() or 1
+    # cores the oracle keeps busy: CPU time of the process (all threads) over wall time; the oracle is mostly Python loops
+    # around numpy calls, so this is close to 1 however many threads the BLAS pool holds
+    cores = max(1, int(round(float(np.sum(cpu_times)) / max(float(np.sum(times)), 1e-9))))
     sample = (f"{n_seq_sample} of {sh.B} sequences x {n_layers_sample} of {cfg.layers} layers of {cfg.name}, "
               f"{steps} verify cycles (mean {np.mean(times):.3f} s each), time scaled to {cfg.layers} layers")
     return tok_s, float(np.mean(times)) * 1e3, cores, sample
@@ -217,8 +221,6 @@ def run_ours(args, cfg):
     # CUDA events on the launching stream.  Graph replay keeps the host out of the measurement; the attention stage is
     # tree_verify_attn without its selection step (tile plan + paired attention kernel + merge of multi-chunk tiles).
     eng.restore(snap)
-    sel_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_ATTN)
-    att_shape = tsv.c_shape(sh, eng.cshape.max_L, tsv.FLAG_SKIP_SELECT)
     inp0 = wl.inputs[0]
     eng.launch_cycle(inp0, refresh=False)           # scratch pads and selections of inp0 are in place for the partial graphs
     torch.cuda.synchronize()
@@ -229,9 +231,11 @@ def run_ours(args, cfg):
                 if name == "branch_state_build":
                     tsv.branch_state_build(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.status)
                 elif name == "select":
-                    tsv.tree_verify_attn(sel_shape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+                    tsv.bench_tree_verify_attn_stages(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None,
+                                                      eng.workspace, eng.status, tsv.STAGE_SELECT)
                 elif name == "attention":
-                    tsv.tree_verify_attn(att_shape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None, eng.workspace, eng.status)
+                    tsv.bench_tree_verify_attn_stages(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None,
+                                                      eng.workspace, eng.status, tsv.STAGE_ATTENTION)
         return f
 
     t_parts = {}
@@ -264,17 +268,30 @@ def run_ours(args, cfg):
     pk = peaks()
     attn_gbs = work["attn_bytes_per_layer"] / (attn_ms * 1e-3) / 1e9
     attn_tf = work["attn_flops_per_layer"] / (attn_ms * 1e-3) / 1e12
-    roofline = {"bound": "hbm", "kernel": "tree_verify_attn attention stage: tile plan + tc_attn_pair_kernel (one layer, all sequences)",
-                "achieved": attn_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / pk["hbm_gbs"],
-                "traffic": NCU_ATTN_TRAFFIC_BYTES, "peak_source": pk["source"], "launch_ms": attn_ms,
-                "algorithmic_bytes_per_launch": work["attn_bytes_per_layer"],
-                "tensor": {"achieved": attn_tf, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                           "frac": attn_tf / pk["bf16_tflops_sustained"], "flops_per_launch": work["attn_flops_per_layer"]}}
+    hbm = {"achieved": attn_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / pk["hbm_gbs"],
+           "algorithmic_bytes_per_launch": work["attn_bytes_per_layer"]}
+    tensor = {"achieved": attn_tf, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": attn_tf / pk["bf16_tflops_sustained"],
+              "flops_per_launch": work["attn_flops_per_layer"]}
+    # which roof governs: the stage's FLOP per algorithmic byte against the ridge of the measured peaks (fp32 storage runs
+    # on the CUDA cores and is judged against the memory roof)
+    ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
+    intensity = work["attn_flops_per_layer"] / work["attn_bytes_per_layer"]
+    bound = "tensor" if (sh.dtype == "bf16" and intensity > ridge) else "hbm"
+    cap = NCU_DRAM.get(cfg.name)
+    roofline = {"bound": bound, "kernel": f"tree_verify_attn attention stage (tile plan + {ATTN_KERNEL.get(cfg.name, 'attention kernels')}), "
+                                          "one layer, all sequences",
+                **(tensor if bound == "tensor" else hbm),
+                "traffic": cap["launch_bytes"] if cap else None,
+                "traffic_note": (f"ncu DRAM read+write of one {cap['kernel']} launch on this workload" if cap else "no ncu capture for this workload"),
+                "peak_source": pk["source"], "launch_ms": attn_ms, "flop_per_byte": intensity, "ridge_flop_per_byte": ridge,
+                "lengths": "algorithmic bytes and FLOPs from the initial prefix lengths (the caches grow by the accepted tokens while timed)",
+                "hbm": hbm, "tensor": tensor}
     cycle_s = sec / K
     cycle = {"full_bytes": work["full_bytes"], "cache_bytes": work["cache_bytes"], "flops": work["flops"],
              "frac_hbm_full": work["full_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
              "frac_hbm_cache": work["cache_bytes"] / cycle_s / 1e9 / pk["hbm_gbs"],
              "frac_tensor_sustained": work["flops"] / cycle_s / 1e12 / pk["bf16_tflops_sustained"],
+             "measured_dram_bytes": cap["cycle_bytes"] if cap else None,
              "stage_ms_per_layer_call": {k: float(v) for k, v in t_parts.items()},
              "accepted_tokens_per_cycle_last": accepted}
 

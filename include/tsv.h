@@ -11,8 +11,12 @@
  *   - Every `void*` / typed pointer inside the structs is a DEVICE pointer unless the
  *     comment says HOST.  The structs themselves and `tsv_shape` live in HOST memory and
  *     are read during the call only.
- *   - The caller owns every buffer.  The library allocates nothing, keeps no state between
- *     calls and never synchronises: all work is enqueued on `stream` and the call returns.
+ *   - The caller owns every buffer.  The library allocates nothing and never synchronises: all
+ *     work is enqueued on `stream` and the call returns.  Between calls it keeps nothing of the
+ *     caller's data; what it does keep per process is set-up it does once (kernel attributes,
+ *     the number of CTA pairs a device holds, the driver entry point for tensor maps), the
+ *     launch counter behind tsv_kernel_launches(), and for tree_verify_attn_static the
+ *     address of its built-in array.
  *   - "storage dtype" = tsv_shape.dtype (fp32 or bf16): all vectors and cache rows.  All
  *     partial-block accumulators, gates and weights are fp32.
  *   - Row-major, innermost dimension contiguous, no padding.  Vector pointers must be
@@ -23,7 +27,10 @@
  *   - Node n of sequence b sits at depth delta_n (root = node 0 = depth 0) and at position
  *     p_n = L[b] + delta_n.  n_csa = L / m_csa and n_hca = L / m_hca committed entries.
  *   - Return value: 0 or a negative TSV_ERR_* for problems the host can see BEFORE any
- *     launch (nothing is enqueued then).  Problems only the device can see (bad parent
+ *     launch (nothing is enqueued then: argument checks, tensor-map encoding and kernel
+ *     attributes all precede the first launch).  Only a failing kernel launch itself
+ *     (TSV_ERR_CUDA out of cudaLaunchKernel) can leave earlier kernels of the same call
+ *     enqueued; skip accept_and_refresh for that cycle then.  Problems only the device can see (bad parent
  *     array, node count, capacity, length) are reported per sequence in `status[b]`
  *     (bit-or of TSV_ST_*): that sequence's outputs are zero-filled and
  *     accept_and_refresh commits nothing for it (L unchanged).  `status` is or-ed into, never
@@ -63,11 +70,8 @@ enum {                         /* per-sequence status bits, device-written */
 };
 
 enum {                         /* tsv_shape.flags */
-  TSV_FLAG_FORCE_SIMT = 1,    /* tree_verify_attn: use the CUDA-core kernels even where the
+  TSV_FLAG_FORCE_SIMT = 1     /* tree_verify_attn: use the CUDA-core kernels even where the
                                   tensor-core kernels apply                                 */
-  TSV_FLAG_SKIP_SELECT = 2,   /* tree_verify_attn (profiling aid): skip the CSA selection and reuse the
-                                  one a previous call on the same inputs left in `workspace`  */
-  TSV_FLAG_SKIP_ATTN = 4      /* tree_verify_attn (profiling aid): selection only, `out` untouched */
 };
 
 /* Problem shape; HOST memory.
@@ -228,7 +232,10 @@ int accept_and_refresh(const tsv_shape *shape, int32_t n_layers, const tsv_cache
  *   - Shapes whose tsv_workspace_bytes() exceeds TSV_STATIC_WORKSPACE_BYTES are refused with
  *     TSV_ERR_LIMIT and nothing is enqueued.
  *   - The first call on each device looks up the array's device address (with that device
- *     current).  Make that first call before starting any stream capture.
+ *     current); that look-up makes the runtime load the library's device code on the device,
+ *     which is when the array's bytes are reserved there.  Make that first call at start-up:
+ *     before the rest of the device memory is handed out, and before starting any stream capture.
+ *     If it fails (TSV_ERR_CUDA), nothing was enqueued and no error is left pending.
  *   - All calls on a device share the one array, which keeps whatever the last call left in
  *     it.  Nothing in it has to start at zero -- every region is written before it is read
  *     within a call -- but two calls that overlap on the GPU (different streams, no

@@ -24,7 +24,8 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 TSV_FP32, TSV_BF16 = 0, 1
-FLAG_FORCE_SIMT, FLAG_SKIP_SELECT, FLAG_SKIP_ATTN = 1, 2, 4
+FLAG_FORCE_SIMT = 1
+STAGE_SELECT, STAGE_ATTENTION = 1, 2      # stages of tree_verify_attn for bench_tree_verify_attn_stages
 ST_NODES, ST_PARENT, ST_LENGTH, ST_CSA_CAP, ST_HCA_CAP, ST_INTERNAL = 1, 2, 4, 8, 16, 32
 ERR_NULL, ERR_ALIGN, ERR_SHAPE, ERR_WORKSPACE, ERR_CUDA, ERR_LIMIT = -1, -2, -3, -4, -5, -6
 
@@ -231,6 +232,25 @@ def tree_verify_attn(shape: CShape, cache: LayerCache, nodes: NodeInputs, scratc
                               _ptr(status), _stream(stream))
     if r:
         raise TsvError(r, "tree_verify_attn")
+
+
+_lib.tsv_bench_tree_verify_attn_stages.restype = C.c_int
+_lib.tsv_bench_tree_verify_attn_stages.argtypes = [C.POINTER(CShape), C.POINTER(CCache), C.POINTER(CNodes), C.POINTER(CScratch),
+                                                   _p, _p, _p, C.c_size_t, _p, _p, C.c_int]
+
+
+def bench_tree_verify_attn_stages(shape: CShape, cache: LayerCache, nodes: NodeInputs, scratch: Scratch, out: torch.Tensor,
+                                  topk_idx: Optional[torch.Tensor], workspace: torch.Tensor, status: torch.Tensor, stages: int,
+                                  stream=None) -> None:
+    """Per-stage timing aid of the benchmark (an export of the library outside its public header): tree_verify_attn
+    restricted to `stages` (STAGE_SELECT | STAGE_ATTENTION).  The attention stage alone reuses the selection that a
+    full call on the same inputs left in `workspace`."""
+    cs, ns, ss = cache.struct(), nodes.struct(), scratch.struct()
+    wp, wn = _aligned(workspace)
+    r = _lib.tsv_bench_tree_verify_attn_stages(C.byref(shape), C.byref(cs), C.byref(ns), C.byref(ss), _ptr(out), _ptr(topk_idx),
+                                               wp, wn, _ptr(status), _stream(stream), stages)
+    if r:
+        raise TsvError(r, "tsv_bench_tree_verify_attn_stages")
 
 
 class LayerPack:

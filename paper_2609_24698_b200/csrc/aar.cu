@@ -102,13 +102,14 @@ __global__ void __launch_bounds__(128) aar_commit_kernel(const tsv_shape s, cons
   }
 }
 
-int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const int32_t* parent, const int32_t* n_nodes,
+int launch_aar(const tsv_shape& s, int n_layers, const tsv_cache* const* caches, const tsv_nodes* const* nodes,
+               const tsv_scratch* const* scratch, const int32_t* parent, const int32_t* n_nodes,
                const int32_t* draft, const int32_t* target, int32_t* accept_len, int32_t* accept_path,
                int32_t* bonus, int32_t* status, cudaStream_t st) {
   AarLayers ls;
   for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
-    for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
+    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].sc = *scratch[l0 + i]; }
     const int last = l0 + ls.n >= n_layers;
     TSV_PREP(aar_walk_kernel);
     aar_walk_kernel<<<s.B, 32, 0, st>>>(s, ls, parent, n_nodes, draft, target, accept_len, accept_path, bonus, status, last);
@@ -116,7 +117,7 @@ int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const i
   }
   for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
-    for (int i = 0; i < ls.n; ++i) ls.l[i] = layers[l0 + i];
+    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].sc = *scratch[l0 + i]; }
     TSV_PREP(aar_commit_kernel);
     aar_commit_kernel<<<dim3(s.B, ls.n), 128, 0, st>>>(s, ls, accept_len, accept_path, status);
     count_launch();

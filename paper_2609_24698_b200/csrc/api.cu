@@ -1,5 +1,5 @@
 // C-ABI front end: argument validation on the host, workspace carve-up, kernel dispatch.
-// No allocation, no synchronisation, no state between calls.
+// No allocation (host or device), no synchronisation.
 #include <math.h>
 
 #include <atomic>
@@ -109,6 +109,19 @@ static int check_scratch(const tsv_scratch* s) {
   return TSV_OK;
 }
 
+// tree_verify_attn after validation.  All host work that can fail (tensor maps, kernel attributes) comes before the
+// first launch, so a negative return means that nothing was enqueued by this call, unless a launch itself fails.
+static int tva_stages(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, void* out,
+                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st, int stages) {
+  int r;
+  TvaTcPrep prep;
+  if (p.tc && (stages & 2) && (r = prepare_tva_tc(s, p, c, nd, out, ws, prep))) return r;
+  if ((stages & 1) && (r = launch_tva_select(s, p, c, nd, sc, topk_idx, ws, status, st))) return r;
+  if (!(stages & 2)) return TSV_OK;
+  if (p.tc) return launch_tva_tc(s, p, prep, c, nd, sc, out, ws, status, st);
+  return launch_tva_simt(s, p, c, nd, sc, out, ws, status, st);
+}
+
 }  // namespace tsv
 
 using namespace tsv;
@@ -159,12 +172,25 @@ int tree_verify_attn(const tsv_shape* shape, const tsv_cache* cache, const tsv_n
   TvaPlan p;
   make_tva_plan(s, p);
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < p.total) return TSV_ERR_WORKSPACE;
-  cudaStream_t st = (cudaStream_t)stream;
-  if (!(s.flags & TSV_FLAG_SKIP_SELECT))
-    if ((r = launch_tva_select(s, p, *cache, *nodes, *scratch, topk_idx, (char*)workspace, status, st))) return r;
-  if (s.flags & TSV_FLAG_SKIP_ATTN) return TSV_OK;
-  if (p.tc) return launch_tva_tc(s, p, *cache, *nodes, *scratch, out, (char*)workspace, status, st);
-  return launch_tva_simt(s, p, *cache, *nodes, *scratch, out, (char*)workspace, status, st);
+  return tva_stages(s, p, *cache, *nodes, *scratch, out, topk_idx, (char*)workspace, status, (cudaStream_t)stream, 3);
+}
+
+// Not part of the public interface (not declared in tsv.h): tree_verify_attn restricted to some of its stages, for
+// per-stage timing by the benchmark.  stages: bit 0 = CSA selection, bit 1 = attention (tile plan + attention kernels).
+// The attention stage alone reuses the selection a previous full call on the same inputs left in `workspace`.
+int tsv_bench_tree_verify_attn_stages(const tsv_shape* shape, const tsv_cache* cache, const tsv_nodes* nodes, const tsv_scratch* scratch,
+                                      void* out, int32_t* topk_idx, void* workspace, size_t workspace_bytes, int32_t* status, void* stream,
+                                      int stages) {
+  if (!shape || !status || !out) return TSV_ERR_NULL;
+  if (!shape_ok(shape)) return TSV_ERR_SHAPE;
+  int r;
+  if ((r = check_cache(cache)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
+  if (!al16(out)) return TSV_ERR_ALIGN;
+  const tsv_shape s = resolved(shape);
+  TvaPlan p;
+  make_tva_plan(s, p);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < p.total) return TSV_ERR_WORKSPACE;
+  return tva_stages(s, p, *cache, *nodes, *scratch, out, topk_idx, (char*)workspace, status, (cudaStream_t)stream, stages & 3);
 }
 
 int accept_and_refresh(const tsv_shape* shape, int32_t n_layers, const tsv_cache* const* caches, const tsv_nodes* const* nodes,
@@ -174,20 +200,11 @@ int accept_and_refresh(const tsv_shape* shape, int32_t n_layers, const tsv_cache
     return TSV_ERR_NULL;
   if (!shape_ok(shape)) return TSV_ERR_SHAPE;
   if (n_layers < 1 || n_layers > 4096) return TSV_ERR_SHAPE;
-  AarLayer stackbuf[64];
-  AarLayer* ls = n_layers <= 64 ? stackbuf : new AarLayer[n_layers];
-  int r = TSV_OK;
-  for (int l = 0; l < n_layers && !r; ++l) {
-    if ((r = check_cache(caches[l])) || (r = check_nodes(nodes[l], false)) || (r = check_scratch(scratch[l]))) break;
-    ls[l].c = *caches[l];
-    ls[l].node_kv = nodes[l]->kv;
-    ls[l].sc = *scratch[l];
-  }
-  if (!r)
-    r = launch_aar(resolved(shape), n_layers, ls, nodes[0]->parent, nodes[0]->n_nodes, draft_tok, target_tok, accept_len,
-                   accept_path, bonus_tok, status, (cudaStream_t)stream);
-  if (ls != stackbuf) delete[] ls;
-  return r;
+  int r;
+  for (int l = 0; l < n_layers; ++l)
+    if ((r = check_cache(caches[l])) || (r = check_nodes(nodes[l], false)) || (r = check_scratch(scratch[l]))) return r;
+  return launch_aar(resolved(shape), n_layers, caches, nodes, scratch, nodes[0]->parent, nodes[0]->n_nodes, draft_tok, target_tok, accept_len,
+                    accept_path, bonus_tok, status, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -49,7 +49,8 @@ struct TvaPlan {
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
 
 int launch_bsb(const tsv_shape& s, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, int32_t* status, cudaStream_t st);
-int launch_aar(const tsv_shape& s, int n_layers, const AarLayer* layers, const int32_t* parent, const int32_t* n_nodes,
+int launch_aar(const tsv_shape& s, int n_layers, const tsv_cache* const* caches, const tsv_nodes* const* nodes,
+               const tsv_scratch* const* scratch, const int32_t* parent, const int32_t* n_nodes,
                const int32_t* draft, const int32_t* target, int32_t* accept_len, int32_t* accept_path,
                int32_t* bonus, int32_t* status, cudaStream_t st);
 // indexer scores of all nodes of a sequence as one small GEMM per tile of entries (bf16, 128-wide indexer rows, D * HI <= 32)
@@ -66,10 +67,17 @@ constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs a
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
 bool tva_tc_pair_usable(const tsv_cache& c);
-int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
-                      int32_t* status, cudaStream_t st);
+// Host-side preparation of the tensor-core attention path: everything that can fail on the host (tensor maps, kernel
+// attributes) is done here, before any kernel of the call is enqueued.
+struct TvaTcPrep {
+  alignas(64) unsigned char maps[14 * 128];   // the paired kernel's tensor maps (a CUtensorMap is 128 bytes)
+  int32_t tma;                                // the contiguous-run path is usable for these caches
+};
+int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, void* out, char* ws, int32_t* status, cudaStream_t st);
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
-int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                   void* out, char* ws, int32_t* status, cudaStream_t st);
 
 }  // namespace tsv

@@ -8,6 +8,8 @@
 // file-scope device array instead, so the call itself allocates nothing.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "tsv.h"
 
 // The workspace.  Every GPU whose context loads this library holds these bytes until exit.
@@ -16,19 +18,26 @@ static __device__ __align__(256) unsigned char g_static_workspace[TSV_STATIC_WOR
 namespace {
 
 constexpr int kMaxDevices = 64;
-void* g_ws_addr[kMaxDevices];          // device address of the array, per device; 0 = not looked up yet
+std::atomic<void*> g_ws_addr[kMaxDevices];   // device address of the array, per device; null = not looked up yet
+                                             // (threads that look it up at the same time store the same value)
 
 // `g_static_workspace` in host code is only a handle for the symbol, not a device address:
 // the address a kernel can use has to be asked for, per device, with that device current.
+// The first look-up on a device also makes the runtime load this library's device code there,
+// which is when the device reserves the array's bytes: it can fail on a device whose memory is
+// already exhausted, so the first call belongs at start-up.
 int static_workspace(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TSV_ERR_CUDA;
-  if (!g_ws_addr[dev]) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return TSV_ERR_CUDA;
-    g_ws_addr[dev] = p;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TSV_ERR_CUDA; }
+  void* p = g_ws_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) {
+      cudaGetLastError();                    // leave no stale error behind for the next call's launch checks
+      return TSV_ERR_CUDA;
+    }
+    g_ws_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_ws_addr[dev];
+  *out = p;
   return TSV_OK;
 }
 

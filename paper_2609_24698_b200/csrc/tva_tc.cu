@@ -30,7 +30,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
                                              const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
-  __shared__ int wsum[9];
   __shared__ int n_cand[8], win_lo[8];
   __shared__ int dense;
   const int tile = blockIdx.x, b = blockIdx.y, D = s.D, H = s.H;
@@ -306,7 +305,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
   const size_t tix = (size_t)blockIdx.y * pl.tc_nt + blockIdx.x;
   int pos = (int)tix;                                 // fetched now, used at the end
-  if (tile_cta && threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // (with TSV_FLAG_SKIP_SELECT: the previous call's)
+  if (tile_cta && threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // (when the attention stage runs alone: the previous call's)
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
   tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
@@ -691,27 +690,45 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
 }
 
-int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
-                  void* out, char* ws, int32_t* status, cudaStream_t st) {
-  TvaPlan p = p_in;
-  p.tc_tma = tva_tc_pair_usable(c) ? 1 : 0;
-  const size_t plan_sm = p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) : 0;   // node bits per entry, cleared by words
-  if (plan_sm > 32 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)
+static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) : 0; }   // node bits per entry, cleared by words
+// The pointer-gather kernel serves tiles whose committed CSA run is longer than twice the selection size (and every
+// tile when the caches do not allow TMA).  With capacities that rule such tiles out it is not launched, nor is the
+// merge kernel: the paired kernel merges the chunks of its own tiles.
+static bool gather_kernel_needed(const tsv_shape& s, const TvaPlan& p, bool tma) {
+  return !tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk);
+}
+
+// Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
+int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
+  prep.tma = tva_tc_pair_usable(c) ? 1 : 0;
+  const size_t plan_sm = plan_smem_bytes(p);
+  if (plan_sm > 32 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess) {
+    cudaGetLastError();
     return TSV_ERR_CUDA;
+  }
+  if (gather_kernel_needed(s, p, prep.tma) &&
+      cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
+    cudaGetLastError();
+    return TSV_ERR_CUDA;
+  }
   TSV_PREP(tc_plan_kernel);
   TSV_PREP(tc_attn_kernel);
   TSV_PREP(tc_combine_kernel);
-  tc_plan_kernel<<<dim3(p.tc_nt + (p.tc_tma ? 1 : 0), s.B), 256, plan_sm, st>>>(s, p, c, nd, sc, ws);   // x: tiles (+ the packing CTA)
+  if (prep.tma) return prepare_tva_tc_pair(s, p, c, nd, out, ws, prep);
+  return TSV_OK;
+}
+
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                  void* out, char* ws, int32_t* status, cudaStream_t st) {
+  TvaPlan p = p_in;
+  p.tc_tma = prep.tma;
+  tc_plan_kernel<<<dim3(p.tc_nt + (p.tc_tma ? 1 : 0), s.B), 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);   // x: tiles (+ the packing CTA)
   count_launch();
   if (p.tc_tma) {
-    const int r = launch_tva_tc_pair(s, p, c, nd, out, ws, status, st);
+    const int r = launch_tva_tc_pair(s, p, prep, out, ws, status, st);
     if (r != TSV_OK) return r;
   }
-  // The pointer-gather kernel serves tiles whose committed CSA run is longer than twice the selection size (and every
-  // tile when the caches do not allow TMA).  With capacities that rule such tiles out it is not launched, nor is the
-  // merge kernel: the paired kernel merges the chunks of its own tiles.
-  if (!p.tc_tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk)) {
-    if (cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) return TSV_ERR_CUDA;
+  if (gather_kernel_needed(s, p, p.tc_tma)) {
     tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
     if (p.tc_chmax > 1) {

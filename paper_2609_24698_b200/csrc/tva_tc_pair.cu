@@ -678,9 +678,12 @@ static bool make_map(CUtensorMap* m, const void* basep, int64_t rows, int box_ro
 
 bool tva_tc_pair_usable(const tsv_cache& c) { return c.csa_rows > 0 && c.hca_rows > 0 && encode_fn() != nullptr; }
 
-int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws,
-                      int32_t* status, cudaStream_t st) {
-  pair::MapSet ms;
+static_assert(sizeof(pair::MapSet) <= sizeof(TvaTcPrep::maps), "tensor-map block of TvaTcPrep too small");
+
+// Everything of the paired kernel's launch that can fail on the host, done before any kernel of the call is enqueued:
+// the 14 tensor maps and the kernel's shared-memory attribute.
+int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
+  pair::MapSet& ms = *reinterpret_cast<pair::MapSet*>(prep.maps);
   const void* bases[4] = {c.csa_kv, c.hca_kv, c.win_kv, ws + p.off_misc};
   const int64_t rows[4] = {c.csa_rows, c.hca_rows, (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
   bool ok = make_map(&ms.q, nd.q, (int64_t)s.B * s.D * s.H, 128) && make_map(&ms.out, out, (int64_t)s.B * s.D * s.H, 32);
@@ -695,6 +698,11 @@ int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c,
     return TSV_ERR_CUDA;
   }
   TSV_PREP(tc_attn_pair_kernel);
+  return TSV_OK;
+}
+
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, void* out, char* ws, int32_t* status, cudaStream_t st) {
+  const pair::MapSet& ms = *reinterpret_cast<const pair::MapSet*>(prep.maps);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * p.tc_nt * s.B, p.tc_chmax, 1);
   cfg.blockDim = dim3(pair::TTHREADS, 1, 1);

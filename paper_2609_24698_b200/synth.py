@@ -229,6 +229,20 @@ def direct_cache(cfg: Config, layer: int, seq: int, L: int) -> Dict[str, np.ndar
     }
 
 
+def direct_arrays(cfg: Config, layer: int, b: int, L: int) -> Dict[str, np.ndarray]:
+    """direct_cache laid out as a committed per-sequence state: window rows placed at their ring slots (pos % w), the
+    open-block states as a one-token fold (max gate = the drawn gate, weight sum 1).  Layout only."""
+    sh = cfg.shape
+    dc = direct_cache(cfg, layer, b, L)
+    win = np.zeros((sh.window, sh.d), dtype=np.float32)
+    nw = dc["win_kv"].shape[0]
+    for i, pos in enumerate(range(L - nw, L)):
+        win[pos % sh.window] = dc["win_kv"][i]
+    return {"csa_kv": dc["csa_kv"], "csa_ik": dc["csa_ik"], "hca_kv": dc["hca_kv"], "win": win,
+            "csa_mx": float(dc["gates"][0]), "csa_s": 1.0, "csa_acc_kv": dc["csa_acc_kv"], "csa_acc_ik": dc["csa_acc_ik"],
+            "hca_mx": float(dc["gates"][1]), "hca_s": 1.0, "hca_acc_kv": dc["hca_acc_kv"]}
+
+
 def small_config(name: str = "tiny", dtype: str = "fp32", B: int = 2, D: int = 6, H: int = 4, d: int = 16,
                  m_csa: int = 2, topk: int = 3, HI: int = 2, di: int = 8, m_hca: int = 3, window: int = 4,
                  L_min: int = 0, L_max: int = 12, seed: int = 0, cfg_id: int = 100, layers: int = 1,

@@ -18,17 +18,7 @@ from . import harness as hz
 from . import synth
 
 
-def direct_arrays(cfg: synth.Config, layer: int, b: int, L: int) -> Dict[str, np.ndarray]:
-    """synth.direct_cache laid out as harness.fill_cache expects (window rows placed at pos % w)."""
-    sh = cfg.shape
-    dc = synth.direct_cache(cfg, layer, b, L)
-    win = np.zeros((sh.window, sh.d), dtype=np.float32)
-    nw = dc["win_kv"].shape[0]
-    for i, pos in enumerate(range(L - nw, L)):
-        win[pos % sh.window] = dc["win_kv"][i]
-    return {"csa_kv": dc["csa_kv"], "csa_ik": dc["csa_ik"], "hca_kv": dc["hca_kv"], "win": win,
-            "csa_mx": float(dc["gates"][0]), "csa_s": 1.0, "csa_acc_kv": dc["csa_acc_kv"], "csa_acc_ik": dc["csa_acc_ik"],
-            "hca_mx": float(dc["gates"][1]), "hca_s": 1.0, "hca_acc_kv": dc["hca_acc_kv"]}
+direct_arrays = synth.direct_arrays      # (kept under this name for the callers of this module)
 
 
 @dataclass

@@ -2,9 +2,10 @@
 (engines that own the whole device pool, plug-ins, latency-critical loops).  Its workspace is an
 array built into the library; this test checks, through the C-ABI, that it gives what
 tree_verify_attn gives with a caller-provided workspace -- on two calls in a row, because the
-built-in array is shared and keeps the previous call's contents -- and that shapes beyond the
-built-in size are refused.  Collected last on purpose (file name), so a failure here cannot hide
-the result of any other test; it also passes when run alone in a fresh process.
+built-in array is shared and keeps the previous call's contents --, that it matches the oracle on
+the tensor-core path (whose plan leaves counters and tile records in the shared array between
+calls), that the second call leaves the device's free memory as it was, and that shapes beyond
+the built-in size are refused.
 """
 import numpy as np
 import pytest
@@ -52,6 +53,45 @@ def test_static_workspace_matches_caller_workspace_twice():
         err = np.max(np.abs(out2.float().cpu().numpy() - ref)) / np.max(np.abs(ref))
         assert err <= 2e-2, err                # the tolerance of the bf16 parity tests; in practice the bits agree
         assert ref_out.any()
+
+
+def test_static_workspace_tensor_core_path_matches_oracle_and_allocates_nothing():
+    """bf16, d = 512 (tcgen05 kernels, single- and multi-chunk tiles), small enough for the built-in array: two cycles in
+    a row against the oracle at the tolerance of the bf16 parity tests; free device memory unchanged across the second call."""
+    from oracle import tsv_oracle as O
+    from paper_2609_24698_b200 import binding as tsv, harness as hz
+    from tests.helpers import oracle_states, per_seq, state_arrays
+    cfg = synth.Config("noalloc_tc", 179, synth.Shape("bf16", 2, 8, 64, 512, 4, 512, 4, 128, 128, 128), L_min=300, L_max=1400, seed=12)
+    sh = cfg.shape
+    lengths = synth.prefix_lengths(cfg)
+    states = oracle_states(cfg, lengths)
+    ccap, hcap = hz.capacities(sh, lengths, 4 * sh.D)
+    max_L = 1500
+    assert tsv.workspace_bytes(sh, max_L) <= tsv.STATIC_WORKSPACE_BYTES
+    eng = hz.VerifyEngine(sh, 1, ccap, hcap, max_L, want_topk=True)
+    for b in range(sh.B):
+        hz.fill_cache(eng.caches[0], sh, b, int(lengths[b]), state_arrays(states[0][b]))
+    for cycle in (0, 1):
+        nodes = synth.node_inputs(cfg, 0, cycle)
+        parent, n_nodes = synth.trees(cfg, cycle)
+        draft, target = synth.tokens(cfg, cycle, parent, n_nodes)
+        inp = hz.InputSet.from_numpy(sh, [nodes], parent, n_nodes, draft, target)
+        out = torch.full_like(eng.out[0], 3.0)
+        tsv.branch_state_build(eng.cshape, eng.caches[0], inp.layers[0], eng.scratch[0], eng.status)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        tsv.tree_verify_attn_static(eng.cshape, eng.caches[0], inp.layers[0], eng.scratch[0], out, eng.topk_idx[0], eng.status)
+        torch.cuda.synchronize()
+        if cycle == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
+        assert int(eng.status.sum()) == 0
+        got = out.float().cpu().numpy().astype(np.float64)
+        for b in range(sh.B):
+            nb = per_seq(nodes, b)
+            sc = O.branch_state_build(states[0][b], sh, nb, parent[b], int(n_nodes[b]))
+            ref, _ = O.tree_verify_attn(states[0][b], sh, nb, parent[b], int(n_nodes[b]), sc)
+            err = np.max(np.abs(got[b] - ref)) / np.max(np.abs(ref))
+            assert err <= 2e-2, (cycle, b, err)
 
 
 def test_static_workspace_refuses_oversized_shapes():
