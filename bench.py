@@ -32,6 +32,8 @@ import numpy as np  # noqa: E402
 # verify cycle.  The captures are summarised under profiles/; workloads without a capture report null.
 NCU_DRAM = {
     "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 70_262_784, "cycle_bytes": None},   # 65.41 MB read + 4.85 MB written
+    # cfg5: tc_attn_kernel 62.28 MB read + 19.15 MB written; all kernels of one cycle 191.7 MB (cold cache per kernel)
+    "cfg5": {"kernel": "tc_attn_kernel", "launch_bytes": 81_427_712, "cycle_bytes": 191_703_808},
 }
 ATTN_KERNEL = {"cfg1": "attn_simt_kernel (fp32 CUDA-core path)", "cfg2": "tc_attn_pair_kernel", "cfg2_chain": "tc_attn_pair_kernel",
                "cfg3": "tc_attn_pair_kernel + tc_attn_kernel (pointer gather) + tc_combine_kernel", "cfg4": "tc_attn_pair_kernel",

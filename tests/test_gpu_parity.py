@@ -413,6 +413,21 @@ def test_budgets_beyond_eight_cuda_core_path(dtype):
         lockstep(cfg, cycles=3, check_recompress=True)
 
 
+
+# ------------------------------------------------------------------------------------------------ variants
+@pytest.mark.parametrize("dtype,big", [("fp32", False), ("bf16", False), ("bf16", True)])
+def test_variant_without_hca_cache(dtype, big):
+    """A layer with no HCA cache (the CSA-only variant the paper's discussion names): an HCA block length beyond any
+    sequence length keeps n_hca at 0 for ever; CUDA-core path (small d) and tensor-core path (bench head shape)."""
+    no_hca = 1 << 30
+    if big:
+        cfg = synth.Config("no_hca_tc", 88, synth.Shape("bf16", 4, 8, 64, 512, 4, 256, 4, 128, no_hca, 128), L_min=200, L_max=2300, seed=8)
+        lockstep(cfg, cycles=3, check_recompress=True)
+    else:
+        cfg = synth.small_config(name="no_hca", dtype=dtype, B=4, D=8, H=6, d=64, m_csa=2, topk=10, HI=2, di=16, m_hca=no_hca, window=12,
+                                 L_min=0, L_max=90, layers=2, seed=87, cfg_id=87, sm_scale=2.0)
+        lockstep(cfg, cycles=5, check_recompress=True)
+
 # ------------------------------------------------------------------------------------------------ the cycle as the benchmark runs it
 def test_graph_replayed_cycles_match_oracle_and_eager():
     """One CUDA graph captured over a fixed input slot and replayed for four cycles (fresh inputs copied into the slot each
