@@ -70,8 +70,18 @@ enum {                         /* per-sequence status bits, device-written */
 };
 
 enum {                         /* tsv_shape.flags */
-  TSV_FLAG_FORCE_SIMT = 1     /* tree_verify_attn: use the CUDA-core kernels even where the
+  TSV_FLAG_FORCE_SIMT = 1,    /* tree_verify_attn: use the CUDA-core kernels even where the
                                   tensor-core kernels apply                                 */
+  TSV_FLAG_HCA_DEFERRED = 2   /* C128-deferred refresh schedule (Section "Performance Optimization": C4 is refreshed
+                                  timely, C128 writes are delayed and combined once the accepted path is known).
+                                  For a sequence in which no HCA block can close inside the tree
+                                  ((L % m_hca) + D < m_hca), branch_state_build builds no HCA branch states: the
+                                  scratch fields hca_mx, hca_s, hca_acc_kv and new_hca_kv of that sequence are left
+                                  untouched (hca_done is written, all 0), and accept_and_refresh folds the accepted
+                                  path's (g_hca, c_hca) into the persistent open HCA block itself, in path order, with
+                                  the arithmetic of branch_state_build -- the committed state is bit-identical to the
+                                  timely schedule's.  Sequences in which a block may close inside the tree take the
+                                  timely path.  Give the same flag to all three calls of a cycle.               */
 };
 
 /* Problem shape; HOST memory.

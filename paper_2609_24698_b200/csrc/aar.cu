@@ -92,12 +92,49 @@ __global__ void __launch_bounds__(128) aar_commit_kernel(const tsv_shape s, cons
     }
   }
   const size_t last = (size_t)b * D + accept_path[(size_t)b * D + al - 1];
-  copy_row16(ly.c.csa_acc_kv + (size_t)b * s.d, ly.sc.csa_acc_kv + last * s.d, s.d * 4, tid, nt);
-  copy_row16(ly.c.csa_acc_ik + (size_t)b * s.di, ly.sc.csa_acc_ik + last * s.di, s.di * 4, tid, nt);
-  copy_row16(ly.c.hca_acc_kv + (size_t)b * s.d, ly.sc.hca_acc_kv + last * s.d, s.d * 4, tid, nt);
+  // Open-block states of the last accepted node.  A block that this node closed leaves an empty state, whose stored numbers
+  // nobody reads (emptiness is known from the position count): that copy is skipped.
+  const bool csa_open = (L + al) % s.m_csa != 0, hca_open = (L + al) % s.m_hca != 0;
+  if (csa_open) {
+    copy_row16(ly.c.csa_acc_kv + (size_t)b * s.d, ly.sc.csa_acc_kv + last * s.d, s.d * 4, tid, nt);
+    copy_row16(ly.c.csa_acc_ik + (size_t)b * s.di, ly.sc.csa_acc_ik + last * s.di, s.di * 4, tid, nt);
+  }
+  const bool hdef = hca_deferred(s, L);
+  if (hdef) {
+    // C128-deferred schedule: branch_state_build built no HCA states for this sequence (no block closes inside its tree);
+    // the accepted tokens are folded into the persistent open block here, in path order, with the arithmetic of the state
+    // build (scalar part by every thread alike, each thread its own vector elements), so the result has the same bits.
+    float mx = ly.c.hca_mx[b], sw = ly.c.hca_s[b];
+    float coef_a[TSV_MAX_D], coef_b[TSV_MAX_D];
+    for (int i = 0; i < al; ++i) {
+      const int n = accept_path[(size_t)b * D + i];
+      const float g = ly.node_g_hca[(size_t)b * D + n];
+      if ((L + i) % s.m_hca == 0) { mx = g; sw = 1.f; coef_a[i] = 0.f; coef_b[i] = 1.f; }
+      else {
+        const float mx2 = fmaxf(mx, g);
+        coef_a[i] = expf(mx - mx2); coef_b[i] = expf(g - mx2);
+        sw = fmaf(sw, coef_a[i], coef_b[i]);
+        mx = mx2;
+      }
+    }
+    for (int e = tid; e < s.d; e += nt) {
+      float acc = ly.c.hca_acc_kv[(size_t)b * s.d + e];
+      for (int i = 0; i < al; ++i) {
+        const size_t nidx = (size_t)b * D + accept_path[(size_t)b * D + i];
+        const float cv = s.dtype == TSV_BF16 ? to_f(reinterpret_cast<const bf16*>(ly.node_c_hca)[nidx * s.d + e])
+                                             : reinterpret_cast<const float*>(ly.node_c_hca)[nidx * s.d + e];
+        acc = (L + i) % s.m_hca == 0 ? cv : fmaf(coef_a[i], acc, coef_b[i] * cv);
+      }
+      ly.c.hca_acc_kv[(size_t)b * s.d + e] = acc;
+    }
+    __syncthreads();                    // every thread has read the old scalars before thread 0 replaces them
+    if (tid == 0) { ly.c.hca_mx[b] = mx; ly.c.hca_s[b] = sw; }
+  } else if (hca_open) {
+    copy_row16(ly.c.hca_acc_kv + (size_t)b * s.d, ly.sc.hca_acc_kv + last * s.d, s.d * 4, tid, nt);
+  }
   if (tid == 0) {
     ly.c.csa_mx[b] = ly.sc.csa_mx[last]; ly.c.csa_s[b] = ly.sc.csa_s[last];
-    ly.c.hca_mx[b] = ly.sc.hca_mx[last]; ly.c.hca_s[b] = ly.sc.hca_s[last];
+    if (!hdef) { ly.c.hca_mx[b] = ly.sc.hca_mx[last]; ly.c.hca_s[b] = ly.sc.hca_s[last]; }
     ly.c.L[b] = L + al;
   }
 }
@@ -109,7 +146,7 @@ int launch_aar(const tsv_shape& s, int n_layers, const tsv_cache* const* caches,
   AarLayers ls;
   for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
-    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].sc = *scratch[l0 + i]; }
+    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].node_c_hca = nodes[l0 + i]->c_hca; ls.l[i].node_g_hca = nodes[l0 + i]->g_hca; ls.l[i].sc = *scratch[l0 + i]; }
     const int last = l0 + ls.n >= n_layers;
     TSV_PREP(aar_walk_kernel);
     aar_walk_kernel<<<s.B, 32, 0, st>>>(s, ls, parent, n_nodes, draft, target, accept_len, accept_path, bonus, status, last);
@@ -117,7 +154,7 @@ int launch_aar(const tsv_shape& s, int n_layers, const tsv_cache* const* caches,
   }
   for (int l0 = 0; l0 < n_layers; l0 += kAarLayersPerLaunch) {
     ls.n = n_layers - l0 < kAarLayersPerLaunch ? n_layers - l0 : kAarLayersPerLaunch;
-    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].sc = *scratch[l0 + i]; }
+    for (int i = 0; i < ls.n; ++i) { ls.l[i].c = *caches[l0 + i]; ls.l[i].node_kv = nodes[l0 + i]->kv; ls.l[i].node_c_hca = nodes[l0 + i]->c_hca; ls.l[i].node_g_hca = nodes[l0 + i]->g_hca; ls.l[i].sc = *scratch[l0 + i]; }
     TSV_PREP(aar_commit_kernel);
     aar_commit_kernel<<<dim3(s.B, ls.n), 128, 0, st>>>(s, ls, accept_len, accept_path, status);
     count_launch();

@@ -51,6 +51,9 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
   const int dim = which == 1 ? di : d;
   const T* cin = reinterpret_cast<const T*>(which == 0 ? nd.c_csa : (which == 1 ? nd.ikc : nd.c_hca));
   const float* pers = which == 0 ? c.csa_acc_kv : (which == 1 ? c.csa_acc_ik : c.hca_acc_kv);
+  // C128-deferred schedule: the HCA slabs of a sequence in which no HCA block can close inside the tree have nothing to do
+  // (they learn the length first, one load, and leave before fetching any vector)
+  if (which == 2 && (s.flags & TSV_FLAG_HCA_DEFERRED) && blockIdx.y * kBsbThreads >= (unsigned)(d + di) && hca_deferred(s, c.L[b])) return;
   // issue this thread's loads before the scalar chain is known (padding slots load too: the memory is there)
   float cv[DMAX];
 #pragma unroll
@@ -67,6 +70,7 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
     for (int n = 0; n < DMAX; ++n) { gc[n] = __shfl_sync(0xffffffffu, gcl, n); gh[n] = __shfl_sync(0xffffffffu, ghl, n); }
   }
 
+  const bool hdef = hca_deferred(s, tm.L) && !tm.status;     // (tm.L is 0 for a flagged length: such a sequence commits nothing)
   if (threadIdx.x == 0) {
     const bool writer = blockIdx.y == 0;
     if (tm.status && writer) atomicOr(status + b, tm.status);
@@ -80,14 +84,14 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
           float mp = pcm, sp = pcs, mq = phm, sq = phs;
           if (n) { mp = cmx[par]; sp = cs[par]; mq = hmx[par]; sq = hs[par]; }
           scalar_fold(fcs[n], m1, s1, p, s.m_csa, mp, sp, gc[n]);
-          scalar_fold(fhs[n], m2, s2, p, s.m_hca, mq, sq, gh[n]);
+          if (hdef) fhs[n].done = 0; else scalar_fold(fhs[n], m2, s2, p, s.m_hca, mq, sq, gh[n]);
         } else {
           fcs[n].done = fhs[n].done = 0;
         }
         cmx[n] = m1; cs[n] = s1; hmx[n] = m2; hs[n] = s2;
         if (writer) {
           sc.csa_mx[(size_t)b * D + n] = m1; sc.csa_s[(size_t)b * D + n] = s1;
-          sc.hca_mx[(size_t)b * D + n] = m2; sc.hca_s[(size_t)b * D + n] = s2;
+          if (!hdef) { sc.hca_mx[(size_t)b * D + n] = m2; sc.hca_s[(size_t)b * D + n] = s2; }
           sc.csa_done[(size_t)b * D + n] = (uint8_t)fcs[n].done;
           sc.hca_done[(size_t)b * D + n] = (uint8_t)fhs[n].done;
         }
@@ -95,7 +99,7 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
     }
   }
   __syncthreads();
-  if (!live) return;
+  if (!live || (which == 2 && hdef)) return;
   const int nn = tm.status ? 0 : tm.nn;
   float* sacc = which == 0 ? sc.csa_acc_kv : (which == 1 ? sc.csa_acc_ik : sc.hca_acc_kv);
   T* newe = reinterpret_cast<T*>(which == 0 ? sc.new_csa_kv : (which == 1 ? sc.new_csa_ik : sc.new_hca_kv));

@@ -130,6 +130,13 @@ __device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, cons
   __syncthreads();
 }
 
+// C128-deferred schedule: no node of this sequence can close an HCA block (a node at depth delta closes one iff
+// (L + delta + 1) % m_hca == 0, and delta <= D - 1), so its HCA branch states are not built and the accepted path is
+// folded into the persistent state at commit time.
+__device__ __forceinline__ bool hca_deferred(const tsv_shape& s, int L) {
+  return (s.flags & TSV_FLAG_HCA_DEFERRED) && L >= 0 && (L % s.m_hca) + s.D < s.m_hca;
+}
+
 __device__ __forceinline__ float softmax_scale(const tsv_shape& s) {
   return s.sm_scale > 0.f ? s.sm_scale : rsqrtf((float)s.d);
 }

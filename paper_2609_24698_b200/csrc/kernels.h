@@ -22,6 +22,8 @@ void count_launch(int n = 1);
 struct AarLayer {
   tsv_cache c;
   const void* node_kv;
+  const void* node_c_hca;      // HCA compression vectors and gate logits of the nodes (C128-deferred schedule)
+  const float* node_g_hca;
   tsv_scratch sc;
 };
 constexpr int kAarLayersPerLaunch = 12;
