@@ -162,7 +162,9 @@ def workload_config(cfg, args):
             "global_batch": sh.B * max(1, args.gpus), "tree_nodes": sh.D, "layers": cfg.layers,
             "parallelism": "single GPU" if args.gpus <= 1 else f"{args.gpus} independent replicas (no collective)",
             "l2_policy": "inputs larger than L2: every cycle reads a different input set (q alone is 268 MB per cycle)",
-            "launch": "one CUDA graph replay per cycle", "hca_refresh_schedule": getattr(args, "schedule", "timely")}
+            "launch": "one CUDA graph replay per cycle", "hca_refresh_schedule": getattr(args, "schedule", "timely"),
+            "cache_layout": (f"paged pool, {args.page_tokens}-token pages, one page table for the CSA and HCA layers"
+                             if getattr(args, "page_tokens", 0) else "flat slab per sequence")}
 
 
 # ------------------------------------------------------------------------------------------ our arm
@@ -183,7 +185,7 @@ def run_ours(args, cfg):
     K, Wm = args.steps, max(3, args.warmup)
     n_sets = 3
     lib_flags = tsv.FLAG_HCA_DEFERRED if args.schedule == "c128-deferred" else 0
-    wl = W.build(cfg, cycles_headroom=2 * (K + Wm) + 8, n_sets=n_sets, flags=lib_flags, device=dev)
+    wl = W.build(cfg, cycles_headroom=2 * (K + Wm) + 8, n_sets=n_sets, flags=lib_flags, device=dev, page_tokens=args.page_tokens)
     eng = wl.engine
     snap = eng.snapshot()
     stream = torch.cuda.current_stream()
@@ -373,6 +375,8 @@ def main():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--page-tokens", type=int, default=0,
+                    help="keep the persistent caches in a paged pool with pages of this many tokens (0: flat slabs per sequence)")
     ap.add_argument("--schedule", default="timely", choices=["timely", "c128-deferred"],
                     help="refresh schedule of the HCA (C128) cache: per-node branch states (timely) or folded at commit time")
     args = ap.parse_args()

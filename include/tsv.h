@@ -122,6 +122,20 @@ typedef struct tsv_cache {
   float *hca_acc_kv;          /* [B][d]                                                     */
   int64_t csa_rows;           /* HOST value: rows allocated in csa_kv / csa_ik (all slabs)  */
   int64_t hca_rows;           /* HOST value: rows allocated in hca_kv                       */
+  /* Paged pool (Section "Temporary Branch States and Compressed-State Handling": a page-based pool seen as one logical
+   * layer and several physical layers that share page-level pointers).  With page_table non-NULL the CSA and HCA entries
+   * of a sequence do not sit in one slab each: logical page lp holds the entries of tokens [lp, lp + 1) * page_tokens, and
+   * ONE table gives its physical page for every physical layer: entry e of the CSA cache (kv and indexer key) is row
+   *     page_table[b][e / epp] * epp + e % epp,   epp = page_tokens / m_csa,
+   * entry h of the HCA cache is row  page_table[b][h / hpp] * hpp + h % hpp,  hpp = page_tokens / m_hca.
+   * csa_row0 / hca_row0 are ignored then (may be NULL); csa_cap / hca_cap still give the entries the sequence's assigned
+   * pages can hold.  page_tokens must be a multiple of m_csa and of m_hca.  The token-level window keeps its ring form
+   * (with window == page_tokens it is one page per sequence).  The tensor-core path fetches CSA rows by 32-row TMA boxes
+   * when epp is a multiple of 32 (e.g. 128-token pages with m_csa = 4: one box per page); otherwise, and for HCA rows
+   * beyond the first 32 entries unless hpp is a multiple of 32, it gathers rows by pointer. */
+  const int32_t *page_table;  /* [B][max_pages] device, or NULL: flat slabs                  */
+  int32_t page_tokens;        /* HOST value                                                 */
+  int32_t max_pages;          /* HOST value: columns of page_table                          */
 } tsv_cache;
 
 /* Per-cycle inputs of ONE layer for all tree nodes; read-only. */

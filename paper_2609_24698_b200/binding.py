@@ -39,13 +39,13 @@ class CShape(C.Structure):
                 ("flags", C.c_int32), ("reserved", C.c_int32)]
 
 
+CACHE_TENSORS = ("L", "csa_kv", "csa_ik", "csa_row0", "csa_cap", "hca_kv", "hca_row0", "hca_cap",
+                 "win_kv", "csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")
+
+
 class CCache(C.Structure):
-    _fields_ = [(n, _p) for n in ("L", "csa_kv", "csa_ik", "csa_row0", "csa_cap", "hca_kv", "hca_row0", "hca_cap",
-                                  "win_kv", "csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")] + \
-               [("csa_rows", C.c_int64), ("hca_rows", C.c_int64)]
-
-
-CACHE_TENSORS = tuple(n for n, t in CCache._fields_ if t is _p)
+    _fields_ = [(n, _p) for n in CACHE_TENSORS] + [("csa_rows", C.c_int64), ("hca_rows", C.c_int64),
+                                                   ("page_table", _p), ("page_tokens", C.c_int32), ("max_pages", C.c_int32)]
 
 
 class CNodes(C.Structure):
@@ -124,12 +124,30 @@ class LayerCache:
     hca_mx: torch.Tensor
     hca_s: torch.Tensor
     hca_acc_kv: torch.Tensor
+    page_table: Optional[torch.Tensor] = None      # [B, max_pages] int32: paged pool (csa_row0 / hca_row0 unused then)
+    page_tokens: int = 0
 
     def struct(self) -> CCache:
-        return CCache(*[_ptr(getattr(self, n)) for n in CACHE_TENSORS], int(self.csa_kv.shape[0]), int(self.hca_kv.shape[0]))
+        pt = self.page_table
+        return CCache(*[_ptr(getattr(self, n)) for n in CACHE_TENSORS], int(self.csa_kv.shape[0]), int(self.hca_kv.shape[0]),
+                      _ptr(pt), int(self.page_tokens), 0 if pt is None else int(pt.shape[1]))
 
     def clone(self) -> "LayerCache":
-        return LayerCache(*[getattr(self, n).clone() for n in CACHE_TENSORS])
+        return LayerCache(*[getattr(self, n).clone() for n in CACHE_TENSORS], page_table=self.page_table, page_tokens=self.page_tokens)
+
+    def csa_row_index(self, shape: synth.Shape, b: int, n: int) -> torch.Tensor:
+        """Physical rows of CSA entries 0 .. n-1 of sequence b (slab, or through the page table)."""
+        return self._rows(b, n, self.csa_row0, shape.m_csa)
+
+    def hca_row_index(self, shape: synth.Shape, b: int, n: int) -> torch.Tensor:
+        return self._rows(b, n, self.hca_row0, shape.m_hca)
+
+    def _rows(self, b: int, n: int, row0: torch.Tensor, block: int) -> torch.Tensor:
+        e = torch.arange(n, dtype=torch.long, device=self.L.device)
+        if self.page_table is None:
+            return int(row0[b]) + e
+        per = self.page_tokens // block
+        return self.page_table[b].long()[e // per] * per + e % per
 
 
 @dataclass
@@ -188,6 +206,38 @@ def alloc_cache(shape: synth.Shape, csa_caps: Sequence[int], hca_caps: Sequence[
         csa_mx=torch.zeros(B, **f32), csa_s=torch.zeros(B, **f32),
         csa_acc_kv=torch.zeros(B, shape.d, **f32), csa_acc_ik=torch.zeros(B, shape.di, **f32),
         hca_mx=torch.zeros(B, **f32), hca_s=torch.zeros(B, **f32), hca_acc_kv=torch.zeros(B, shape.d, **f32))
+
+
+def alloc_cache_paged(shape: synth.Shape, csa_caps: Sequence[int], hca_caps: Sequence[int], page_tokens: int, seed: int = 0,
+                      device="cuda") -> LayerCache:
+    """Empty caches over a paged pool: every sequence gets the pages its capacities ask for, drawn from one pool in a
+    shuffled order (pages of different sequences interleave), and ONE page table serves the CSA and the HCA layer."""
+    import numpy as np
+    assert page_tokens % shape.m_csa == 0 and page_tokens % shape.m_hca == 0
+    epp, hpp = page_tokens // shape.m_csa, page_tokens // shape.m_hca
+    need = [max(-(-int(c) // epp), -(-int(h) // hpp), 1) for c, h in zip(csa_caps, hca_caps)]
+    n_pages, max_pages = sum(need), max(need)
+    perm = np.random.default_rng(seed).permutation(n_pages)
+    table = np.full((shape.B, max_pages), -1, dtype=np.int32)
+    k = 0
+    for lp in range(max_pages):                       # page by page over the sequences: neighbours in a sequence are far apart
+        for b in range(shape.B):
+            if lp < need[b]:
+                table[b, lp] = perm[k]; k += 1
+    flat = alloc_cache(shape, [n_pages * epp], [n_pages * hpp], device)     # one slab per layer = the pool
+    B = shape.B
+    i32 = dict(dtype=torch.int32, device=device)
+    f32 = dict(dtype=torch.float32, device=device)
+    dt = torch_dtype(shape)
+    return LayerCache(
+        L=torch.zeros(B, **i32), csa_kv=flat.csa_kv, csa_ik=flat.csa_ik,
+        csa_row0=torch.zeros(B, dtype=torch.int64, device=device), csa_cap=torch.tensor([n * epp for n in need], **i32),
+        hca_kv=flat.hca_kv, hca_row0=torch.zeros(B, dtype=torch.int64, device=device), hca_cap=torch.tensor([n * hpp for n in need], **i32),
+        win_kv=torch.zeros(B, shape.window, shape.d, dtype=dt, device=device),
+        csa_mx=torch.zeros(B, **f32), csa_s=torch.zeros(B, **f32),
+        csa_acc_kv=torch.zeros(B, shape.d, **f32), csa_acc_ik=torch.zeros(B, shape.di, **f32),
+        hca_mx=torch.zeros(B, **f32), hca_s=torch.zeros(B, **f32), hca_acc_kv=torch.zeros(B, shape.d, **f32),
+        page_table=torch.from_numpy(table).to(device), page_tokens=page_tokens)
 
 
 def alloc_scratch(shape: synth.Shape, device="cuda") -> Scratch:

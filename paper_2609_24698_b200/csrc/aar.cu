@@ -82,12 +82,12 @@ __global__ void __launch_bounds__(128) aar_commit_kernel(const tsv_shape s, cons
     const size_t nidx = (size_t)b * D + n;
     copy_row16((char*)ly.c.win_kv + ((size_t)b * s.window + pos % s.window) * rowb, (const char*)ly.node_kv + nidx * rowb, (int)rowb, tid, nt);
     if (ly.sc.csa_done[nidx]) {
-      const size_t row = (size_t)ly.c.csa_row0[b] + pos / s.m_csa;
+      const size_t row = (size_t)csa_rows_of(ly.c, s, b)(pos / s.m_csa);
       copy_row16((char*)ly.c.csa_kv + row * rowb, (const char*)ly.sc.new_csa_kv + nidx * rowb, (int)rowb, tid, nt);
       copy_row16((char*)ly.c.csa_ik + row * ikb, (const char*)ly.sc.new_csa_ik + nidx * ikb, (int)ikb, tid, nt);
     }
     if (ly.sc.hca_done[nidx]) {
-      const size_t row = (size_t)ly.c.hca_row0[b] + pos / s.m_hca;
+      const size_t row = (size_t)hca_rows_of(ly.c, s, b)(pos / s.m_hca);
       copy_row16((char*)ly.c.hca_kv + row * rowb, (const char*)ly.sc.new_hca_kv + nidx * rowb, (int)rowb, tid, nt);
     }
   }

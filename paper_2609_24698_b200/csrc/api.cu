@@ -79,11 +79,14 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
 
 static inline bool al16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
-static int check_cache(const tsv_cache* c) {
+static int check_cache(const tsv_cache* c, const tsv_shape* s) {
   if (!c) return TSV_ERR_NULL;
-  const void* all[] = {c->L, c->csa_kv, c->csa_ik, c->csa_row0, c->csa_cap, c->hca_kv, c->hca_row0, c->hca_cap, c->win_kv,
+  const void* all[] = {c->L, c->csa_kv, c->csa_ik, c->csa_cap, c->hca_kv, c->hca_cap, c->win_kv,
                        c->csa_mx, c->csa_s, c->csa_acc_kv, c->csa_acc_ik, c->hca_mx, c->hca_s, c->hca_acc_kv};
   for (const void* p : all) if (!p) return TSV_ERR_NULL;
+  if (c->page_table) {      // paged pool: one table for all physical layers; the page size divides into whole blocks
+    if (c->page_tokens < 1 || c->max_pages < 1 || c->page_tokens % s->m_csa || c->page_tokens % s->m_hca) return TSV_ERR_SHAPE;
+  } else if (!c->csa_row0 || !c->hca_row0) return TSV_ERR_NULL;
   const void* vec[] = {c->csa_kv, c->csa_ik, c->hca_kv, c->win_kv, c->csa_acc_kv, c->csa_acc_ik, c->hca_acc_kv};
   for (const void* p : vec) if (!al16(p)) return TSV_ERR_ALIGN;
   return TSV_OK;
@@ -157,7 +160,7 @@ int branch_state_build(const tsv_shape* shape, const tsv_cache* cache, const tsv
   if (!shape || !status) return TSV_ERR_NULL;
   if (!shape_ok(shape)) return TSV_ERR_SHAPE;
   int r;
-  if ((r = check_cache(cache)) || (r = check_nodes(nodes, false)) || (r = check_scratch(scratch))) return r;
+  if ((r = check_cache(cache, shape)) || (r = check_nodes(nodes, false)) || (r = check_scratch(scratch))) return r;
   return launch_bsb(resolved(shape), *cache, *nodes, *scratch, status, (cudaStream_t)stream);
 }
 
@@ -166,7 +169,7 @@ int tree_verify_attn(const tsv_shape* shape, const tsv_cache* cache, const tsv_n
   if (!shape || !status || !out) return TSV_ERR_NULL;
   if (!shape_ok(shape)) return TSV_ERR_SHAPE;
   int r;
-  if ((r = check_cache(cache)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
+  if ((r = check_cache(cache, shape)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
   if (!al16(out)) return TSV_ERR_ALIGN;
   const tsv_shape s = resolved(shape);
   TvaPlan p;
@@ -184,7 +187,7 @@ int tsv_bench_tree_verify_attn_stages(const tsv_shape* shape, const tsv_cache* c
   if (!shape || !status || !out) return TSV_ERR_NULL;
   if (!shape_ok(shape)) return TSV_ERR_SHAPE;
   int r;
-  if ((r = check_cache(cache)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
+  if ((r = check_cache(cache, shape)) || (r = check_nodes(nodes, true)) || (r = check_scratch(scratch))) return r;
   if (!al16(out)) return TSV_ERR_ALIGN;
   const tsv_shape s = resolved(shape);
   TvaPlan p;
@@ -202,7 +205,7 @@ int accept_and_refresh(const tsv_shape* shape, int32_t n_layers, const tsv_cache
   if (n_layers < 1 || n_layers > 4096) return TSV_ERR_SHAPE;
   int r;
   for (int l = 0; l < n_layers; ++l)
-    if ((r = check_cache(caches[l])) || (r = check_nodes(nodes[l], false)) || (r = check_scratch(scratch[l]))) return r;
+    if ((r = check_cache(caches[l], shape)) || (r = check_nodes(nodes[l], false)) || (r = check_scratch(scratch[l]))) return r;
   return launch_aar(resolved(shape), n_layers, caches, nodes, scratch, nodes[0]->parent, nodes[0]->n_nodes, draft_tok, target_tok, accept_len,
                     accept_path, bonus_tok, status, (cudaStream_t)stream);
 }

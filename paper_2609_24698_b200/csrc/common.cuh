@@ -50,6 +50,32 @@ __device__ __forceinline__ void st16(bf16* p, const float* v) {
   *reinterpret_cast<uint4*>(p) = o;
 }
 
+// ---------------------------------------------------------------- cache rows
+// Row of entry e of one sequence in one physical layer of the cache: a slab starting at row0 (flat caches), or through
+// the sequence's page-table row with `per_page` entries of this layer per page (paged pool).
+struct RowAddr {
+  const int32_t* pt;
+  int32_t per_page;
+  int64_t row0;
+  __device__ __forceinline__ int64_t operator()(int e) const {
+    return pt ? (int64_t)__ldg(pt + e / per_page) * per_page + e % per_page : row0 + e;
+  }
+};
+__device__ __forceinline__ RowAddr csa_rows_of(const tsv_cache& c, const tsv_shape& s, int b) {
+  RowAddr r;
+  r.pt = c.page_table ? c.page_table + (size_t)b * c.max_pages : nullptr;
+  r.per_page = c.page_table ? c.page_tokens / s.m_csa : 1;
+  r.row0 = c.page_table ? 0 : c.csa_row0[b];
+  return r;
+}
+__device__ __forceinline__ RowAddr hca_rows_of(const tsv_cache& c, const tsv_shape& s, int b) {
+  RowAddr r;
+  r.pt = c.page_table ? c.page_table + (size_t)b * c.max_pages : nullptr;
+  r.per_page = c.page_table ? c.page_tokens / s.m_hca : 1;
+  r.row0 = c.page_table ? 0 : c.hca_row0[b];
+  return r;
+}
+
 // ---------------------------------------------------------------- tree metadata
 // Built by ONE thread of a CTA into shared memory, then read by all after a barrier.
 struct TreeMeta {

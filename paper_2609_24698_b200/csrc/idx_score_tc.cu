@@ -86,7 +86,8 @@ __global__ void __launch_bounds__(kItThreads) idx_score_tc_kernel(const tsv_shap
       cp16(bq + (c16 >> 3) * (kItN * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4), iq + (v ? (size_t)row * 256 + c16 * 16 : 0), v);
     }
   }
-  const char* ik = reinterpret_cast<const char*>(c.csa_ik) + (size_t)c.csa_row0[b] * 256;
+  const char* ik = reinterpret_cast<const char*>(c.csa_ik);
+  const RowAddr ikrow = csa_rows_of(c, s, b);
   auto load_tile = [&](int t) {                           // entries e0 + 128 t ..: two K slices of [128 rows x 128 bytes]
     const uint32_t dst = a0 + (uint32_t)(t & 1) * kItA;
     const int r0 = e0 + t * kItRows;
@@ -94,7 +95,7 @@ __global__ void __launch_bounds__(kItThreads) idx_score_tc_kernel(const tsv_shap
     for (int i = 0; i < kItRows * 16 / kItThreads; ++i) {
       const int idx = tid + kItThreads * i, row = idx >> 4, c16 = idx & 15;
       const bool v = r0 + row < n_csa;
-      cp16(dst + (c16 >> 3) * (kItRows * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4), ik + (v ? (size_t)(r0 + row) * 256 + c16 * 16 : 0), v);
+      cp16(dst + (c16 >> 3) * (kItRows * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4), ik + (v ? (size_t)ikrow(r0 + row) * 256 + c16 * 16 : 0), v);
     }
     cp_commit();
   };

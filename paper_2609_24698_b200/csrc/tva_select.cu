@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
   if (!need_any || (int)(blockIdx.x * blockDim.x) >= tm.n_csa) return;
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   const bool live = e < tm.n_csa;
-  const T* ikrow = reinterpret_cast<const T*>(c.csa_ik) + ((size_t)c.csa_row0[b] + (live ? e : 0)) * di;
+  const T* ikrow = reinterpret_cast<const T*>(c.csa_ik) + (size_t)csa_rows_of(c, s, b)(live ? e : 0) * di;
   float* scores = reinterpret_cast<float*>(ws + pl.off_scores) + (size_t)b * D * pl.score_ld;
   constexpr int V = Vec<T>::N;
   const int npg = min(32 / HI, (D + (int)gridDim.z - 1) / (int)gridDim.z);   // nodes per group; blockIdx.z owns a slab of nodes
@@ -149,7 +149,8 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
 #pragma unroll
     for (int j = 0; j < V; ++j) { q[h][j] = h < HI ? t0[j] : 0.f; q[h][V + j] = h < HI ? t1[j] : 0.f; }
   }
-  const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
+  const T* ik0 = reinterpret_cast<const T*>(c.csa_ik);
+  const RowAddr ikr = csa_rows_of(c, s, b);
   float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
   const int n_csa = tm.n_csa, e_base = blockIdx.x * kRows256PerCta, e_end = min(n_csa, e_base + kRows256PerCta);
 #pragma unroll 1
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int e = base + grp + 32 * u;
-      const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)(e < n_csa ? e : 0) * di) + gl * 2;
+      const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)ikr(e < n_csa ? e : 0) * di) + gl * 2;
       raw[u][0] = __ldg(rowp); raw[u][1] = __ldg(rowp + 1);
     }
 #pragma unroll
@@ -282,7 +283,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * HI * di;
     for (int i = threadIdx.x; i < HI * di; i += blockDim.x) iq_sm[i] = to_f(iq[i]);
     __syncthreads();
-    const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)c.csa_row0[b] * di;
+    const T* ik0 = reinterpret_cast<const T*>(c.csa_ik);
+    const RowAddr ikr = csa_rows_of(c, s, b);
     float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
     if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
       // Rows of 256 bytes (the benchmark's indexer width).  Few CTAs rank and each is a chain of its own, so load latency
@@ -315,7 +317,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
           const int idx = threadIdx.x + 256 * i, row = idx >> 4, c16 = idx & 15;
           if (row < nrow)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kStagePitch + c16 * 16),
-                         "l"(ikb + (size_t)(base + row) * 256 + c16 * 16) : "memory");
+                         "l"(ikb + (size_t)ikr(base + row) * 256 + c16 * 16) : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
       };
@@ -362,7 +364,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
         uint4 raw[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-          raw[u] = (c0 + u < di / V) ? __ldg(reinterpret_cast<const uint4*>(ik0 + (size_t)e * di + (c0 + u) * V)) : make_uint4(0, 0, 0, 0);
+          raw[u] = (c0 + u < di / V) ? __ldg(reinterpret_cast<const uint4*>(ik0 + (size_t)ikr(e) * di + (c0 + u) * V)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           if (c0 + u < di / V) {

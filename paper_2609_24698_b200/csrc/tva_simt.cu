@@ -46,13 +46,13 @@ __device__ __forceinline__ const T* key_row(int j, const NodeKeys& nk, const Tre
   const size_t d = s.d;
   if (j < nk.n_sel) {
     const int idx = sel[j];
-    if (idx < tm.n_csa) return reinterpret_cast<const T*>(c.csa_kv) + ((size_t)c.csa_row0[b] + idx) * d;
+    if (idx < tm.n_csa) return reinterpret_cast<const T*>(c.csa_kv) + (size_t)csa_rows_of(c, s, b)(idx) * d;
     int a = nk.newc[0];
     for (int i = 0; i < nk.n_newc; ++i) if (nk.newc_blk[i] == idx) a = nk.newc[i];
     return reinterpret_cast<const T*>(sc.new_csa_kv) + ((size_t)b * s.D + a) * d;
   }
   j -= nk.n_sel;
-  if (j < nk.n_hca) return reinterpret_cast<const T*>(c.hca_kv) + ((size_t)c.hca_row0[b] + j) * d;
+  if (j < nk.n_hca) return reinterpret_cast<const T*>(c.hca_kv) + (size_t)hca_rows_of(c, s, b)(j) * d;
   j -= nk.n_hca;
   if (j < nk.n_newh) return reinterpret_cast<const T*>(sc.new_hca_kv) + ((size_t)b * s.D + nk.newh[j]) * d;
   j -= nk.n_newh;

@@ -45,10 +45,16 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   __shared__ int64_t row0_sm[2];
   if (threadIdx.x >= 64 && threadIdx.x < 64 + D) cdone[threadIdx.x - 64] = sc.csa_done[(size_t)b * D + threadIdx.x - 64];
   if (threadIdx.x >= 96 && threadIdx.x < 96 + D) hdone[threadIdx.x - 96] = sc.hca_done[(size_t)b * D + threadIdx.x - 96];
-  if (threadIdx.x == 40) row0_sm[0] = c.csa_row0[b];
-  if (threadIdx.x == 41) row0_sm[1] = c.hca_row0[b];
+  if (threadIdx.x == 40) row0_sm[0] = c.page_table ? 0 : c.csa_row0[b];
+  if (threadIdx.x == 41) row0_sm[1] = c.page_table ? 0 : c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
-  const int64_t csa_row0 = row0_sm[0], hca_row0 = row0_sm[1];
+  // rows of the sequence's CSA and HCA entries: slabs, or through the page table of a paged pool
+  RowAddr csa_row, hca_row;
+  csa_row.pt = hca_row.pt = c.page_table ? c.page_table + (size_t)b * c.max_pages : nullptr;
+  csa_row.per_page = c.page_table ? c.page_tokens / s.m_csa : 1; hca_row.per_page = c.page_table ? c.page_tokens / s.m_hca : 1;
+  csa_row.row0 = row0_sm[0]; hca_row.row0 = row0_sm[1];
+  // runs of consecutive rows exist in a paged pool only where a page holds whole 32-row boxes of the layer
+  const bool csa_runs = !c.page_table || csa_row.per_page % kBoxRows == 0, hca_runs = !c.page_table || hca_row.per_page % kBoxRows == 0;
   if (blockIdx.x >= (unsigned)pl.tc_nt) {
     // The extra CTA of the sequence (grid x = tiles + 1): rows that are small and scattered (few HCA entries, tree nodes,
     // entries closed inside the tree) are packed into one contiguous per-sequence buffer so that TMA boxes can fetch
@@ -66,7 +72,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
     auto row_src = [&](int r) -> const uint4* {
       const char* src = nullptr;
-      if (r < nh_in) src = (const char*)c.hca_kv + ((size_t)hca_row0 + r) * rowb;
+      if (r < nh_in) src = (const char*)c.hca_kv + (size_t)hca_row(r) * rowb;
       else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
       else if (r < n_misc) {
         int ord = r - nh_in - tm.nn;
@@ -170,13 +176,13 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     // Ranked nodes still take the contiguous-run path while the run is at most twice the selection size: all committed
     // entries are staged and the unselected ones are masked per node.
-    if (dense || n_csa <= 2 * s.topk) {
+    if ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax)) {
       int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
       // four runs, each padded to whole boxes: committed CSA entries, HCA entries (when too many for the packed rows),
       // the window ring, the packed rows.  One pass over all keys: a thread finds the run of its key by comparison, so
       // the runs' (short, latency-bound) mask computations overlap instead of following each other.
       const int cnt[4] = {n_csa, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, min(tm.L, s.window), n_misc};
-      const int64_t start[4] = {csa_row0, hca_row0, (int64_t)b * s.window, (int64_t)b * pl.tc_misc_rows};
+      const int64_t start[4] = {0, 0, (int64_t)b * s.window, (int64_t)b * pl.tc_misc_rows};
       int k0[5];                                       // first key of each run
       k0[0] = 0;
 #pragma unroll
@@ -185,7 +191,8 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       for (int bi = threadIdx.x; bi < kb / kBoxRows; bi += blockDim.x) {
         const int k = bi * kBoxRows;
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
-        box[bi] = make_int2(g, (int)(start[g] + (k - k0[g])));
+        // (a box of a cache run never crosses a page: it starts on a multiple of 32 entries and per_page is one too)
+        box[bi] = make_int2(g, (int)(g == 0 ? csa_row(k - k0[0]) : g == 1 ? hca_row(k - k0[1]) : start[g] + (k - k0[g])));
       }
       for (int k = threadIdx.x; k < kb; k += blockDim.x) {
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
@@ -244,7 +251,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       const uint32_t sel_m = __ballot_sync(0xffffffffu, m != 0);
       if (m) {
         const int pos = pos0 + __popc(sel_m & lt);
-        kptr[pos] = (uint64_t)((const char*)c.csa_kv + ((size_t)csa_row0 + i) * rowb); kmask[pos] = (uint8_t)m;
+        kptr[pos] = (uint64_t)((const char*)c.csa_kv + (size_t)csa_row(i) * rowb); kmask[pos] = (uint8_t)m;
       }
       pos0 += __popc(sel_m);
     }
@@ -252,7 +259,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   }
   // committed HCA entries
   for (int i = threadIdx.x; i < tm.n_hca; i += blockDim.x) {
-    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + ((size_t)hca_row0 + i) * rowb); kmask[base + i] = (uint8_t)validbits;
+    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + (size_t)hca_row(i) * rowb); kmask[base + i] = (uint8_t)validbits;
   }
   base += tm.n_hca;
   // committed window positions seen by at least one node of the tile
@@ -694,8 +701,15 @@ static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size
 // The pointer-gather kernel serves tiles whose committed CSA run is longer than twice the selection size (and every
 // tile when the caches do not allow TMA).  With capacities that rule such tiles out it is not launched, nor is the
 // merge kernel: the paired kernel merges the chunks of its own tiles.
-static bool gather_kernel_needed(const tsv_shape& s, const TvaPlan& p, bool tma) {
-  return !tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk);
+static bool gather_kernel_needed(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, bool tma) {
+  if (!tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk)) return true;
+  // paged pool: tiles whose cache rows cannot be fetched as 32-row boxes take the pointer-gather kernel as well
+  if (c.page_table) {
+    const int epp = c.page_tokens / s.m_csa, hpp = c.page_tokens / s.m_hca;
+    if (epp % kBoxRows) return true;
+    if (hpp % kBoxRows && s.max_L / s.m_hca > kHcaMiscMax) return true;
+  }
+  return false;
 }
 
 // Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
@@ -706,7 +720,7 @@ int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, con
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
-  if (gather_kernel_needed(s, p, prep.tma) &&
+  if (gather_kernel_needed(s, p, c, prep.tma) &&
       cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();
     return TSV_ERR_CUDA;
@@ -728,7 +742,7 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep
     const int r = launch_tva_tc_pair(s, p, prep, out, ws, status, st);
     if (r != TSV_OK) return r;
   }
-  if (gather_kernel_needed(s, p, p.tc_tma)) {
+  if (gather_kernel_needed(s, p, c, p.tc_tma)) {
     tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
     if (p.tc_chmax > 1) {

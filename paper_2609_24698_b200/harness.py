@@ -37,14 +37,15 @@ def fill_cache(cache: tsv.LayerCache, shape: synth.Shape, b: int, L: int, arrays
     dev = cache.L.device
     up = lambda a, t=dt: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev).to(t)
     cache.L[b] = int(L)
-    r0 = int(cache.csa_row0[b]); n = arrays["csa_kv"].shape[0]
+    n = arrays["csa_kv"].shape[0]
     assert n <= int(cache.csa_cap[b])
     if n:
-        cache.csa_kv[r0:r0 + n] = up(arrays["csa_kv"]); cache.csa_ik[r0:r0 + n] = up(arrays["csa_ik"])
-    h0 = int(cache.hca_row0[b]); n = arrays["hca_kv"].shape[0]
+        rows = cache.csa_row_index(shape, b, n)
+        cache.csa_kv[rows] = up(arrays["csa_kv"]); cache.csa_ik[rows] = up(arrays["csa_ik"])
+    n = arrays["hca_kv"].shape[0]
     assert n <= int(cache.hca_cap[b])
     if n:
-        cache.hca_kv[h0:h0 + n] = up(arrays["hca_kv"])
+        cache.hca_kv[cache.hca_row_index(shape, b, n)] = up(arrays["hca_kv"])
     cache.win_kv[b] = up(arrays["win"])
     f = torch.float32
     cache.csa_mx[b] = float(arrays["csa_mx"]); cache.csa_s[b] = float(arrays["csa_s"])
@@ -112,10 +113,13 @@ class VerifyEngine:
     """Owns the persistent caches, scratch pads, workspace and outputs of an n-layer stack."""
 
     def __init__(self, shape: synth.Shape, n_layers: int, csa_caps, hca_caps, max_L: int, flags: int = 0,
-                 want_topk: bool = False, device="cuda"):
+                 want_topk: bool = False, device="cuda", page_tokens: int = 0):
         self.shape, self.n_layers, self.device = shape, n_layers, device
         self.cshape = tsv.c_shape(shape, max_L, flags)
-        self.caches = [tsv.alloc_cache(shape, csa_caps, hca_caps, device) for _ in range(n_layers)]
+        if page_tokens:         # paged pool: per layer its own pool and page table (different shuffles)
+            self.caches = [tsv.alloc_cache_paged(shape, csa_caps, hca_caps, page_tokens, seed=l, device=device) for l in range(n_layers)]
+        else:
+            self.caches = [tsv.alloc_cache(shape, csa_caps, hca_caps, device) for _ in range(n_layers)]
         self.scratch = [tsv.alloc_scratch(shape, device) for _ in range(n_layers)]
         self.workspace = tsv.alloc_workspace(shape, max_L, flags, device)
         dt = tsv.torch_dtype(shape)

@@ -29,12 +29,12 @@ class Workload:
     inputs: List[hz.InputSet]
 
 
-def build(cfg: synth.Config, cycles_headroom: int, n_sets: int = 3, flags: int = 0, device="cuda") -> Workload:
+def build(cfg: synth.Config, cycles_headroom: int, n_sets: int = 3, flags: int = 0, device="cuda", page_tokens: int = 0) -> Workload:
     sh = cfg.shape
     lengths = synth.prefix_lengths(cfg)
     ccap, hcap = hz.capacities(sh, lengths, cycles_headroom * sh.D)
     max_L = int(lengths.max()) + (cycles_headroom + 1) * sh.D
-    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=False, device=device)
+    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=False, device=device, page_tokens=page_tokens)
     for l in range(cfg.layers):
         for b in range(sh.B):
             hz.fill_cache(eng.caches[l], sh, b, int(lengths[b]), direct_arrays(cfg, l, b, int(lengths[b])))

@@ -24,7 +24,7 @@ def _np(t):
 
 def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None, check_recompress=False,
              parent_fn=None, return_engine=False, plant=None, graph=False, recompress_pairs=None, on_cycle=None,
-             per_row=False, incremental_caches=False):
+             per_row=False, incremental_caches=False, page_tokens=0):
     """Advance oracle and device cycle by cycle from the same prefix; compare everything each cycle.
     out_pairs: None = compare attention outputs of every (layer, seq); else callable cycle -> iterable of pairs.
     plant: callable(states, lengths) editing the oracle's prefix states in place before they are uploaded.
@@ -35,6 +35,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
     on_cycle: callable(cycle, engine, states) for extra bookkeeping.
     incremental_caches: per cycle compare only the cache rows appended in that cycle (plus lengths, window, open-block
            states); all rows are compared after the last cycle and every tenth cycle.
+    page_tokens: the persistent caches live in a paged pool with pages of that many tokens (shuffled page tables).
     per_row: also require every (node, head) output row to be within the tolerance of ITS OWN max magnitude (for inputs
            where a few rows are far larger than the rest, so that the tensor-wide bound would say little about the others)."""
     from paper_2609_24698_b200 import binding as tsv, harness as hz
@@ -49,7 +50,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
                      for l in range(cfg.layers)]                 # per tensor: list of pieces, joined when checked
     ccap, hcap = hz.capacities(sh, lengths, cycles * sh.D)
     max_L = int(lengths.max()) + (cycles + 1) * sh.D
-    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=True)
+    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=True, page_tokens=page_tokens)
     for l in range(cfg.layers):
         for b in range(sh.B):
             hz.fill_cache(eng.caches[l], sh, b, int(lengths[b]), state_arrays(states[l][b]))
@@ -169,19 +170,26 @@ def compare_caches(eng, states, sh, tol, committed=None, recompress_pairs=None, 
         f = {k: _np(getattr(cache, k)) for k in ("csa_mx", "csa_s", "csa_acc_kv", "csa_acc_ik", "hca_mx", "hca_s", "hca_acc_kv")}
         lo_c = [0 if prev_L is None else prev_L[l][b] // sh.m_csa for b in range(sh.B)]
         lo_h = [0 if prev_L is None else prev_L[l][b] // sh.m_hca for b in range(sh.B)]
+        if cache.page_table is not None:                                        # paged pool: physical rows through the page table
+            tab = cache.page_table.cpu().numpy().astype(np.int64)
+            epp, hpp = cache.page_tokens // sh.m_csa, cache.page_tokens // sh.m_hca
+            phys_c = lambda b, i: int(tab[b, i // epp]) * epp + i % epp
+            phys_h = lambda b, i: int(tab[b, i // hpp]) * hpp + i % hpp
+        else:
+            phys_c = lambda b, i: int(r0c[b]) + i
+            phys_h = lambda b, i: int(r0h[b]) + i
         if prev_L is None:
             ckv, cik, hkv = _np(cache.csa_kv), _np(cache.csa_ik), _np(cache.hca_kv)
-            row_c = lambda b, i: r0c[b] + i
-            row_h = lambda b, i: r0h[b] + i
+            row_c, row_h = phys_c, phys_h
         else:                                                                     # gather only the appended rows
-            ic = [int(r0c[b]) + i for b, S in enumerate(states[l]) for i in range(lo_c[b], S.L // sh.m_csa)]
-            ih = [int(r0h[b]) + i for b, S in enumerate(states[l]) for i in range(lo_h[b], S.L // sh.m_hca)]
+            ic = [phys_c(b, i) for b, S in enumerate(states[l]) for i in range(lo_c[b], S.L // sh.m_csa)]
+            ih = [phys_h(b, i) for b, S in enumerate(states[l]) for i in range(lo_h[b], S.L // sh.m_hca)]
             tc_ = torch.tensor(ic, dtype=torch.long, device=cache.csa_kv.device)
             th_ = torch.tensor(ih, dtype=torch.long, device=cache.csa_kv.device)
             ckv, cik, hkv = _np(cache.csa_kv[tc_]), _np(cache.csa_ik[tc_]), _np(cache.hca_kv[th_])
             pc_, ph_ = {r: j for j, r in enumerate(ic)}, {r: j for j, r in enumerate(ih)}
-            row_c = lambda b, i: pc_[int(r0c[b]) + i]
-            row_h = lambda b, i: ph_[int(r0h[b]) + i]
+            row_c = lambda b, i: pc_[phys_c(b, i)]
+            row_h = lambda b, i: ph_[phys_h(b, i)]
         for b, S in enumerate(states[l]):
             assert int(Ls[b]) == S.L                                            # committed length: exact
             n_csa, n_hca = S.L // sh.m_csa, S.L // sh.m_hca
@@ -424,6 +432,29 @@ def test_budgets_beyond_eight_cuda_core_path(dtype):
 
 
 
+
+
+# ------------------------------------------------------------------------------------------------ paged pool
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_paged_pool_small(dtype):
+    """Caches in a paged pool (pages of 12 tokens = 6 CSA entries = 4 HCA entries, one shuffled page table for both
+    physical layers, pages of different sequences interleaved), CUDA-core path: ranked selections, blocks closing in the
+    tree, entries appended across page boundaries by the refresh; recompression check every cycle."""
+    cfg = synth.small_config(name="paged", dtype=dtype, B=5, D=7, H=4, d=32, m_csa=2, topk=8, HI=2, di=16, m_hca=3, window=9,
+                             L_min=0, L_max=80, layers=2, seed=93, cfg_id=93, sm_scale=2.0)
+    lockstep(cfg, cycles=8, check_recompress=True, page_tokens=12)
+
+
+@pytest.mark.parametrize("page_tokens,m_csa,topk,lengths", [(128, 4, 512, [300, 1100, 2040, 2500, 3900]), (128, 4, 128, [600, 900, 1500, 2600]),
+                                                            (256, 4, 512, [700, 1300, 2040]), (128, 16, 64, [900, 1500, 4000])])
+def test_paged_pool_tensor_core_path(page_tokens, m_csa, topk, lengths):
+    """Benchmark head shape over a paged pool.  128-token pages hold exactly one 32-row TMA box of CSA entries (m = 4) and
+    one HCA entry: contiguous-run tiles fetch page by page (single- and multi-chunk), ranked and long tiles gather by
+    pointer; 256-token pages hold two boxes; with m = 16 a page holds 8 CSA entries and every tile gathers by pointer."""
+    heads = dict(BENCH_HEADS, m_csa=m_csa)
+    cfg = synth.Config(f"paged_tc_{page_tokens}_{m_csa}_{topk}", 94, synth.Shape("bf16", len(lengths), 8, topk=topk, **heads), layers=1,
+                       L_min=1, L_max=1, seed=page_tokens + topk)
+    lockstep(cfg, cycles=3, lengths=lengths, page_tokens=page_tokens, check_recompress="final")
 
 # ------------------------------------------------------------------------------------------------ refresh schedules
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
