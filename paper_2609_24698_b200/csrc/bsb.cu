@@ -34,7 +34,8 @@ __device__ __forceinline__ void scalar_fold(FoldCoef& fc, float& mx_out, float& 
 
 constexpr int kBsbThreads = 128;
 
-template <typename T, int DMAX>
+// DEFER: the C128-deferred schedule is on (a separate instantiation, so that the timely schedule's code is untouched by it)
+template <typename T, int DMAX, bool DEFER>
 __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, const tsv_cache c, const tsv_nodes nd,
                                                           const tsv_scratch sc, int32_t* __restrict__ status) {
   extern __shared__ float hist[];                      // [D][kBsbThreads] post-fold value of this thread's element per node
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
   const float* pers = which == 0 ? c.csa_acc_kv : (which == 1 ? c.csa_acc_ik : c.hca_acc_kv);
   // C128-deferred schedule: the HCA slabs of a sequence in which no HCA block can close inside the tree have nothing to do
   // (they learn the length first, one load, and leave before fetching any vector)
-  if (which == 2 && (s.flags & TSV_FLAG_HCA_DEFERRED) && blockIdx.y * kBsbThreads >= (unsigned)(d + di) && hca_deferred(s, c.L[b])) return;
+  if (DEFER && which == 2 && blockIdx.y * kBsbThreads >= (unsigned)(d + di) && hca_deferred(s, c.L[b])) return;
   // issue this thread's loads before the scalar chain is known (padding slots load too: the memory is there)
   float cv[DMAX];
 #pragma unroll
@@ -70,7 +71,7 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
     for (int n = 0; n < DMAX; ++n) { gc[n] = __shfl_sync(0xffffffffu, gcl, n); gh[n] = __shfl_sync(0xffffffffu, ghl, n); }
   }
 
-  const bool hdef = hca_deferred(s, tm.L) && !tm.status;     // (tm.L is 0 for a flagged length: such a sequence commits nothing)
+  const bool hdef = DEFER && hca_deferred(s, tm.L) && !tm.status;     // (tm.L is 0 for a flagged length: such a sequence commits nothing)
   if (threadIdx.x == 0) {
     const bool writer = blockIdx.y == 0;
     if (tm.status && writer) atomicOr(status + b, tm.status);
@@ -129,17 +130,20 @@ int launch_bsb(const tsv_shape& s, const tsv_cache& c, const tsv_nodes& nd, cons
   const int elems = 2 * s.d + s.di;
   const dim3 grid(s.B, (elems + kBsbThreads - 1) / kBsbThreads);
   const size_t sm = (size_t)s.D * kBsbThreads * sizeof(float);
-  TSV_PREP((bsb_kernel<bf16, 8>));
-  TSV_PREP((bsb_kernel<float, 8>));
-  TSV_PREP((bsb_kernel<bf16, TSV_MAX_D>));
-  TSV_PREP((bsb_kernel<float, TSV_MAX_D>));
-  if (s.D <= 8) {
-    if (s.dtype == TSV_BF16) bsb_kernel<bf16, 8><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
-    else bsb_kernel<float, 8><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+  const bool defer = (s.flags & TSV_FLAG_HCA_DEFERRED) != 0, bf = s.dtype == TSV_BF16, small = s.D <= 8;
+#define TSV_BSB_LAUNCH(T_, DM_, DF_)                                              \
+  do {                                                                            \
+    TSV_PREP((bsb_kernel<T_, DM_, DF_>));                                         \
+    bsb_kernel<T_, DM_, DF_><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status); \
+  } while (0)
+  if (small) {
+    if (bf) { if (defer) TSV_BSB_LAUNCH(bf16, 8, true); else TSV_BSB_LAUNCH(bf16, 8, false); }
+    else { if (defer) TSV_BSB_LAUNCH(float, 8, true); else TSV_BSB_LAUNCH(float, 8, false); }
   } else {
-    if (s.dtype == TSV_BF16) bsb_kernel<bf16, TSV_MAX_D><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
-    else bsb_kernel<float, TSV_MAX_D><<<grid, kBsbThreads, sm, st>>>(s, c, nd, sc, status);
+    if (bf) { if (defer) TSV_BSB_LAUNCH(bf16, TSV_MAX_D, true); else TSV_BSB_LAUNCH(bf16, TSV_MAX_D, false); }
+    else { if (defer) TSV_BSB_LAUNCH(float, TSV_MAX_D, true); else TSV_BSB_LAUNCH(float, TSV_MAX_D, false); }
   }
+#undef TSV_BSB_LAUNCH
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }

@@ -60,6 +60,10 @@ struct RowAddr {
   __device__ __forceinline__ int64_t operator()(int e) const {
     return pt ? (int64_t)__ldg(pt + e / per_page) * per_page + e % per_page : row0 + e;
   }
+  // the same row relative to row0 (row0 is 0 in a paged pool): for code that keeps a base pointer of the slab
+  __device__ __forceinline__ int64_t rel(int e) const {
+    return pt ? (int64_t)__ldg(pt + e / per_page) * per_page + e % per_page : (int64_t)e;
+  }
 };
 __device__ __forceinline__ RowAddr csa_rows_of(const tsv_cache& c, const tsv_shape& s, int b) {
   RowAddr r;

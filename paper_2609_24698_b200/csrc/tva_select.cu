@@ -149,8 +149,8 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
 #pragma unroll
     for (int j = 0; j < V; ++j) { q[h][j] = h < HI ? t0[j] : 0.f; q[h][V + j] = h < HI ? t1[j] : 0.f; }
   }
-  const T* ik0 = reinterpret_cast<const T*>(c.csa_ik);
   const RowAddr ikr = csa_rows_of(c, s, b);
+  const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)ikr.row0 * di;
   float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
   const int n_csa = tm.n_csa, e_base = blockIdx.x * kRows256PerCta, e_end = min(n_csa, e_base + kRows256PerCta);
 #pragma unroll 1
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int e = base + grp + 32 * u;
-      const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)ikr(e < n_csa ? e : 0) * di) + gl * 2;
+      const uint4* rowp = reinterpret_cast<const uint4*>(ik0 + (size_t)ikr.rel(e < n_csa ? e : 0) * di) + gl * 2;
       raw[u][0] = __ldg(rowp); raw[u][1] = __ldg(rowp + 1);
     }
 #pragma unroll
@@ -187,7 +187,9 @@ __global__ void __launch_bounds__(256) idx_score_rows256_kernel(const tsv_shape 
 // staging area of the rows a ranking CTA scores itself (256-byte indexer rows, padded in shared memory)
 constexpr int kStageRows = 128, kStagePitch = 272;   // two buffers of kStageRows rows
 
-template <typename T>
+// PAGED: the caches live in a paged pool (a separate instantiation: the flat layout's ranking path is a tuned latency
+// chain and keeps exactly its code)
+template <typename T, bool PAGED>
 __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                    const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
                                                    int32_t* __restrict__ status) {
@@ -283,8 +285,9 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     const T* iq = reinterpret_cast<const T*>(nd.iq) + ((size_t)b * D + n) * HI * di;
     for (int i = threadIdx.x; i < HI * di; i += blockDim.x) iq_sm[i] = to_f(iq[i]);
     __syncthreads();
-    const T* ik0 = reinterpret_cast<const T*>(c.csa_ik);
-    const RowAddr ikr = csa_rows_of(c, s, b);
+    RowAddr ikr;
+    if (PAGED) ikr = csa_rows_of(c, s, b); else { ikr.pt = nullptr; ikr.per_page = 1; ikr.row0 = c.csa_row0[b]; }
+    const T* ik0 = reinterpret_cast<const T*>(c.csa_ik) + (size_t)ikr.row0 * di;
     float* sw = reinterpret_cast<float*>(ws + pl.off_scores) + ((size_t)b * D + n) * pl.score_ld;
     if ((size_t)di * sizeof(T) == 256 && HI <= 4 && blockDim.x == 256) {
       // Rows of 256 bytes (the benchmark's indexer width).  Few CTAs rank and each is a chain of its own, so load latency
@@ -312,12 +315,22 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
       auto issue = [&](int rd) {                         // rows [rd kStageRows, ..) into buffer rd & 1; one group per call
         const int base = rd * kStageRows, nrow = min(kStageRows, n_csa - base);
         const uint32_t dst = stage_s + (uint32_t)(rd & 1) * (kStageRows * kStagePitch);
+        if (PAGED) {                                       // paged pool: a page-table look-up per row
 #pragma unroll
-        for (int i = 0; i < kStageRows * 16 / 256; ++i) {
-          const int idx = threadIdx.x + 256 * i, row = idx >> 4, c16 = idx & 15;
-          if (row < nrow)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kStagePitch + c16 * 16),
-                         "l"(ikb + (size_t)ikr(base + row) * 256 + c16 * 16) : "memory");
+          for (int i = 0; i < kStageRows * 16 / 256; ++i) {
+            const int idx = threadIdx.x + 256 * i, row = idx >> 4, c16 = idx & 15;
+            if (row < nrow)
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kStagePitch + c16 * 16),
+                           "l"(ikb + (size_t)ikr.rel(base + row) * 256 + c16 * 16) : "memory");
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < kStageRows * 16 / 256; ++i) {
+            const int idx = threadIdx.x + 256 * i, row = idx >> 4, c16 = idx & 15;
+            if (row < nrow)
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + row * kStagePitch + c16 * 16),
+                           "l"(ikb + (size_t)(base + row) * 256 + c16 * 16) : "memory");
+          }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
       };
@@ -364,7 +377,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
         uint4 raw[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-          raw[u] = (c0 + u < di / V) ? __ldg(reinterpret_cast<const uint4*>(ik0 + (size_t)ikr(e) * di + (c0 + u) * V)) : make_uint4(0, 0, 0, 0);
+          raw[u] = (c0 + u < di / V) ? __ldg(reinterpret_cast<const uint4*>(ik0 + (size_t)(PAGED ? ikr.rel(e) : (int64_t)e) * di + (c0 + u) * V)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           if (c0 + u < di / V) {
@@ -605,16 +618,18 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
     }
   }
   dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
-  TSV_PREP(topk_kernel<bf16>);
-  TSV_PREP(topk_kernel<float>);
+  const bool paged = c.page_table != nullptr;
   size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...
   if (p.idx_fused && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) sm2 += (size_t)2 * kStageRows * kStagePitch + (size_t)kIdxFusedMax * sizeof(float);   // ... the staged rows (two buffers), the scores
-  if (sm2 > 48 * 1024) {
-    if (bf) cudaFuncSetAttribute(topk_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
-    else cudaFuncSetAttribute(topk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
-  }
-  if (bf) topk_kernel<bf16><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
-  else topk_kernel<float><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);
+#define TSV_TOPK_LAUNCH(T_, PG_)                                                                                        \
+  do {                                                                                                                  \
+    TSV_PREP((topk_kernel<T_, PG_>));                                                                                   \
+    if (sm2 > 48 * 1024) cudaFuncSetAttribute(topk_kernel<T_, PG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2); \
+    topk_kernel<T_, PG_><<<g2, 256, sm2, st>>>(s, p, c, nd, sc, topk_idx, ws, status);                                  \
+  } while (0)
+  if (bf) { if (paged) TSV_TOPK_LAUNCH(bf16, true); else TSV_TOPK_LAUNCH(bf16, false); }
+  else { if (paged) TSV_TOPK_LAUNCH(float, true); else TSV_TOPK_LAUNCH(float, false); }
+#undef TSV_TOPK_LAUNCH
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }

@@ -434,6 +434,29 @@ def test_budgets_beyond_eight_cuda_core_path(dtype):
 
 
 
+
+def test_refresh_skips_copies_nobody_reads():
+    """The refresh moves only what a later reader can see: when the last accepted node closes a CSA (HCA) block, the open
+    block is empty afterwards and its stored accumulator is never read, so it is not copied (the persistent accumulator
+    keeps its old bits); rejected branches are never copied at all.  Parity with the oracle holds through such cycles."""
+    cfg = synth.small_config(name="refresh_skip", dtype="bf16", B=8, D=8, H=4, d=32, m_csa=2, topk=8, HI=2, di=16, m_hca=4, window=10,
+                             L_min=0, L_max=40, layers=1, seed=95, cfg_id=95, p=0.8)
+    seen = {"csa": 0, "hca": 0}
+    prev = {}
+    def watch(cyc, eng, states):
+        c = eng.caches[0]
+        L = c.L.cpu().numpy()
+        for b in range(cfg.shape.B):
+            if cyc in prev:
+                if L[b] % cfg.shape.m_csa == 0 and L[b] != prev[cyc]["L"][b]:
+                    assert torch.equal(c.csa_acc_kv[b], prev[cyc]["csa"][b]); seen["csa"] += 1
+                if L[b] % cfg.shape.m_hca == 0 and L[b] != prev[cyc]["L"][b]:
+                    assert torch.equal(c.hca_acc_kv[b], prev[cyc]["hca"][b]); seen["hca"] += 1
+        prev[cyc + 1] = {"L": L.copy(), "csa": c.csa_acc_kv.clone(), "hca": c.hca_acc_kv.clone()}
+    lockstep(cfg, cycles=10, check_recompress=True, on_cycle=watch)
+    assert seen["csa"] > 5 and seen["hca"] > 2
+
+
 # ------------------------------------------------------------------------------------------------ paged pool
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_paged_pool_small(dtype):
