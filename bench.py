@@ -31,7 +31,7 @@ import numpy as np  # noqa: E402
 # attention stage with the bytes of ONE of its launches (one layer), and, where captured, the sum over all kernels of one
 # verify cycle.  The captures are summarised under profiles/; workloads without a capture report null.
 NCU_DRAM = {
-    "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 70_262_784, "cycle_bytes": None},   # 65.41 MB read + 4.85 MB written
+    "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 70_355_456, "cycle_bytes": None},   # 65.62 MB read + 4.73 MB written
     # cfg5: tc_attn_kernel 62.28 MB read + 19.15 MB written; all kernels of one cycle 191.7 MB (cold cache per kernel)
     "cfg5": {"kernel": "tc_attn_kernel", "launch_bytes": 81_427_712, "cycle_bytes": 191_703_808},
 }
