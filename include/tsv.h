@@ -128,14 +128,18 @@ typedef struct tsv_cache {
    * ONE table gives its physical page for every physical layer: entry e of the CSA cache (kv and indexer key) is row
    *     page_table[b][e / epp] * epp + e % epp,   epp = page_tokens / m_csa,
    * entry h of the HCA cache is row  page_table[b][h / hpp] * hpp + h % hpp,  hpp = page_tokens / m_hca.
+   * The third physical layer is the token-level KV: win_kv is then not a ring but a pool of tok_rows rows, the KV of the
+   * token at position p in row  page_table[b][p / page_tokens] * page_tokens + p % page_tokens  (only the last `window`
+   * positions of a sequence are ever read; the refresh writes position L + i of every accepted node).
    * csa_row0 / hca_row0 are ignored then (may be NULL); csa_cap / hca_cap still give the entries the sequence's assigned
-   * pages can hold.  page_tokens must be a multiple of m_csa and of m_hca.  The token-level window keeps its ring form
-   * (with window == page_tokens it is one page per sequence).  The tensor-core path fetches CSA rows by 32-row TMA boxes
-   * when epp is a multiple of 32 (e.g. 128-token pages with m_csa = 4: one box per page); otherwise, and for HCA rows
-   * beyond the first 32 entries unless hpp is a multiple of 32, it gathers rows by pointer. */
-  const int32_t *page_table;  /* [B][max_pages] device, or NULL: flat slabs                  */
+   * pages can hold, and the pages must cover positions up to L + D - 1.  page_tokens must be a multiple of m_csa and of
+   * m_hca.  The tensor-core path fetches rows by 32-row TMA boxes where a page holds whole boxes of the layer (CSA: epp a
+   * multiple of 32, e.g. 128-token pages with m_csa = 4: one box per page; window: page_tokens a multiple of 32); otherwise,
+   * and for HCA rows beyond the first 32 entries unless hpp is a multiple of 32, it gathers rows by pointer. */
+  const int32_t *page_table;  /* [B][max_pages] device, or NULL: flat slabs and window ring   */
   int32_t page_tokens;        /* HOST value                                                 */
   int32_t max_pages;          /* HOST value: columns of page_table                          */
+  int64_t tok_rows;           /* HOST value: rows allocated in win_kv when it is a token pool */
 } tsv_cache;
 
 /* Per-cycle inputs of ONE layer for all tree nodes; read-only. */

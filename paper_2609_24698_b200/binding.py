@@ -45,7 +45,7 @@ CACHE_TENSORS = ("L", "csa_kv", "csa_ik", "csa_row0", "csa_cap", "hca_kv", "hca_
 
 class CCache(C.Structure):
     _fields_ = [(n, _p) for n in CACHE_TENSORS] + [("csa_rows", C.c_int64), ("hca_rows", C.c_int64),
-                                                   ("page_table", _p), ("page_tokens", C.c_int32), ("max_pages", C.c_int32)]
+                                                   ("page_table", _p), ("page_tokens", C.c_int32), ("max_pages", C.c_int32), ("tok_rows", C.c_int64)]
 
 
 class CNodes(C.Structure):
@@ -130,7 +130,8 @@ class LayerCache:
     def struct(self) -> CCache:
         pt = self.page_table
         return CCache(*[_ptr(getattr(self, n)) for n in CACHE_TENSORS], int(self.csa_kv.shape[0]), int(self.hca_kv.shape[0]),
-                      _ptr(pt), int(self.page_tokens), 0 if pt is None else int(pt.shape[1]))
+                      _ptr(pt), int(self.page_tokens), 0 if pt is None else int(pt.shape[1]),
+                      0 if pt is None else int(self.win_kv.shape[0]))
 
     def clone(self) -> "LayerCache":
         return LayerCache(*[getattr(self, n).clone() for n in CACHE_TENSORS], page_table=self.page_table, page_tokens=self.page_tokens)
@@ -141,6 +142,12 @@ class LayerCache:
 
     def hca_row_index(self, shape: synth.Shape, b: int, n: int) -> torch.Tensor:
         return self._rows(b, n, self.hca_row0, shape.m_hca)
+
+    def tok_row_index(self, shape: synth.Shape, b: int, positions: torch.Tensor) -> torch.Tensor:
+        """Physical rows of win_kv that hold the token-level KV of the given positions of sequence b."""
+        if self.page_table is None:
+            return b * shape.window + positions % shape.window       # rows of win_kv viewed as [B * window, d]
+        return self.page_table[b].long()[positions // self.page_tokens] * self.page_tokens + positions % self.page_tokens
 
     def _rows(self, b: int, n: int, row0: torch.Tensor, block: int) -> torch.Tensor:
         e = torch.arange(n, dtype=torch.long, device=self.L.device)
@@ -211,7 +218,8 @@ def alloc_cache(shape: synth.Shape, csa_caps: Sequence[int], hca_caps: Sequence[
 def alloc_cache_paged(shape: synth.Shape, csa_caps: Sequence[int], hca_caps: Sequence[int], page_tokens: int, seed: int = 0,
                       device="cuda") -> LayerCache:
     """Empty caches over a paged pool: every sequence gets the pages its capacities ask for, drawn from one pool in a
-    shuffled order (pages of different sequences interleave), and ONE page table serves the CSA and the HCA layer."""
+    shuffled order (pages of different sequences interleave), and ONE page table serves the three physical layers: CSA
+    entries, HCA entries and the token-level KV (win_kv becomes a pool of page_tokens rows per page)."""
     import numpy as np
     assert page_tokens % shape.m_csa == 0 and page_tokens % shape.m_hca == 0
     epp, hpp = page_tokens // shape.m_csa, page_tokens // shape.m_hca
@@ -233,7 +241,7 @@ def alloc_cache_paged(shape: synth.Shape, csa_caps: Sequence[int], hca_caps: Seq
         L=torch.zeros(B, **i32), csa_kv=flat.csa_kv, csa_ik=flat.csa_ik,
         csa_row0=torch.zeros(B, dtype=torch.int64, device=device), csa_cap=torch.tensor([n * epp for n in need], **i32),
         hca_kv=flat.hca_kv, hca_row0=torch.zeros(B, dtype=torch.int64, device=device), hca_cap=torch.tensor([n * hpp for n in need], **i32),
-        win_kv=torch.zeros(B, shape.window, shape.d, dtype=dt, device=device),
+        win_kv=torch.zeros(n_pages * page_tokens, shape.d, dtype=dt, device=device),     # token-level pool, rows by position
         csa_mx=torch.zeros(B, **f32), csa_s=torch.zeros(B, **f32),
         csa_acc_kv=torch.zeros(B, shape.d, **f32), csa_acc_ik=torch.zeros(B, shape.di, **f32),
         hca_mx=torch.zeros(B, **f32), hca_s=torch.zeros(B, **f32), hca_acc_kv=torch.zeros(B, shape.d, **f32),

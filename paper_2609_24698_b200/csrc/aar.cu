@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(128) aar_commit_kernel(const tsv_shape s, cons
     const int n = accept_path[(size_t)b * D + i];
     const int pos = L + i;
     const size_t nidx = (size_t)b * D + n;
-    copy_row16((char*)ly.c.win_kv + ((size_t)b * s.window + pos % s.window) * rowb, (const char*)ly.node_kv + nidx * rowb, (int)rowb, tid, nt);
+    copy_row16((char*)ly.c.win_kv + (size_t)tok_row_of(ly.c, s, b, pos) * rowb, (const char*)ly.node_kv + nidx * rowb, (int)rowb, tid, nt);
     if (ly.sc.csa_done[nidx]) {
       const size_t row = (size_t)csa_rows_of(ly.c, s, b)(pos / s.m_csa);
       copy_row16((char*)ly.c.csa_kv + row * rowb, (const char*)ly.sc.new_csa_kv + nidx * rowb, (int)rowb, tid, nt);

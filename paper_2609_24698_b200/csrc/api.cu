@@ -85,7 +85,7 @@ static int check_cache(const tsv_cache* c, const tsv_shape* s) {
                        c->csa_mx, c->csa_s, c->csa_acc_kv, c->csa_acc_ik, c->hca_mx, c->hca_s, c->hca_acc_kv};
   for (const void* p : all) if (!p) return TSV_ERR_NULL;
   if (c->page_table) {      // paged pool: one table for all physical layers; the page size divides into whole blocks
-    if (c->page_tokens < 1 || c->max_pages < 1 || c->page_tokens % s->m_csa || c->page_tokens % s->m_hca) return TSV_ERR_SHAPE;
+    if (c->page_tokens < 1 || c->max_pages < 1 || c->page_tokens % s->m_csa || c->page_tokens % s->m_hca || c->tok_rows < 1) return TSV_ERR_SHAPE;
   } else if (!c->csa_row0 || !c->hca_row0) return TSV_ERR_NULL;
   const void* vec[] = {c->csa_kv, c->csa_ik, c->hca_kv, c->win_kv, c->csa_acc_kv, c->csa_acc_ik, c->hca_acc_kv};
   for (const void* p : vec) if (!al16(p)) return TSV_ERR_ALIGN;

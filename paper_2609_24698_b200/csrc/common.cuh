@@ -80,6 +80,12 @@ __device__ __forceinline__ RowAddr hca_rows_of(const tsv_cache& c, const tsv_sha
   return r;
 }
 
+// Row of the token-level KV of position pos: slot pos % window of the sequence's ring, or through the page table.
+__device__ __forceinline__ int64_t tok_row_of(const tsv_cache& c, const tsv_shape& s, int b, int pos) {
+  if (c.page_table) return (int64_t)__ldg(c.page_table + (size_t)b * c.max_pages + pos / c.page_tokens) * c.page_tokens + pos % c.page_tokens;
+  return (int64_t)b * s.window + pos % s.window;
+}
+
 // ---------------------------------------------------------------- tree metadata
 // Built by ONE thread of a CTA into shared memory, then read by all after a barrier.
 struct TreeMeta {

@@ -56,7 +56,7 @@ __device__ __forceinline__ const T* key_row(int j, const NodeKeys& nk, const Tre
   j -= nk.n_hca;
   if (j < nk.n_newh) return reinterpret_cast<const T*>(sc.new_hca_kv) + ((size_t)b * s.D + nk.newh[j]) * d;
   j -= nk.n_newh;
-  if (j < nk.n_win) return reinterpret_cast<const T*>(c.win_kv) + ((size_t)b * s.window + (nk.win_lo + j) % s.window) * d;
+  if (j < nk.n_win) return reinterpret_cast<const T*>(c.win_kv) + (size_t)tok_row_of(c, s, b, nk.win_lo + j) * d;
   j -= nk.n_win;
   return reinterpret_cast<const T*>(nd.kv) + ((size_t)b * s.D + nk.tree[j]) * d;
 }

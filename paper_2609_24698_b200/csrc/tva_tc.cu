@@ -54,7 +54,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   csa_row.per_page = c.page_table ? c.page_tokens / s.m_csa : 1; hca_row.per_page = c.page_table ? c.page_tokens / s.m_hca : 1;
   csa_row.row0 = row0_sm[0]; hca_row.row0 = row0_sm[1];
   // runs of consecutive rows exist in a paged pool only where a page holds whole 32-row boxes of the layer
-  const bool csa_runs = !c.page_table || csa_row.per_page % kBoxRows == 0, hca_runs = !c.page_table || hca_row.per_page % kBoxRows == 0;
+  const bool csa_runs = !c.page_table || (csa_row.per_page % kBoxRows == 0 && c.page_tokens % kBoxRows == 0), hca_runs = !c.page_table || hca_row.per_page % kBoxRows == 0;
   if (blockIdx.x >= (unsigned)pl.tc_nt) {
     // The extra CTA of the sequence (grid x = tiles + 1): rows that are small and scattered (few HCA entries, tree nodes,
     // entries closed inside the tree) are packed into one contiguous per-sequence buffer so that TMA boxes can fetch
@@ -181,7 +181,11 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       // four runs, each padded to whole boxes: committed CSA entries, HCA entries (when too many for the packed rows),
       // the window ring, the packed rows.  One pass over all keys: a thread finds the run of its key by comparison, so
       // the runs' (short, latency-bound) mask computations overlap instead of following each other.
-      const int cnt[4] = {n_csa, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, min(tm.L, s.window), n_misc};
+      // the window: the ring in slot order, or (paged pool) the positions from the 32-aligned start of the box that holds
+      // the oldest window position up to L - 1 (the positions before the window are masked like every position a node
+      // cannot see)
+      const int win_a = c.page_table ? (max(0, tm.L - s.window) & ~(kBoxRows - 1)) : 0;
+      const int cnt[4] = {n_csa, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, c.page_table ? tm.L - win_a : min(tm.L, s.window), n_misc};
       const int64_t start[4] = {0, 0, (int64_t)b * s.window, (int64_t)b * pl.tc_misc_rows};
       int k0[5];                                       // first key of each run
       k0[0] = 0;
@@ -192,7 +196,8 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         const int k = bi * kBoxRows;
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
         // (a box of a cache run never crosses a page: it starts on a multiple of 32 entries and per_page is one too)
-        box[bi] = make_int2(g, (int)(g == 0 ? csa_row(k - k0[0]) : g == 1 ? hca_row(k - k0[1]) : start[g] + (k - k0[g])));
+        box[bi] = make_int2(g, (int)(g == 0 ? csa_row(k - k0[0]) : g == 1 ? hca_row(k - k0[1]) : (g == 2 && c.page_table) ? tok_row_of(c, s, b, win_a + k - k0[2])
+                                                                                                            : start[g] + (k - k0[g])));
       }
       for (int k = threadIdx.x; k < kb; k += blockDim.x) {
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
@@ -202,7 +207,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
           if (g == 0) m = dense ? validbits : cmask[i];
           else if (g == 1) m = validbits;
           else if (g == 2) {
-            const int pos = tm.L - 1 - ((tm.L - 1 - i) % s.window);
+            const int pos = c.page_table ? win_a + i : tm.L - 1 - ((tm.L - 1 - i) % s.window);
             for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
           } else if (i < nh_in) m = validbits;
           else if (i < nh_in + tm.nn) {
@@ -269,7 +274,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int pos = lo + i;
     uint32_t m = 0;
     for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
-    kptr[base + i] = (uint64_t)((const char*)c.win_kv + ((size_t)b * s.window + pos % s.window) * rowb); kmask[base + i] = (uint8_t)m;
+    kptr[base + i] = (uint64_t)((const char*)c.win_kv + (size_t)tok_row_of(c, s, b, pos) * rowb); kmask[base + i] = (uint8_t)m;
   }
   base += max(0, tm.L - lo);
   __syncthreads();
@@ -691,7 +696,8 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   int64_t mk = uni + s.max_L / s.m_hca + s.window + 3 * (int64_t)s.D + 8;
   const int64_t br = kBoxRows;
   p.tc_misc_rows = (int32_t)((kHcaMiscMax + 3 * s.D + br - 1) / br * br);
-  const int64_t runs = (p.cand_cap + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + p.tc_misc_rows;
+  // (+ one box: in a paged pool the window run starts on a 32-aligned position and may be a box longer than the window)
+  const int64_t runs = (p.cand_cap + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
   if (runs > mk) mk = runs;
   p.tc_maxk = (int32_t)((mk + 127) / 128 * 128);
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
@@ -706,7 +712,7 @@ static bool gather_kernel_needed(const tsv_shape& s, const TvaPlan& p, const tsv
   // paged pool: tiles whose cache rows cannot be fetched as 32-row boxes take the pointer-gather kernel as well
   if (c.page_table) {
     const int epp = c.page_tokens / s.m_csa, hpp = c.page_tokens / s.m_hca;
-    if (epp % kBoxRows) return true;
+    if (epp % kBoxRows || c.page_tokens % kBoxRows) return true;
     if (hpp % kBoxRows && s.max_L / s.m_hca > kHcaMiscMax) return true;
   }
   return false;

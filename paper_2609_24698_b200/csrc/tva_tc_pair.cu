@@ -685,7 +685,7 @@ static_assert(sizeof(pair::MapSet) <= sizeof(TvaTcPrep::maps), "tensor-map block
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
   pair::MapSet& ms = *reinterpret_cast<pair::MapSet*>(prep.maps);
   const void* bases[4] = {c.csa_kv, c.hca_kv, c.win_kv, ws + p.off_misc};
-  const int64_t rows[4] = {c.csa_rows, c.hca_rows, (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
+  const int64_t rows[4] = {c.csa_rows, c.hca_rows, c.page_table ? c.tok_rows : (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
   bool ok = make_map(&ms.q, nd.q, (int64_t)s.B * s.D * s.H, 128) && make_map(&ms.out, out, (int64_t)s.B * s.D * s.H, 32);
   for (int a = 0; a < 4 && ok; ++a)
     for (int k = 0; k < 3 && ok; ++k) ok = make_map(&ms.src[a][k], bases[a], rows[a], 32 << k);

@@ -46,7 +46,12 @@ def fill_cache(cache: tsv.LayerCache, shape: synth.Shape, b: int, L: int, arrays
     assert n <= int(cache.hca_cap[b])
     if n:
         cache.hca_kv[cache.hca_row_index(shape, b, n)] = up(arrays["hca_kv"])
-    cache.win_kv[b] = up(arrays["win"])
+    if cache.page_table is None:
+        cache.win_kv[b] = up(arrays["win"])
+    else:                       # token-level pool: the last min(L, window) positions, taken from their ring slots
+        pos = torch.arange(max(0, int(L) - shape.window), int(L), dtype=torch.long, device=dev)
+        if pos.numel():
+            cache.win_kv[cache.tok_row_index(shape, b, pos)] = up(arrays["win"])[pos % shape.window]
     f = torch.float32
     cache.csa_mx[b] = float(arrays["csa_mx"]); cache.csa_s[b] = float(arrays["csa_s"])
     cache.hca_mx[b] = float(arrays["hca_mx"]); cache.hca_s[b] = float(arrays["hca_s"])

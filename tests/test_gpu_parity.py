@@ -198,7 +198,12 @@ def compare_caches(eng, states, sh, tol, committed=None, recompress_pairs=None, 
             rh = [row_h(b, i) for i in range(lo_h[b], n_hca)]
             assert rel_err(ckv[rc], S.csa_kv[lo_c[b]:]) <= tol and rel_err(cik[rc], S.csa_ik[lo_c[b]:]) <= tol
             assert rel_err(hkv[rh], S.hca_kv[lo_h[b]:]) <= tol
-            assert np.array_equal(win[b], S.win)                                 # token-level KV: copies, exact
+            if cache.page_table is None:
+                assert np.array_equal(win[b], S.win)                             # token-level KV: copies, exact
+            else:                                                                # token pool: the window's positions, by page
+                for pos in range(max(0, S.L - sh.window), S.L):
+                    r = int(tab[b, pos // cache.page_tokens]) * cache.page_tokens + pos % cache.page_tokens
+                    assert np.array_equal(win[r], S.win[pos % sh.window])
             assert f["csa_mx"][b] == S.csa_part.mx and f["hca_mx"][b] == S.hca_part.mx
             assert abs(f["csa_s"][b] - S.csa_part.s) <= TOL_STATE * max(1.0, S.csa_part.s)
             assert abs(f["hca_s"][b] - S.hca_part.s) <= TOL_STATE * max(1.0, S.hca_part.s)
