@@ -61,6 +61,10 @@ void launch_idx_score_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& 
                          int32_t* status, cudaStream_t st);
 int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
+// per-node top-k of long candidate lists by a thread-block cluster per node
+bool topk_long_applies(const tsv_shape& s, const TvaPlan& p);
+int launch_topk_long(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                     int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
 
@@ -72,7 +76,7 @@ bool tva_tc_pair_usable(const tsv_cache& c);
 // Host-side preparation of the tensor-core attention path: everything that can fail on the host (tensor maps, kernel
 // attributes) is done here, before any kernel of the call is enqueued.
 struct TvaTcPrep {
-  alignas(64) unsigned char maps[14 * 128];   // the paired kernel's tensor maps (a CUtensorMap is 128 bytes)
+  alignas(64) unsigned char maps[19 * 128];   // the paired kernel's tensor maps (a CUtensorMap is 128 bytes)
   int32_t tma;                                // the contiguous-run path is usable for these caches
 };
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);

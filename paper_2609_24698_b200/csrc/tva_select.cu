@@ -8,27 +8,9 @@
 //   topk_kernel       one CTA per (sequence, node): 4-pass 8-bit radix select on the order-
 //                     preserving integer image of the fp32 score, then one ordered compaction
 //                     pass.  In-tree entries (closed at strict ancestors) are scored here.
-#include "kernels.h"
+#include "select_common.cuh"
 
 namespace tsv {
-
-// Strict ancestors of n that closed a CSA / HCA block, root first (ascending block index).
-struct PathEntries {
-  int32_t n_newc, n_newh;
-  int32_t newc[TSV_MAX_D], newc_blk[TSV_MAX_D];
-  int32_t newh[TSV_MAX_D];
-};
-
-__device__ inline void path_entries(PathEntries& pe, const TreeMeta& tm, const tsv_shape& s, int n,
-                                    const uint8_t* csa_done_b, const uint8_t* hca_done_b) {
-  pe.n_newc = pe.n_newh = 0;
-  const uint32_t a = tm.anc[n] & ~(1u << n);
-  for (int j = 0; j < n; ++j) {
-    if (!((a >> j) & 1u)) continue;
-    if (csa_done_b[j]) { pe.newc[pe.n_newc] = j; pe.newc_blk[pe.n_newc++] = (tm.L + tm.depth[j]) / s.m_csa; }
-    if (hca_done_b[j]) pe.newh[pe.n_newh++] = j;
-  }
-}
 
 template <typename T>
 __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
@@ -97,11 +79,6 @@ __global__ void __launch_bounds__(256) idx_score_kernel(const tsv_shape s, const
       }
     }
   }
-}
-
-__device__ __forceinline__ uint32_t order_key(float f) {       // larger float -> larger key
-  const uint32_t u = __float_as_uint(f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
 // 16 raw bytes of storage elements widened to fp32 (the tag argument selects the storage type)
@@ -202,37 +179,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
   if (blockIdx.x == (unsigned)s.D) {
-    // Extra CTA column (only with the tensor-core attention path): CTA (D, 0) ranks the 256-row tiles of all sequences by
-    // the number of keys they will stage, most first, so that the paired attention kernel starts the long tiles first
-    // and the short ones fill the tail.  The counts follow from lengths, node counts and done flags alone (for tiles on
-    // the contiguous-run path they are exact; for pointer-gather tiles an estimate: only the order depends on them), so
-    // the ranking is ready before the plan kernel runs and each plan CTA can leave its record at its final position.
-    if (blockIdx.y != 0) return;
-    __shared__ int32_t nk_est[2048];
-    const int D = s.D, nt = pl.tc_nt, ntile = s.B * nt, npt = 256 / s.H;
-    int32_t* pos = reinterpret_cast<int32_t*>(ws + pl.off_pos);
-    if (ntile > 2048) { for (int i = threadIdx.x; i < ntile; i += blockDim.x) pos[i] = i; return; }
-    auto r32 = [](int x) { return (x + kBoxRows - 1) / kBoxRows * kBoxRows; };
-    for (int i = threadIdx.x; i < ntile; i += blockDim.x) {
-      const int b = i / nt, tile = i - b * nt;
-      const int L = c.L[b], nn = nd.n_nodes[b];
-      int est = 0;
-      if (L >= 0 && (int64_t)L + D <= s.max_L && nn >= 1 && nn <= D && tile * npt < nn) {
-        int ncd = 0, nhd = 0;
-        for (int j = 0; j < nn; ++j) { ncd += sc.csa_done[(size_t)b * D + j] != 0; nhd += sc.hca_done[(size_t)b * D + j] != 0; }
-        const int n_csa = L / s.m_csa, n_hca = L / s.m_hca, nh_in = n_hca <= kHcaMiscMax ? n_hca : 0, win = min(L, s.window);
-        if (n_csa <= 2 * s.topk) est = r32(n_csa) + (n_hca > kHcaMiscMax ? r32(n_hca) : 0) + r32(win) + r32(nh_in + nn + ncd + nhd);
-        else est = min(n_csa, npt * s.topk) + n_hca + win + 3 * nn;
-      }
-      nk_est[i] = est;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < ntile; i += blockDim.x) {
-      const int ki = nk_est[i];
-      int rank = 0;
-      for (int j = 0; j < ntile; ++j) { const int kj = nk_est[j]; rank += (kj > ki) || (kj == ki && j < i); }
-      pos[i] = rank;
-    }
+    // extra CTA column (only with the tensor-core attention path): CTA (D, 0) ranks the attention tiles
+    if (blockIdx.y == 0) rank_tiles(s, pl, c, nd, sc, ws);
     return;
   }
   const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk;
@@ -617,6 +565,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
       count_launch();
     }
   }
+  if (topk_long_applies(s, p)) return launch_topk_long(s, p, c, nd, sc, topk_idx, ws, status, st);
   dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
   const bool paged = c.page_table != nullptr;
   size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...

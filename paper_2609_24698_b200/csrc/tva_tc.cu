@@ -38,7 +38,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   uint64_t* kptr = reinterpret_cast<uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
-  const int32_t* selcnt = reinterpret_cast<const int32_t*>(ws + pl.off_selcnt) + (size_t)b * D;
   const int32_t* sel = reinterpret_cast<const int32_t*>(ws + pl.off_sel) + (size_t)b * D * s.topk;
   // the done flags and the cache row offsets are fetched together with the tree scalars (one memory latency for all)
   __shared__ uint8_t cdone[TSV_MAX_D], hdone[TSV_MAX_D];
@@ -175,8 +174,37 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     // Ranked nodes still take the contiguous-run path while the run is at most twice the selection size: all committed
-    // entries are staged and the unselected ones are masked per node.
-    if ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax)) {
+    // entries are staged and the unselected ones are masked per node.  Beyond that (or where a paged pool's pages do not
+    // hold whole boxes) the tile is GATHERED: the same four runs, but the first holds only the committed entries some node
+    // of the tile selected, and every key is named by its row (array << 30 | row) for four-row TMA gathers.
+    const bool runs_ok = (dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax);
+    int n_uni = n_csa;                                 // keys of the first run
+    __shared__ int uni_tot;
+    uint32_t* krow = reinterpret_cast<uint32_t*>(kptr);
+    if (!runs_ok) {
+      // Ordered compaction of the selected entries: a thread owns a contiguous share of the entries, counts its selected
+      // ones (four mask bytes per word), one block scan, then writes its rows and masks at consecutive positions.
+      __shared__ int wsum_c[9];
+      const uint32_t* cm32 = reinterpret_cast<const uint32_t*>(cmask);
+      const int per = ((n_csa + 255) / 256 + 3) & ~3, beg = min(n_csa, (int)threadIdx.x * per), end = min(n_csa, beg + per);
+      const uint32_t dmask = dense ? validbits : 0u;  // (a dense tile comes here only from a paged pool with odd pages)
+      int cnt = 0;
+      for (int i = beg; i < end; i += 4) {
+        uint32_t w = dense ? 0x01010101u * dmask : cm32[i >> 2];
+        if (end - i < 4) w &= (1u << (8 * (end - i))) - 1u;
+        cnt += (w & 0xFFu ? 1 : 0) + (w & 0xFF00u ? 1 : 0) + (w & 0xFF0000u ? 1 : 0) + (w & 0xFF000000u ? 1 : 0);
+      }
+      int total;
+      int pos = block_excl_scan_256(cnt, wsum_c, total);
+      if (threadIdx.x == 0) uni_tot = total;
+      for (int i = beg; i < end; ++i) {
+        const uint32_t m = dense ? dmask : (uint32_t)cmask[i];
+        if (m) { krow[pos] = (uint32_t)csa_row(i); kmask[pos] = (uint8_t)m; ++pos; }
+      }
+      __syncthreads();
+      n_uni = uni_tot;
+    }
+    {
       int2* box = reinterpret_cast<int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
       // four runs, each padded to whole boxes: committed CSA entries, HCA entries (when too many for the packed rows),
       // the window ring, the packed rows.  One pass over all keys: a thread finds the run of its key by comparison, so
@@ -185,26 +213,31 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       // the oldest window position up to L - 1 (the positions before the window are masked like every position a node
       // cannot see)
       const int win_a = c.page_table ? (max(0, tm.L - s.window) & ~(kBoxRows - 1)) : 0;
-      const int cnt[4] = {n_csa, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, c.page_table ? tm.L - win_a : min(tm.L, s.window), n_misc};
+      const int cnt[4] = {n_uni, tm.n_hca > kHcaMiscMax ? tm.n_hca : 0, c.page_table ? tm.L - win_a : min(tm.L, s.window), n_misc};
       const int64_t start[4] = {0, 0, (int64_t)b * s.window, (int64_t)b * pl.tc_misc_rows};
       int k0[5];                                       // first key of each run
       k0[0] = 0;
 #pragma unroll
       for (int g = 0; g < 4; ++g) k0[g + 1] = k0[g] + (cnt[g] + kBoxRows - 1) / kBoxRows * kBoxRows;
       const int kb = k0[4];
-      for (int bi = threadIdx.x; bi < kb / kBoxRows; bi += blockDim.x) {
-        const int k = bi * kBoxRows;
-        const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
-        // (a box of a cache run never crosses a page: it starts on a multiple of 32 entries and per_page is one too)
-        box[bi] = make_int2(g, (int)(g == 0 ? csa_row(k - k0[0]) : g == 1 ? hca_row(k - k0[1]) : (g == 2 && c.page_table) ? tok_row_of(c, s, b, win_a + k - k0[2])
-                                                                                                            : start[g] + (k - k0[g])));
+      // row of key i of run g (g >= 1, or the whole CSA slab as run 0 of a contiguous-run tile)
+      auto run_row = [&](int g, int i) -> int64_t {
+        return g == 0 ? csa_row(i) : g == 1 ? hca_row(i) : (g == 2 && c.page_table) ? tok_row_of(c, s, b, win_a + i) : start[g] + i;
+      };
+      if (runs_ok) {
+        for (int bi = threadIdx.x; bi < kb / kBoxRows; bi += blockDim.x) {
+          const int k = bi * kBoxRows;
+          const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
+          // (a box of a cache run never crosses a page: it starts on a multiple of 32 entries and per_page is one too)
+          box[bi] = make_int2(g, (int)run_row(g, k - k0[g]));
+        }
       }
       for (int k = threadIdx.x; k < kb; k += blockDim.x) {
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
         const int i = k - k0[g];
         uint32_t m = 0;
         if (i < cnt[g]) {
-          if (g == 0) m = dense ? validbits : cmask[i];
+          if (g == 0) m = runs_ok ? (dense ? validbits : cmask[i]) : kmask[k];
           else if (g == 1) m = validbits;
           else if (g == 2) {
             const int pos = c.page_table ? win_a + i : tm.L - 1 - ((tm.L - 1 - i) % s.window);
@@ -225,8 +258,10 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
           }
         }
         kmask[k] = (uint8_t)m;
+        // gathered tiles: the key's row; the padding of a run repeats the run's first row (masked)
+        if (!runs_ok && (g > 0 || i >= cnt[0])) krow[k] = ((uint32_t)g << 30) | (uint32_t)(cnt[g] ? run_row(g, i < cnt[g] ? i : 0) : 0);
       }
-      if (threadIdx.x == 0) { *nkeys = kb; *mode = 1; }
+      if (threadIdx.x == 0) { *nkeys = kb; *mode = runs_ok ? 1 : 2; }
       return;
     }
   }
@@ -289,14 +324,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         if (j == n) continue;
         if (hdone[j]) mh |= 1u << nl;
         if (cdone[j]) {
-          bool in = n_cand[nl] <= s.topk;
-          if (!in) {                                         // ranked: is the entry's block index in the node's selection?
-            const int blk = (tm.L + tm.depth[j]) / s.m_csa, cnt = selcnt[n];
-            const int32_t* sl = sel + (size_t)n * s.topk;
-            int a = 0, z = cnt - 1;
-            while (a <= z) { const int mid = (a + z) >> 1; const int v = sl[mid]; if (v == blk) { in = true; break; } if (v < blk) a = mid + 1; else z = mid - 1; }
-          }
-          if (in) mc |= 1u << nl;
+          if (newc_selected(nl, j)) mc |= 1u << nl;        // ranked nodes: is the entry in the node's selection?
         }
       }
       const size_t nrow = (size_t)b * D + j;
@@ -631,7 +659,7 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   const size_t tix = (size_t)b * pl.tc_nt + tile, rix = (size_t)b * 2 * pl.tc_nt + rt;
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   int nch, CL;
-  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] == 1) return;     // the paired kernel merges its own chunks
+  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 0) return;     // a tile of the paired kernel
   chunking(nk, nch, CL);
   if (nk <= 0 || nch <= 1) return;
   const int rows_seq = s.D * s.H, row0 = rt * BM;
@@ -683,6 +711,67 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   }
 }
 
+// Merge of the paired kernel's tiles of more than two chunks: every chunk left its NORMALISED partial output (bf16) with
+// the row's (reference max, sum); the row's output is the average of the partial outputs weighted by sum * 2^(max - row max).
+// grid (128-row tiles, sequences, groups of 8 rows): a warp merges one row, a lane owns 16 consecutive columns; the chunks
+// are accumulated in order, four chunks' loads in flight.
+__global__ void __launch_bounds__(256) tc_combine_pair_kernel(const tsv_shape s, const TvaPlan pl, void* __restrict__ out_, const char* __restrict__ ws) {
+  using namespace tc;
+  const int rt = blockIdx.x, tile = rt >> 1, b = blockIdx.y;
+  const size_t tix = (size_t)b * pl.tc_nt + tile, rix = (size_t)b * 2 * pl.tc_nt + rt;
+  const int mode = reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix];
+  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
+  if ((mode != 1 && mode != 2) || nk <= 0) return;
+  int nch, CL;
+  chunking_x(nk, nch, CL);
+  if (nch <= 2) return;                                          // the paired kernel wrote or merged these itself
+  const int rows_seq = s.D * s.H, row0 = rt * BM;
+  const int lane = threadIdx.x & 31, row = blockIdx.z * 8 + (threadIdx.x >> 5);
+  if (row >= BM || row0 + row >= rows_seq) return;
+  // (a chunk's bf16 tile lies at the start of the chunk's slot of BM x DH floats)
+  const uint4* po = reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(ws + pl.off_tpo) + (rix * pl.tc_chmax * 2 * BM + row) * DH) + 2 * lane;
+  const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM + row;
+  float m = -INFINITY;
+  for (int ch = lane; ch < nch; ch += 32) { const float2 ml = pml[(size_t)ch * BM]; if (ml.y > 0.f) m = fmaxf(m, ml.x); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float l = 0.f, acc[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+  for (int c0 = 0; c0 < nch; c0 += 4) {
+    float2 ml[4];
+    uint4 v[4][2];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int ch = c0 + u < nch ? c0 + u : nch - 1;
+      ml[u] = pml[(size_t)ch * BM];
+      v[u][0] = po[(size_t)ch * 2 * BM * (DH / 8)]; v[u][1] = po[(size_t)ch * 2 * BM * (DH / 8) + 1];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (c0 + u >= nch || !(ml[u].y > 0.f)) continue;
+      const float w = ml[u].y * exp2f(ml[u].x - m);
+      l += w;
+      const uint32_t wd[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w, v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        acc[2 * k] = fmaf(__uint_as_float(wd[k] << 16), w, acc[2 * k]);
+        acc[2 * k + 1] = fmaf(__uint_as_float(wd[k] & 0xFFFF0000u), w, acc[2 * k + 1]);
+      }
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  uint32_t o[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+    o[k] = *reinterpret_cast<const uint32_t*>(&h2);
+  }
+  uint4* orow = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0 + row) * DH) + 2 * lane;
+  orow[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  orow[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 bool tva_tc_eligible(const tsv_shape& s) {
   return s.dtype == TSV_BF16 && s.d == tc::DH && s.H >= 32 && s.H <= 128 && (128 % s.H) == 0 && !(s.flags & TSV_FLAG_FORCE_SIMT);
 }
@@ -699,24 +788,17 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   // (+ one box: in a paged pool the window run starts on a 32-aligned position and may be a box longer than the window)
   const int64_t runs = (p.cand_cap + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
   if (runs > mk) mk = runs;
+  // gathered tiles: the union of the nodes' selections, HCA entries, window and packed rows as four runs padded to boxes
+  const int64_t gath = (uni + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
+  if (gath > mk) mk = gath;
   p.tc_maxk = (int32_t)((mk + 127) / 128 * 128);
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
 }
 
 static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) : 0; }   // node bits per entry, cleared by words
-// The pointer-gather kernel serves tiles whose committed CSA run is longer than twice the selection size (and every
-// tile when the caches do not allow TMA).  With capacities that rule such tiles out it is not launched, nor is the
-// merge kernel: the paired kernel merges the chunks of its own tiles.
-static bool gather_kernel_needed(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, bool tma) {
-  if (!tma || (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk)) return true;
-  // paged pool: tiles whose cache rows cannot be fetched as 32-row boxes take the pointer-gather kernel as well
-  if (c.page_table) {
-    const int epp = c.page_tokens / s.m_csa, hpp = c.page_tokens / s.m_hca;
-    if (epp % kBoxRows || c.page_tokens % kBoxRows) return true;
-    if (hpp % kBoxRows && s.max_L / s.m_hca > kHcaMiscMax) return true;
-  }
-  return false;
-}
+// The pointer-gather kernel (and its merge kernel) serves every tile when the caches do not allow TMA (the caller gave no
+// row counts of the cache arrays); otherwise all tiles go to the paired kernel.
+static bool gather_kernel_needed(bool tma) { return !tma; }
 
 // Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
@@ -726,7 +808,7 @@ int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, con
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
-  if (gather_kernel_needed(s, p, c, prep.tma) &&
+  if (gather_kernel_needed(prep.tma) &&
       cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();
     return TSV_ERR_CUDA;
@@ -734,6 +816,7 @@ int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, con
   TSV_PREP(tc_plan_kernel);
   TSV_PREP(tc_attn_kernel);
   TSV_PREP(tc_combine_kernel);
+  TSV_PREP(tc_combine_pair_kernel);
   if (prep.tma) return prepare_tva_tc_pair(s, p, c, nd, out, ws, prep);
   return TSV_OK;
 }
@@ -747,8 +830,12 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep
   if (p.tc_tma) {
     const int r = launch_tva_tc_pair(s, p, prep, out, ws, status, st);
     if (r != TSV_OK) return r;
+    if ((p.tc_maxk + tc::NCX - 1) / tc::NCX > 2) {               // some tile may have more than two chunks
+      tc_combine_pair_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);
+      count_launch();
+    }
   }
-  if (gather_kernel_needed(s, p, c, p.tc_tma)) {
+  if (gather_kernel_needed(p.tc_tma)) {
     tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
     count_launch();
     if (p.tc_chmax > 1) {

@@ -1,5 +1,6 @@
-// tree_verify_attn, tensor-core kernel for key lists made of contiguous runs, run by PAIRS of CTAs
-// (thread-block cluster of 2, tcgen05 cta_group::2).
+// tree_verify_attn, tensor-core kernel run by PAIRS of CTAs (thread-block cluster of 2, tcgen05 cta_group::2), for key
+// lists made of contiguous runs (fetched as TMA boxes) and for key lists of scattered rows (fetched four rows at a
+// time by TMA gather).
 //
 // A pair covers 256 query rows of one sequence (256/H consecutive tree nodes x H heads); each CTA owns
 // 128 of them in its own tensor memory.  The two SMs execute every MMA together (M = 256): the B operand
@@ -75,6 +76,12 @@ __device__ __forceinline__ void tma_box2(uint32_t dst, const CUtensorMap* map, i
   asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
 }
+// four rows of a 2D tensor, given by their row indices, as four consecutive 128-byte lines of this CTA's shared memory
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int x, const uint4& code, uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"((int)(code.x & 0x3FFFFFFFu)), "r"((int)(code.y & 0x3FFFFFFFu)),
+                 "r"((int)(code.z & 0x3FFFFFFFu)), "r"((int)(code.w & 0x3FFFFFFFu)), "r"(bar_cluster_addr) : "memory");
+}
 __device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
@@ -105,7 +112,10 @@ struct alignas(64) MapSet {
   CUtensorMap q;          // 128-row boxes
   CUtensorMap out;        // 32-row boxes (stores)
   CUtensorMap src[4][3];  // [csa, hca, window, packed misc][32, 64, 128 rows]
+  CUtensorMap row[4];     // the same arrays with one-row boxes: gathers of four rows by index
+  CUtensorMap part;       // normalised partial outputs of tiles of more than two chunks (bf16, 32-row boxes, stores)
 };
+constexpr int NMAPS = 19;
 
 constexpr uint32_t OOB_BOX = 0x3FFFFF00u;   // map 0, a row beyond every tensor: the box is zero-filled
 
@@ -131,11 +141,12 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const size_t tix = (size_t)b * pl.tc_nt + tile;
-  if (tid < 14)      // the descriptors of all 14 tensor maps are fetched while the plan is read
+  if (tid < NMAPS)   // the descriptors of all tensor maps are fetched while the plan is read
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps) + (uint64_t)tid * sizeof(CUtensorMap)) : "memory");
   const size_t rix = (size_t)b * 2 * pl.tc_nt + 2 * tile + rank;  // this CTA's 128-row tile (partials of multi-chunk tiles)
   // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
-  if (rec.y != 1) return;                                      // not a contiguous-run tile
+  if (rec.y != 1 && rec.y != 2) return;                        // neither a contiguous-run tile nor a gathered one
+  const bool gather = rec.y == 2;                              // the key list is a list of row codes (array << 30 | row), not of boxes
   const int nk = rec.z;
   const int rows_seq = s.D * s.H, row0 = tile * PR + (int)rank * BM;           // first of this CTA's rows within the sequence
   if (nk <= 0) {                                               // flagged sequence or padding-only tile: zeros
@@ -174,7 +185,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   {
     const int2* box_g = reinterpret_cast<const int2*>(ws + pl.off_box) + tix * (size_t)(pl.tc_maxk / kBoxRows);
     const uint8_t* kmask_g = reinterpret_cast<const uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
-    if (tid < NCX / kBoxRows) {
+    if (tid < NCX / kBoxRows && !gather) {
       uint32_t v = OOB_BOX;
       if (cbeg + tid * kBoxRows < cend) { const int2 bx = box_g[cbeg / kBoxRows + tid]; v = ((uint32_t)bx.x << 30) | (uint32_t)bx.y; }
       sm.box[tid] = v;
@@ -218,11 +229,23 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       }
       __syncwarp();
     };
+    // Gathered tiles: the keys' row codes stay in global memory (the tile plan left them there, four-aligned groups
+    // never mix arrays); lane l fetches the codes of rows 4 l .. 4 l + 3 of a stage itself.  Keys past the end of the list
+    // read row 0 of the first array (they are masked).
+    // (the list shares the tile's slot of 8 bytes per key with the row pointers of the pointer-gather kernel)
+    const uint4* code_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(ws + pl.off_kptr + tix * (size_t)pl.tc_maxk * 8) + cbeg);
+    auto codes_at = [&](int key) { return cbeg + key < cend ? __ldg(code_g + (key >> 2)) : make_uint4(0u, 0u, 0u, 0u); };
+    uint4 kcode = make_uint4(0u, 0u, 0u, 0u);                                // this lane's codes of the current piece's K stages
+    int kcode_pc = -1;
     auto issue_k = [&](int gk) {
       const int pc = gk >> 3, dk = gk & 7, sl = gk % NKS, use = gk / NKS;
       const uint32_t slot = ring + (uint32_t)(NQS + sl) * SLOTP;
       const uint32_t fb_leader = map_to_rank(smem_u32(&sm.fullK[sl]), 0);
       const int bytes = min(256, CL - pc * 256) * 64;                        // bytes THIS CTA copies in the stage
+      if (gather && kcode_pc != pc) {                                        // this CTA's half of the piece's keys: bytes / 128 rows
+        kcode_pc = pc;
+        if (lane * 512 < bytes) kcode = codes_at(pc * 256 + (int)rank * (bytes >> 7) + 4 * lane);
+      }
       if (lane == 0) {
         if (use > 0 && !fail && !mbar_wait(&sm.emptyK[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
         if (rank == 0) mbar_expect_tx(&sm.fullK[sl], 2 * bytes);              // bytes of both CTAs
@@ -230,7 +253,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
       __syncwarp();
       // this CTA's half of the piece's keys: boxes [rank * nb, rank * nb + nb) of the piece
       const int nb = bytes / BOXB, i0 = pc * (256 / kBoxRows) + (int)rank * nb;
-      if (consecutive(i0, nb)) {                                             // nb = 4 (128 rows) or 2 (64 rows)
+      if (gather) {
+        if (lane * 512 < bytes) tma_gather4(slot + lane * 512, &maps.row[kcode.x >> 30], dk * 64, kcode, fb_leader);
+      } else if (consecutive(i0, nb)) {                                             // nb = 4 (128 rows) or 2 (64 rows)
         if (lane == 0) { const uint32_t bx = sm.box[i0]; tma_box2(slot, &maps.src[bx >> 30][nb == 4 ? 2 : 1], dk * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
       } else if (lane < nb) {
         const uint32_t bx = sm.box[i0 + lane];
@@ -255,12 +280,17 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         const int sl = gv % NSX, use = gv / NSX;
         const uint32_t slot = ring + (uint32_t)sl * SLOTP;
         const uint32_t fb_leader = map_to_rank(smem_u32(&sm.fullV[sl]), 0);
+        uint4 vcode = make_uint4(0u, 0u, 0u, 0u);                 // (fetched before the wait for the slot)
+        if (gather) vcode = codes_at(NQ == 2 ? kb * 64 + 4 * (lane & 15) : kb * 128 + 4 * lane);
         if (lane == 0) {
           if (use > 0 && !fail && !mbar_wait(&sm.emptyV[sl], (uint32_t)(use - 1) & 1u)) fail = 1;
           if (rank == 0) mbar_expect_tx(&sm.fullV[sl], 2 * SLOTP);
         }
         __syncwarp();
-        if (NQ == 2) {            // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
+        if (gather) {             // NQ == 2: 16 row groups x 2 slices of 64 dims; else 32 row groups x this CTA's 64 dims
+          if (NQ == 2) tma_gather4(slot + (lane >> 4) * 8192 + (lane & 15) * 512, &maps.row[vcode.x >> 30], (part * 4 + (int)rank * 2 + (lane >> 4)) * 64, vcode, fb_leader);
+          else tma_gather4(slot + lane * 512, &maps.row[vcode.x >> 30], (part * 2 + (int)rank) * 64, vcode, fb_leader);
+        } else if (NQ == 2) {     // 64 keys x this CTA's 128 dims: key boxes i = 0..1, 64-wide slices j = 0..1
           const int i0 = kb * (64 / kBoxRows);
           if (consecutive(i0, 2)) {
             if (lane < 2) { const uint32_t bx = sm.box[i0]; tma_box2(slot + lane * 8192, &maps.src[bx >> 30][1], (part * 4 + (int)rank * 2 + lane) * 64, (int)(bx & 0x3FFFFFFFu), fb_leader); }
@@ -512,8 +542,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         const uint32_t* r0 = ro + cg * 64;
         const uint32_t* r1 = ro + cg * 64 + 32;
         const int col = part * OW + hh * cw + c0;
-        if (nch == 1 && full_tile) {
-          // stage the 32 x 64 bf16 tile in the 128-byte swizzle pattern and store it with one TMA request
+        if ((nch == 1 && full_tile) || nch > 2) {
+          // stage the 32 x 64 bf16 tile in the 128-byte swizzle pattern and store it with one TMA request: into the output,
+          // or (tiles of more than two chunks) into the chunk's tile of normalised partial outputs, which a merge kernel
+          // combines with the chunks' (max, sum)
           if (store_pending) {
             if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             __syncwarp();
@@ -533,8 +565,11 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
           if (lane == 0) {
+            const CUtensorMap* omap = nch > 2 ? &maps.part : &maps.out;
+            // (a chunk's bf16 tile lies at the start of the chunk's slot for an fp32 tile: 2 BM rows of 1 KiB per slot)
+            const int orow = nch > 2 ? (int)((rix * pl.tc_chmax + chunk) * 2 * BM) + q4 * 32 : b * rows_seq + row0 + q4 * 32;
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                         ::"l"(reinterpret_cast<uint64_t>(&maps.out)), "r"(col), "r"(b * rows_seq + row0 + q4 * 32), "r"(stage) : "memory");
+                         ::"l"(reinterpret_cast<uint64_t>(omap)), "r"(col), "r"(orow), "r"(stage) : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           store_pending = true;
@@ -567,9 +602,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
     }
     if (store_pending && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    if (nch > 1) {
-      // Tiles of several chunks: each chunk leaves its unnormalised part of O with (max, sum) per row; the CTA that
+    if (nch == 2) {
+      // Tiles of two chunks: each chunk leaves its unnormalised part of O with (max, sum) per row; the CTA that
       // finishes a 128-row tile last merges the parts (fixed order, so the result does not depend on who was last).
+      // (More chunks: a merge kernel follows; one CTA would take too long over them.)
       __threadfence();
       compute_sync();
       if (warp == 2 && lane == 0) {
@@ -681,14 +717,20 @@ bool tva_tc_pair_usable(const tsv_cache& c) { return c.csa_rows > 0 && c.hca_row
 static_assert(sizeof(pair::MapSet) <= sizeof(TvaTcPrep::maps), "tensor-map block of TvaTcPrep too small");
 
 // Everything of the paired kernel's launch that can fail on the host, done before any kernel of the call is enqueued:
-// the 14 tensor maps and the kernel's shared-memory attribute.
+// the tensor maps and the kernel's shared-memory attribute.
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
   pair::MapSet& ms = *reinterpret_cast<pair::MapSet*>(prep.maps);
   const void* bases[4] = {c.csa_kv, c.hca_kv, c.win_kv, ws + p.off_misc};
   const int64_t rows[4] = {c.csa_rows, c.hca_rows, c.page_table ? c.tok_rows : (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
   bool ok = make_map(&ms.q, nd.q, (int64_t)s.B * s.D * s.H, 128) && make_map(&ms.out, out, (int64_t)s.B * s.D * s.H, 32);
-  for (int a = 0; a < 4 && ok; ++a)
+  for (int a = 0; a < 4 && ok; ++a) {
     for (int k = 0; k < 3 && ok; ++k) ok = make_map(&ms.src[a][k], bases[a], rows[a], 32 << k);
+    ok = ok && make_map(&ms.row[a], bases[a], rows[a], 1);
+  }
+  // partial outputs: per (128-row tile, chunk) a slot of 128 x 512 fp32 (tiles of two chunks); tiles of more than two
+  // chunks store 128 x 512 bf16 at the start of the slot: as rows of 1 KiB the buffer has 2 x 128 rows per slot
+  if (p.tc_chmax > 2) ok = ok && make_map(&ms.part, ws + p.off_tpo, (int64_t)s.B * 2 * p.tc_nt * p.tc_chmax * 2 * tc::BM, 32);
+  else ms.part = ms.out;                                                       // (never used: no tile has more than two chunks)
   if (!ok) {
     fprintf(stderr, "tsv: cuTensorMapEncodeTiled failed\n");
     return TSV_ERR_CUDA;

@@ -24,7 +24,7 @@ def _np(t):
 
 def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None, check_recompress=False,
              parent_fn=None, return_engine=False, plant=None, graph=False, recompress_pairs=None, on_cycle=None,
-             per_row=False, incremental_caches=False, page_tokens=0):
+             per_row=False, incremental_caches=False, page_tokens=0, exact_topk=False):
     """Advance oracle and device cycle by cycle from the same prefix; compare everything each cycle.
     out_pairs: None = compare attention outputs of every (layer, seq); else callable cycle -> iterable of pairs.
     plant: callable(states, lengths) editing the oracle's prefix states in place before they are uploaded.
@@ -36,6 +36,8 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
     incremental_caches: per cycle compare only the cache rows appended in that cycle (plus lengths, window, open-block
            states); all rows are compared after the last cycle and every tenth cycle.
     page_tokens: the persistent caches live in a paged pool with pages of that many tokens (shuffled page tables).
+    exact_topk: the device's selection must BE the oracle's (for inputs whose scores tie exactly, where the tie band of the
+           usual check would accept a wrong tie-break).
     per_row: also require every (node, head) output row to be within the tolerance of ITS OWN max magnitude (for inputs
            where a few rows are far larger than the rest, so that the tensor-wide bound would say little about the others)."""
     from paper_2609_24698_b200 import binding as tsv, harness as hz
@@ -127,6 +129,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
             g_idx = eng.topk_idx[l][b].cpu().numpy()
             same = all([check_topk(sh, states[l][b], nb, parent[b], n, scs[(l, b)], g_idx[n], ref_sel[n]) for n in range(nn)])
             assert np.all(g_idx[nn:] == -1)
+            assert same or not exact_topk, f"cycle {cyc} layer {l} seq {b}: selection differs from the oracle's"
             if not same:       # inside the tie band: evaluate the oracle with the device's selection
                 ref_out, _ = O.tree_verify_attn(states[l][b], sh, nb, parent[b], nn, scs[(l, b)], forced_sel=[g_idx[n] for n in range(nn)])
             e = rel_err(_np(eng.out[l][b]), ref_out)
@@ -356,6 +359,33 @@ def test_long_candidate_lists_tensor_core_scoring(D, HI):
     cfg = synth.small_config(name=f"long_lists_tc_d{D}_hi{HI}", dtype="bf16", B=3, D=D, H=4, d=16, m_csa=2, topk=24, HI=HI,
                              di=128, m_hca=32, window=16, L_min=4200, L_max=5200, layers=1, seed=78 + HI, cfg_id=73)
     lockstep(cfg, cycles=2)
+
+
+def _plant_tied_indexer_keys(every=60):
+    """`plant` hook: every committed CSA entry gets the indexer key of entry 0, except each `every`-th one, so that the
+    k-th largest score is shared by nearly all candidates and the selection is decided by the tie rule (lower index)."""
+    def hook(states, lengths):
+        for layer in states:
+            for S in layer:
+                keep = np.arange(S.csa_ik.shape[0]) % every == every - 1
+                S.csa_ik[~keep] = S.csa_ik[0]
+    return hook
+
+
+@pytest.mark.parametrize("dtype,di", [("fp32", 8), ("bf16", 128)])
+def test_long_candidate_lists_exact_ties_across_the_cluster(dtype, di):
+    """Long lists are selected by a cluster of CTAs per node, each holding a share of the candidates: with nearly all
+    scores equal, the threshold's ties span every CTA of the cluster and the lowest indices must win."""
+    cfg = synth.small_config(name="long_ties", dtype=dtype, B=3, D=6, H=4, d=16, m_csa=2, topk=100, HI=2, di=di, m_hca=32,
+                             window=16, L_min=4700, L_max=5600, layers=1, seed=91, cfg_id=74)
+    lockstep(cfg, cycles=2, plant=_plant_tied_indexer_keys(), exact_topk=True)
+
+
+def test_candidate_lists_beyond_the_cluster_capacity():
+    """More than 65536 candidates per node: the single-CTA selection that re-reads the score array pass after pass."""
+    cfg = synth.small_config(name="huge_lists", dtype="bf16", B=1, D=4, H=4, d=16, m_csa=2, topk=40, HI=2, di=128, m_hca=64,
+                             window=16, L_min=131500, L_max=131500, layers=1, seed=92, cfg_id=75)
+    lockstep(cfg, cycles=1)
 
 
 def test_ranked_short_candidate_lists_bf16():
