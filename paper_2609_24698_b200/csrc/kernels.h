@@ -80,7 +80,8 @@ struct TvaTcPrep {
   int32_t tma;                                // the contiguous-run path is usable for these caches
 };
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
-int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, void* out, char* ws, int32_t* status, cudaStream_t st);
+// general: gathered tiles or tiles of more than two chunks may occur (else the instantiation without that code runs)
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, bool general, void* out, char* ws, int32_t* status, cudaStream_t st);
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,

@@ -26,6 +26,9 @@ namespace tsv {
 
 
 // ------------------------------------------------------------------------------------------------ plan
+// GENERAL: gathered tiles may occur (see gathered_tiles_possible); the instantiation without them keeps the short
+// latency chain of the contiguous-run plan.
+template <bool GENERAL>
 __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
                                              const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
   __shared__ TreeMeta tm;
@@ -177,7 +180,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     // entries are staged and the unselected ones are masked per node.  Beyond that (or where a paged pool's pages do not
     // hold whole boxes) the tile is GATHERED: the same four runs, but the first holds only the committed entries some node
     // of the tile selected, and every key is named by its row (array << 30 | row) for four-row TMA gathers.
-    const bool runs_ok = (dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax);
+    const bool runs_ok = !GENERAL || ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax));
     int n_uni = n_csa;                                 // keys of the first run
     __shared__ int uni_tot;
     uint32_t* krow = reinterpret_cast<uint32_t*>(kptr);
@@ -339,6 +342,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
 // Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the scheduling
 // position the selection kernel computed for it (most keys first): the paired attention kernel takes the tiles in that
 // order and learns all it needs about its tile from one load.
+template <bool GENERAL>
 __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
@@ -348,7 +352,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   if (tile_cta && threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // (when the attention stage runs alone: the previous call's)
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
-  tc_plan_tile(s, pl, c, nd, sc, ws, cmask_sm);
+  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm);
   if (tile_cta && threadIdx.x == 0) {                 // thread 0 wrote the tile's key count and mode itself
     if (pos < 0 || pos >= s.B * pl.tc_nt) pos = (int)tix;
     reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
@@ -799,12 +803,24 @@ static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size
 // The pointer-gather kernel (and its merge kernel) serves every tile when the caches do not allow TMA (the caller gave no
 // row counts of the cache arrays); otherwise all tiles go to the paired kernel.
 static bool gather_kernel_needed(bool tma) { return !tma; }
+// Can the plan kernel produce a gathered tile for these capacities?  (A committed CSA run longer than twice the
+// selection size, or a paged pool whose pages do not hold whole 32-row boxes of a layer.)
+static bool gathered_tiles_possible(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c) {
+  if (p.need_scores && p.cand_cap > 2 * (int64_t)s.topk) return true;
+  if (c.page_table) {
+    const int epp = c.page_tokens / s.m_csa, hpp = c.page_tokens / s.m_hca;
+    if (epp % kBoxRows || c.page_tokens % kBoxRows) return true;
+    if (hpp % kBoxRows && s.max_L / s.m_hca > kHcaMiscMax) return true;
+  }
+  return false;
+}
 
 // Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
   prep.tma = tva_tc_pair_usable(c) ? 1 : 0;
   const size_t plan_sm = plan_smem_bytes(p);
-  if (plan_sm > 32 * 1024 && cudaFuncSetAttribute(tc_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess) {
+  if (plan_sm > 32 * 1024 && (cudaFuncSetAttribute(tc_plan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess ||
+                              cudaFuncSetAttribute(tc_plan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)) {
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
@@ -813,7 +829,8 @@ int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, con
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
-  TSV_PREP(tc_plan_kernel);
+  TSV_PREP(tc_plan_kernel<true>);
+  TSV_PREP(tc_plan_kernel<false>);
   TSV_PREP(tc_attn_kernel);
   TSV_PREP(tc_combine_kernel);
   TSV_PREP(tc_combine_pair_kernel);
@@ -825,12 +842,16 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
   TvaPlan p = p_in;
   p.tc_tma = prep.tma;
-  tc_plan_kernel<<<dim3(p.tc_nt + (p.tc_tma ? 1 : 0), s.B), 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);   // x: tiles (+ the packing CTA)
+  const bool gathered = !p.tc_tma || gathered_tiles_possible(s, p, c);
+  const dim3 pgrid(p.tc_nt + (p.tc_tma ? 1 : 0), s.B);                                                            // x: tiles (+ the packing CTA)
+  if (gathered) tc_plan_kernel<true><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
+  else tc_plan_kernel<false><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
   count_launch();
   if (p.tc_tma) {
-    const int r = launch_tva_tc_pair(s, p, prep, out, ws, status, st);
+    const bool many = (p.tc_maxk + tc::NCX - 1) / tc::NCX > 2;   // some tile may have more than two chunks
+    const int r = launch_tva_tc_pair(s, p, prep, many || gathered, out, ws, status, st);
     if (r != TSV_OK) return r;
-    if ((p.tc_maxk + tc::NCX - 1) / tc::NCX > 2) {               // some tile may have more than two chunks
+    if (many) {
       tc_combine_pair_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);
       count_launch();
     }

@@ -126,6 +126,11 @@ constexpr uint32_t OOB_BOX = 0x3FFFFF00u;   // map 0, a row beyond every tensor:
 //   K stages:  piece after piece, per slice dk  [this CTA's half of the piece's keys x 64 dims]
 //   V stages (after the last S product): CL <= 512: per half of d, per 64 keys:  [64 keys x this CTA's 128 of the half's 256 dims]
 //                                        else       per quarter of d, per 128 keys: [128 keys x this CTA's 64 of the quarter's 128 dims]
+//
+// GENERAL: gathered tiles and tiles of more than two chunks may occur.  Shapes whose capacities rule both out (the
+// benchmark's) run the instantiation without that code: the kernel is one long dependency chain per tile and its
+// timing follows the code layout.
+template <bool GENERAL>
 __global__ void __launch_bounds__(pair::TTHREADS, 1)
 tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s,
                     const TvaPlan pl, void* __restrict__ out_, char* __restrict__ ws, int32_t* __restrict__ status) {
@@ -141,12 +146,12 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const size_t tix = (size_t)b * pl.tc_nt + tile;
-  if (tid < NMAPS)   // the descriptors of all tensor maps are fetched while the plan is read
+  if (tid < (GENERAL ? NMAPS : 14))   // the descriptors of the tensor maps in use are fetched while the plan is read
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps) + (uint64_t)tid * sizeof(CUtensorMap)) : "memory");
   const size_t rix = (size_t)b * 2 * pl.tc_nt + 2 * tile + rank;  // this CTA's 128-row tile (partials of multi-chunk tiles)
   // every exit below is taken by both CTAs of the pair alike (it depends on the pair's plan only)
-  if (rec.y != 1 && rec.y != 2) return;                        // neither a contiguous-run tile nor a gathered one
-  const bool gather = rec.y == 2;                              // the key list is a list of row codes (array << 30 | row), not of boxes
+  if (rec.y != 1 && !(GENERAL && rec.y == 2)) return;          // neither a contiguous-run tile nor a gathered one
+  const bool gather = GENERAL && rec.y == 2;                              // the key list is a list of row codes (array << 30 | row), not of boxes
   const int nk = rec.z;
   const int rows_seq = s.D * s.H, row0 = tile * PR + (int)rank * BM;           // first of this CTA's rows within the sequence
   if (nk <= 0) {                                               // flagged sequence or padding-only tile: zeros
@@ -542,7 +547,8 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         const uint32_t* r0 = ro + cg * 64;
         const uint32_t* r1 = ro + cg * 64 + 32;
         const int col = part * OW + hh * cw + c0;
-        if ((nch == 1 && full_tile) || nch > 2) {
+        const bool many = GENERAL && nch > 2;
+        if ((nch == 1 && full_tile) || many) {
           // stage the 32 x 64 bf16 tile in the 128-byte swizzle pattern and store it with one TMA request: into the output,
           // or (tiles of more than two chunks) into the chunk's tile of normalised partial outputs, which a merge kernel
           // combines with the chunks' (max, sum)
@@ -565,9 +571,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
           if (lane == 0) {
-            const CUtensorMap* omap = nch > 2 ? &maps.part : &maps.out;
+            const CUtensorMap* omap = many ? &maps.part : &maps.out;
             // (a chunk's bf16 tile lies at the start of the chunk's slot for an fp32 tile: 2 BM rows of 1 KiB per slot)
-            const int orow = nch > 2 ? (int)((rix * pl.tc_chmax + chunk) * 2 * BM) + q4 * 32 : b * rows_seq + row0 + q4 * 32;
+            const int orow = many ? (int)((rix * pl.tc_chmax + chunk) * 2 * BM) + q4 * 32 : b * rows_seq + row0 + q4 * 32;
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
                          ::"l"(reinterpret_cast<uint64_t>(omap)), "r"(col), "r"(orow), "r"(stage) : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -602,7 +608,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
     }
     if (store_pending && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    if (nch == 2) {
+    if (GENERAL ? nch == 2 : nch > 1) {
       // Tiles of two chunks: each chunk leaves its unnormalised part of O with (max, sum) per row; the CTA that
       // finishes a 128-row tile last merges the parts (fixed order, so the result does not depend on who was last).
       // (More chunks: a merge kernel follows; one CTA would take too long over them.)
@@ -735,15 +741,17 @@ int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c
     fprintf(stderr, "tsv: cuTensorMapEncodeTiled failed\n");
     return TSV_ERR_CUDA;
   }
-  if (cudaFuncSetAttribute(tc_attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_X) != cudaSuccess) {
+  if (cudaFuncSetAttribute(tc_attn_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_X) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_attn_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_X) != cudaSuccess) {
     fprintf(stderr, "tsv: cannot set %d bytes of dynamic shared memory: %s\n", pair::SMEM_X, cudaGetErrorString(cudaGetLastError()));
     return TSV_ERR_CUDA;
   }
-  TSV_PREP(tc_attn_pair_kernel);
+  TSV_PREP(tc_attn_pair_kernel<true>);
+  TSV_PREP(tc_attn_pair_kernel<false>);
   return TSV_OK;
 }
 
-int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, void* out, char* ws, int32_t* status, cudaStream_t st) {
+int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, bool general, void* out, char* ws, int32_t* status, cudaStream_t st) {
   const pair::MapSet& ms = *reinterpret_cast<const pair::MapSet*>(prep.maps);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * p.tc_nt * s.B, p.tc_chmax, 1);
@@ -755,10 +763,11 @@ int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& pr
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel, ms, s, p, out, ws, status);
+  const cudaError_t le = general ? cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel<true>, ms, s, p, out, ws, status)
+                                 : cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel<false>, ms, s, p, out, ws, status);
   if (le != cudaSuccess) {
     int ncl = -1;
-    cudaOccupancyMaxActiveClusters(&ncl, tc_attn_pair_kernel, &cfg);
+    cudaOccupancyMaxActiveClusters(&ncl, tc_attn_pair_kernel<true>, &cfg);
     fprintf(stderr, "tsv: cluster launch failed: %s (max active clusters %d, grid %d x %d x %d)\n", cudaGetErrorString(le), ncl,
             cfg.gridDim.x, cfg.gridDim.y, cfg.gridDim.z);
   }
