@@ -133,10 +133,17 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   // Ranked nodes: node bits per committed CSA entry (cmask) and, per node, which blocks closed inside the tree are in
   // its selection (bit = block index - n_csa).  One pass over the selections of all the tile's nodes: the loads of a
   // batch are issued together (the tile CTA of a ranked sequence is on the critical path of the whole stage).
+  //
+  // Where gathered tiles may occur the array is padded by one word after every `per` entries (per: the power of two that
+  // spreads the entries over the CTA's threads): the compaction below gives a thread `per` consecutive entries, and
+  // without the padding the threads of a warp would all read the same bank.
   __shared__ uint32_t newc_bits[8];
+  int psh = 3;                                         // log2(per)
+  if (GENERAL) while ((256 << psh) < n_csa) ++psh;
+  auto phys = [&](int i) { return GENERAL ? i + ((i >> psh) << 2) : i; };
   if (!dense) {
     uint32_t* cm32 = reinterpret_cast<uint32_t*>(cmask);
-    for (int i = threadIdx.x; i < (n_csa + 3) / 4; i += blockDim.x) cm32[i] = 0;
+    for (int i = threadIdx.x; i < (phys(n_csa) + 3) / 4; i += blockDim.x) cm32[i] = 0;
     if (threadIdx.x < 8) newc_bits[threadIdx.x] = 0;
     __syncthreads();
     uint32_t allbits = 0;                              // nodes that take every committed entry
@@ -154,13 +161,13 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         if (idx[u] < 0) continue;
-        if (idx[u] < n_csa) atomicOr(cm32 + (idx[u] >> 2), (1u << nls[u]) << (8 * (idx[u] & 3)));
+        if (idx[u] < n_csa) atomicOr(cm32 + (phys(idx[u]) >> 2), (1u << nls[u]) << (8 * (idx[u] & 3)));
         else if (idx[u] - n_csa < 32) atomicOr(&newc_bits[nls[u]], 1u << (idx[u] - n_csa));
       }
     }
     __syncthreads();
     if (allbits) {
-      for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[i] |= (uint8_t)allbits;
+      for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[phys(i)] |= (uint8_t)allbits;
       __syncthreads();
     }
   }
@@ -185,24 +192,30 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     __shared__ int uni_tot;
     uint32_t* krow = reinterpret_cast<uint32_t*>(kptr);
     if (!runs_ok) {
-      // Ordered compaction of the selected entries: a thread owns a contiguous share of the entries, counts its selected
-      // ones (four mask bytes per word), one block scan, then writes its rows and masks at consecutive positions.
+      // Ordered compaction of the selected entries: a thread owns `per` consecutive entries, counts its selected ones
+      // (four mask bytes per word), one block scan, then writes its rows and masks at consecutive positions.
       __shared__ int wsum_c[9];
       const uint32_t* cm32 = reinterpret_cast<const uint32_t*>(cmask);
-      const int per = ((n_csa + 255) / 256 + 3) & ~3, beg = min(n_csa, (int)threadIdx.x * per), end = min(n_csa, beg + per);
-      const uint32_t dmask = dense ? validbits : 0u;  // (a dense tile comes here only from a paged pool with odd pages)
+      const int per = 1 << psh, beg = min(n_csa, (int)threadIdx.x << psh), end = min(n_csa, beg + per);
+      const uint32_t* mine = cm32 + (phys(beg) >> 2);  // this thread's words (its share starts on a word: per is a multiple of 8)
+      const uint32_t dmask = dense ? validbits : 0u;   // (a dense tile comes here only from a paged pool with odd pages)
       int cnt = 0;
       for (int i = beg; i < end; i += 4) {
-        uint32_t w = dense ? 0x01010101u * dmask : cm32[i >> 2];
+        uint32_t w = dense ? 0x01010101u * dmask : mine[(i - beg) >> 2];
         if (end - i < 4) w &= (1u << (8 * (end - i))) - 1u;
         cnt += (w & 0xFFu ? 1 : 0) + (w & 0xFF00u ? 1 : 0) + (w & 0xFF0000u ? 1 : 0) + (w & 0xFF000000u ? 1 : 0);
       }
       int total;
       int pos = block_excl_scan_256(cnt, wsum_c, total);
       if (threadIdx.x == 0) uni_tot = total;
-      for (int i = beg; i < end; ++i) {
-        const uint32_t m = dense ? dmask : (uint32_t)cmask[i];
-        if (m) { krow[pos] = (uint32_t)csa_row(i); kmask[pos] = (uint8_t)m; ++pos; }
+      for (int i = beg; i < end; i += 4) {
+        uint32_t w = dense ? 0x01010101u * dmask : mine[(i - beg) >> 2];
+        if (end - i < 4) w &= (1u << (8 * (end - i))) - 1u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t m = (w >> (8 * j)) & 0xFFu;
+          if (m) { krow[pos] = (uint32_t)csa_row(i + j); kmask[pos] = (uint8_t)m; ++pos; }
+        }
       }
       __syncthreads();
       n_uni = uni_tot;
@@ -235,12 +248,13 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
           box[bi] = make_int2(g, (int)run_row(g, k - k0[g]));
         }
       }
-      for (int k = threadIdx.x; k < kb; k += blockDim.x) {
+      // (gathered tiles: the compaction above has written the keys of the first run already)
+      for (int k = (runs_ok ? 0 : n_uni) + threadIdx.x; k < kb; k += blockDim.x) {
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
         const int i = k - k0[g];
         uint32_t m = 0;
         if (i < cnt[g]) {
-          if (g == 0) m = runs_ok ? (dense ? validbits : cmask[i]) : kmask[k];
+          if (g == 0) m = dense ? validbits : cmask[phys(i)];       // (contiguous-run tiles only: see the loop's start)
           else if (g == 1) m = validbits;
           else if (g == 2) {
             const int pos = c.page_table ? win_a + i : tm.L - 1 - ((tm.L - 1 - i) % s.window);
@@ -262,7 +276,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         }
         kmask[k] = (uint8_t)m;
         // gathered tiles: the key's row; the padding of a run repeats the run's first row (masked)
-        if (!runs_ok && (g > 0 || i >= cnt[0])) krow[k] = ((uint32_t)g << 30) | (uint32_t)(cnt[g] ? run_row(g, i < cnt[g] ? i : 0) : 0);
+        if (!runs_ok) krow[k] = ((uint32_t)g << 30) | (uint32_t)(cnt[g] ? run_row(g, i < cnt[g] ? i : 0) : 0);
       }
       if (threadIdx.x == 0) { *nkeys = kb; *mode = runs_ok ? 1 : 2; }
       return;
@@ -278,7 +292,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int share = ((n_csa + 7) / 8 + 31) & ~31;
     const int beg = min(n_csa, w * share), end = min(n_csa, beg + share);
-    auto mask_of = [&](int i) -> uint32_t { return i < end ? (dense ? validbits : (uint32_t)cmask[i]) : 0u; };
+    auto mask_of = [&](int i) -> uint32_t { return i < end ? (dense ? validbits : (uint32_t)cmask[phys(i)]) : 0u; };
     int cnt = 0;
     for (int i0 = beg; i0 < end; i0 += 32) cnt += mask_of(i0 + lane) != 0;
 #pragma unroll
@@ -715,7 +729,7 @@ __global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, cons
   }
 }
 
-// Merge of the paired kernel's tiles of more than two chunks: every chunk left its NORMALISED partial output (bf16) with
+// Merge of the paired kernel's multi-chunk tiles (launched with its general instantiation): every chunk left its NORMALISED partial output (bf16) with
 // the row's (reference max, sum); the row's output is the average of the partial outputs weighted by sum * 2^(max - row max).
 // grid (128-row tiles, sequences, groups of 8 rows): a warp merges one row, a lane owns 16 consecutive columns; the chunks
 // are accumulated in order, four chunks' loads in flight.
@@ -727,8 +741,8 @@ __global__ void __launch_bounds__(256) tc_combine_pair_kernel(const tsv_shape s,
   const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
   if ((mode != 1 && mode != 2) || nk <= 0) return;
   int nch, CL;
-  chunking_x(nk, nch, CL);
-  if (nch <= 2) return;                                          // the paired kernel wrote or merged these itself
+  chunking_x(nk, true, nch, CL);
+  if (nch <= 1) return;                                          // the paired kernel wrote the output itself
   const int rows_seq = s.D * s.H, row0 = rt * BM;
   const int lane = threadIdx.x & 31, row = blockIdx.z * 8 + (threadIdx.x >> 5);
   if (row >= BM || row0 + row >= rows_seq) return;
@@ -799,7 +813,7 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
 }
 
-static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) : 0; }   // node bits per entry, cleared by words
+static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) + 4 * 256 + 16 : 0; }   // node bits per entry, cleared by words (+ the padding words)
 // The pointer-gather kernel (and its merge kernel) serves every tile when the caches do not allow TMA (the caller gave no
 // row counts of the cache arrays); otherwise all tiles go to the paired kernel.
 static bool gather_kernel_needed(bool tma) { return !tma; }
@@ -848,10 +862,12 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep
   else tc_plan_kernel<false><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
   count_launch();
   if (p.tc_tma) {
-    const bool many = (p.tc_maxk + tc::NCX - 1) / tc::NCX > 2;   // some tile may have more than two chunks
-    const int r = launch_tva_tc_pair(s, p, prep, many || gathered, out, ws, status, st);
+    // general: some tile may have more than two chunks of the longest kind, or be gathered; then every multi-chunk tile
+    // leaves bf16 partial outputs for the merge kernel
+    const bool general = (p.tc_maxk + tc::NCX - 1) / tc::NCX > 2 || gathered;
+    const int r = launch_tva_tc_pair(s, p, prep, general, out, ws, status, st);
     if (r != TSV_OK) return r;
-    if (many) {
+    if (general && p.tc_chmax > 1) {
       tc_combine_pair_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);
       count_launch();
     }

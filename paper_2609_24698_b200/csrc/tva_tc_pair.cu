@@ -163,7 +163,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     return;
   }
   int nch, CL;
-  chunking_x(nk, nch, CL);
+  chunking_x(nk, GENERAL, nch, CL);
   if (chunk >= nch) return;
   const int cbeg = chunk * CL, cend = min(nk, cbeg + CL);
 
@@ -547,10 +547,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         const uint32_t* r0 = ro + cg * 64;
         const uint32_t* r1 = ro + cg * 64 + 32;
         const int col = part * OW + hh * cw + c0;
-        const bool many = GENERAL && nch > 2;
+        const bool many = GENERAL && nch > 1;
         if ((nch == 1 && full_tile) || many) {
           // stage the 32 x 64 bf16 tile in the 128-byte swizzle pattern and store it with one TMA request: into the output,
-          // or (tiles of more than two chunks) into the chunk's tile of normalised partial outputs, which a merge kernel
+          // or (multi-chunk tiles, where a merge kernel follows) into the chunk's tile of normalised partial outputs, which a merge kernel
           // combines with the chunks' (max, sum)
           if (store_pending) {
             if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -608,10 +608,10 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
         reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_run, l_row);
     }
     if (store_pending && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    if (GENERAL ? nch == 2 : nch > 1) {
-      // Tiles of two chunks: each chunk leaves its unnormalised part of O with (max, sum) per row; the CTA that
-      // finishes a 128-row tile last merges the parts (fixed order, so the result does not depend on who was last).
-      // (More chunks: a merge kernel follows; one CTA would take too long over them.)
+    if (!GENERAL && nch > 1) {
+      // Tiles of two chunks where nothing longer can occur: each chunk leaves its unnormalised part of O with (max, sum)
+      // per row; the CTA that finishes a 128-row tile last merges the parts (fixed order, so the result does not depend
+      // on who was last).  (In general a merge kernel follows: one CTA would take too long over many chunks.)
       __threadfence();
       compute_sync();
       if (warp == 2 && lane == 0) {
@@ -733,10 +733,11 @@ int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c
     for (int k = 0; k < 3 && ok; ++k) ok = make_map(&ms.src[a][k], bases[a], rows[a], 32 << k);
     ok = ok && make_map(&ms.row[a], bases[a], rows[a], 1);
   }
-  // partial outputs: per (128-row tile, chunk) a slot of 128 x 512 fp32 (tiles of two chunks); tiles of more than two
-  // chunks store 128 x 512 bf16 at the start of the slot: as rows of 1 KiB the buffer has 2 x 128 rows per slot
-  if (p.tc_chmax > 2) ok = ok && make_map(&ms.part, ws + p.off_tpo, (int64_t)s.B * 2 * p.tc_nt * p.tc_chmax * 2 * tc::BM, 32);
-  else ms.part = ms.out;                                                       // (never used: no tile has more than two chunks)
+  // partial outputs: per (128-row tile, chunk) a slot of 128 x 512 fp32 (used so by the instantiation that merges inside
+  // the kernel); the general instantiation stores 128 x 512 bf16 at the start of the slot: as rows of 1 KiB the buffer
+  // has 2 x 128 rows per slot
+  if (p.tc_chmax > 1) ok = ok && make_map(&ms.part, ws + p.off_tpo, (int64_t)s.B * 2 * p.tc_nt * p.tc_chmax * 2 * tc::BM, 32);
+  else ms.part = ms.out;                                                       // (never used: no tile has more than one chunk)
   if (!ok) {
     fprintf(stderr, "tsv: cuTensorMapEncodeTiled failed\n");
     return TSV_ERR_CUDA;
