@@ -61,6 +61,10 @@ void launch_idx_score_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& 
                          int32_t* status, cudaStream_t st);
 int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
+// per-node top-k of short candidate lists with the benchmark's indexer shape (scores, ranks and selects in one CTA)
+bool topk_fused_applies(const tsv_shape& s, const TvaPlan& p);
+int launch_topk_fused(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st);
 // per-node top-k of long candidate lists by a thread-block cluster per node
 bool topk_long_applies(const tsv_shape& s, const TvaPlan& p);
 int launch_topk_long(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,

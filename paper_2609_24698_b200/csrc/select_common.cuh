@@ -34,9 +34,9 @@ __device__ __forceinline__ uint32_t order_key(float f) {       // larger float -
 // launch).  The counts follow from lengths, node counts and done flags alone (for tiles on the contiguous-run path they
 // are exact; for pointer-gather tiles an estimate: only the order depends on them), so the ranking is ready before the
 // plan kernel runs and each plan CTA can leave its record at its final position.
-__device__ __forceinline__ void rank_tiles(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
-                                           const tsv_scratch& sc, char* __restrict__ ws) {
-  __shared__ int32_t nk_est[2048];
+// nk_est: shared memory for 2048 ints.
+__device__ __forceinline__ void rank_tiles_in(int32_t* nk_est, const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
+                                              const tsv_scratch& sc, char* __restrict__ ws) {
   const int D = s.D, nt = pl.tc_nt, ntile = s.B * nt, npt = 256 / s.H;
   int32_t* pos = reinterpret_cast<int32_t*>(ws + pl.off_pos);
   if (ntile > 2048) { for (int i = threadIdx.x; i < ntile; i += blockDim.x) pos[i] = i; return; }
@@ -61,6 +61,11 @@ __device__ __forceinline__ void rank_tiles(const tsv_shape& s, const TvaPlan& pl
     for (int j = 0; j < ntile; ++j) { const int kj = nk_est[j]; rank += (kj > ki) || (kj == ki && j < i); }
     pos[i] = rank;
   }
+}
+__device__ __forceinline__ void rank_tiles(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
+                                           const tsv_scratch& sc, char* __restrict__ ws) {
+  __shared__ int32_t nk_est[2048];
+  rank_tiles_in(nk_est, s, pl, c, nd, sc, ws);
 }
 
 }  // namespace tsv

@@ -566,6 +566,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
     }
   }
   if (topk_long_applies(s, p)) return launch_topk_long(s, p, c, nd, sc, topk_idx, ws, status, st);
+  if (topk_fused_applies(s, p)) return launch_topk_fused(s, p, c, nd, sc, topk_idx, ws, status, st);
   dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
   const bool paged = c.page_table != nullptr;
   size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...

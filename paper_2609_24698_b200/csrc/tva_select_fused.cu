@@ -1,0 +1,267 @@
+// Per-node top-k for short candidate lists (at most kIdxFusedMax committed entries) with 128-wide bf16 indexer rows (the
+// benchmark's): one CTA per (sequence, node) that scores, ranks and selects.  Same result as topk_kernel (the exact k
+// largest scores, ties to the lower index, ascending output); built so that
+//   * nodes that do not rank (nearly all of them) are a short chain and ALL CTAs of the launch are resident at once
+//     (four CTAs per SM: 64 registers, shared memory sized by the host for it), and
+//   * a node that ranks -- its CTA is the critical path of the whole stage -- overlaps what it can: the first rows are
+//     requested as soon as the length is known, the scores come from warp-level tensor-core products (mma.sync: the
+//     rows of a round as A, the node's indexer queries as B) so that a round costs its copies only, the radix keys stay
+//     in registers, and the selected indices are written after ONE block scan.
+#include <mma.h>
+
+#include "select_common.cuh"
+
+namespace tsv {
+
+namespace fsel {
+
+constexpr int DI = 128;                       // indexer width (bf16: 256-byte rows)
+constexpr int KPT = 9;                        // candidates per thread: 9 x 256 >= kIdxFusedMax + TSV_MAX_D
+static_assert(kIdxFusedMax + TSV_MAX_D <= KPT * 256, "candidate lists must fit the in-register keys");
+
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+}  // namespace fsel
+
+// Dynamic shared memory: [4][128] bf16 queries (heads beyond HI zero) | scores [score_cap] fp32 | two buffers of `rows`
+// staged indexer rows of 256 bytes (16-byte pieces XOR-swizzled by the row, so that ldmatrix reads without conflicts).
+template <bool PAGED>
+__global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+                                                            const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
+                                                            int32_t* __restrict__ status, const int rows, const int score_cap) {
+  using namespace fsel;
+  extern __shared__ __align__(128) unsigned char dsm[];
+  __shared__ TreeMeta tm;
+  __shared__ TreeStage tstage;
+  __shared__ PathEntries pe;
+  __shared__ float extra[TSV_MAX_D];
+  __shared__ int hist[2][256];                         // radix histogram; the buffers alternate between passes
+  __shared__ int wsum[9];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_remaining;
+  __shared__ int64_t row0_sm;
+  bf16* iqs = reinterpret_cast<bf16*>(dsm);
+  float* ssm = reinterpret_cast<float*>(dsm + 4 * DI * 2);
+  unsigned char* stage = dsm + 4 * DI * 2 + (size_t)score_cap * 4;
+  const int t = threadIdx.x;
+  if (blockIdx.x == (unsigned)s.D) {                  // extra CTA column (tensor-core attention path): CTA (D, 0) ranks the attention tiles
+    if (blockIdx.y == 0) rank_tiles_in(reinterpret_cast<int32_t*>(stage), s, pl, c, nd, sc, ws);
+    return;
+  }
+  const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk, HI = s.HI;
+  int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
+  int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
+  int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
+  if (!PAGED && t == 64) row0_sm = c.csa_row0[b];     // (in flight together with the tree's loads)
+  coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  const bool live = !tm.status && n < tm.nn;
+  const int n_csa = tm.n_csa;
+  // A node ranks iff its committed entries plus the blocks closed at its strict ancestors exceed k; at most depth(n)
+  // ancestors can have closed one, so the rows are requested now where that bound allows ranking (the done flags
+  // arrive two memory latencies later).
+  const bool may_rank = live && n_csa + tm.depth[n] > k;
+  RowAddr ikr;
+  if (PAGED) ikr = csa_rows_of(c, s, b); else { ikr.pt = nullptr; ikr.per_page = 1; ikr.row0 = row0_sm; }
+  const char* ikb = reinterpret_cast<const char*>(c.csa_ik) + (size_t)ikr.row0 * (DI * 2);
+  const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+  const int nrd = (n_csa + rows - 1) / rows;
+  auto issue = [&](int rd) {                           // rows [rd * rows, ..) into buffer rd & 1; one copy group per call
+    const int base = rd * rows, nrow = min(rows, n_csa - base);
+    const uint32_t dst = stage_s + (uint32_t)(rd & 1) * (uint32_t)(rows * 256);
+    for (int idx = t; idx < nrow * 16; idx += 256) {
+      const int row = idx >> 4, c16 = idx & 15;
+      cp16(dst + row * 256 + ((c16 ^ (row & 7)) << 4), ikb + (size_t)(PAGED ? ikr.rel(base + row) : (int64_t)(base + row)) * 256 + c16 * 16);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  if (may_rank) issue(0);
+  if (t == 0) {
+    if (tm.status && n == 0) atomicOr(status + b, tm.status);
+    if (live) path_entries(pe, tm, s, n, sc.csa_done + (size_t)b * D, sc.hca_done + (size_t)b * D);
+  }
+  __syncthreads();
+  if (!live) {
+    for (int i = t; i < k; i += 256) { sel[i] = -1; if (usr) usr[i] = -1; }
+    if (t == 0) *selcnt = 0;
+    return;
+  }
+  const int n_cand = n_csa + pe.n_newc;
+  if (n_cand <= k) {                                   // everything is selected: no ranking
+    for (int i = t; i < k; i += 256) {
+      const int v = i < n_csa ? i : (i < n_cand ? pe.newc_blk[i - n_csa] : -1);
+      sel[i] = v; if (usr) usr[i] = v;
+    }
+    if (t == 0) *selcnt = n_cand;
+    if (may_rank) asm volatile("cp.async.wait_group 0;" ::: "memory");     // (requested in vain: the bound was not reached)
+    return;
+  }
+  // ---------------------------------------------------------------------------------------------- the node ranks
+  const int lane = t & 31, w = t >> 5;
+  if (may_rank && nrd > 1) issue(1); else asm volatile("cp.async.commit_group;" ::: "memory");
+  // queries (raw bf16) to shared memory, head weights of this lane's two C columns to registers
+  const bf16* iq = reinterpret_cast<const bf16*>(nd.iq) + ((size_t)b * D + n) * HI * DI;
+  if (t < 64) reinterpret_cast<uint4*>(iqs)[t] = t < HI * 16 ? __ldg(reinterpret_cast<const uint4*>(iq) + t) : make_uint4(0u, 0u, 0u, 0u);
+  const int g = lane >> 2, tq = lane & 3;
+  const float* iwp = nd.iw + ((size_t)b * D + n) * HI;
+  const float iw0 = 2 * tq < HI ? iwp[2 * tq] : 0.f, iw1 = 2 * tq + 1 < HI ? iwp[2 * tq + 1] : 0.f;
+  // scores of the in-tree entries on this node's path: warp w takes entries w, w + 8, ...
+  for (int i = w; i < pe.n_newc; i += 8) {
+    const bf16* ik = reinterpret_cast<const bf16*>(sc.new_csa_ik) + ((size_t)b * D + pe.newc[i]) * DI;
+    float tot = 0.f;
+    for (int h = 0; h < HI; ++h) {
+      float p = 0.f;
+      for (int x = lane; x < DI; x += 32) p = fmaf(to_f(iq[h * DI + x]), to_f(ik[x]), p);
+      p = warp_sum(p);
+      tot = fmaf(iwp[h], fmaxf(p, 0.f), tot);
+    }
+    if (lane == 0) extra[i] = tot;
+  }
+  hist[0][t] = 0;
+  if (t == 0) { sh_prefix = 0; sh_remaining = k; }
+  __syncthreads();
+  // B fragments of the eight k-steps: column g = head g (zero beyond HI), k = 16 ks + 2 tq (+ 8)
+  uint32_t bq[8][2];
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    bq[ks][0] = g < 4 ? *reinterpret_cast<const uint32_t*>(iqs + g * DI + ks * 16 + 2 * tq) : 0u;
+    bq[ks][1] = g < 4 ? *reinterpret_cast<const uint32_t*>(iqs + g * DI + ks * 16 + 2 * tq + 8) : 0u;
+  }
+  for (int rd = 0; rd < nrd; ++rd) {                   // uniform trip count: barriers and shuffles below
+    asm volatile("cp.async.wait_group 1;" ::: "memory");   // round rd has landed (this thread's copies)
+    __syncthreads();
+    const int base = rd * rows, nrow = min(rows, n_csa - base);
+    const uint32_t buf = stage_s + (uint32_t)(rd & 1) * (uint32_t)(rows * 256);
+    for (int r0 = 16 * w; r0 < nrow; r0 += 128) {       // a warp scores 16 rows per step
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const int row = r0 + (lane & 15);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        uint32_t a[4];
+        ldmatrix_x4(buf + row * 256 + (((ks * 2 + (lane >> 4)) ^ (row & 7)) << 4), a);
+        mma_bf16_16816(acc, a, bq[ks][0], bq[ks][1]);
+      }
+      // C: rows g and g + 8 of the step, columns (heads) 2 tq and 2 tq + 1
+      float lo = fmaf(iw1, fmaxf(acc[1], 0.f), iw0 * fmaxf(acc[0], 0.f)), hi = fmaf(iw1, fmaxf(acc[3], 0.f), iw0 * fmaxf(acc[2], 0.f));
+      lo += __shfl_xor_sync(0xffffffffu, lo, 1);
+      hi += __shfl_xor_sync(0xffffffffu, hi, 1);
+      if (tq == 0) {
+        if (r0 + g < nrow) ssm[base + r0 + g] = lo;
+        if (r0 + g + 8 < nrow) ssm[base + r0 + g + 8] = hi;
+      }
+    }
+    __syncthreads();                                   // the buffer is refilled; the scores are visible
+    if (rd + 2 < nrd) issue(rd + 2); else asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  // order-preserving keys of this thread's candidates [KPT t, KPT t + KPT)
+  uint32_t key[KPT];
+  const int i0 = KPT * t;
+#pragma unroll
+  for (int j = 0; j < KPT; ++j) {
+    const int i = i0 + j;
+    key[j] = i < n_cand ? order_key(i < n_csa ? ssm[i] : extra[i - n_csa]) : 0u;
+  }
+  const int nmine = min(KPT, max(0, n_cand - i0));
+  uint32_t mask = 0;
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    const uint32_t prefix = sh_prefix;
+    int* hcur = hist[pass & 1];
+    hist[(pass & 1) ^ 1][t] = 0;                       // for the next pass (last read before the previous pass's closing barrier)
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+      const bool in = j < nmine && (key[j] & mask) == prefix;
+      const uint32_t bin = in ? (key[j] >> shift) & 255u : 256u;
+      // the scores of one list share their high digits: when the whole warp hits one bin, one lane adds for all
+      int uniform;
+      __match_all_sync(0xffffffffu, bin, &uniform);
+      if (uniform) { if (in && lane == 0) atomicAdd(&hcur[bin], 32); }
+      else if (in) atomicAdd(&hcur[bin], 1);
+    }
+    __syncthreads();
+    if (t < 32) {                                      // warp 0 finds the bin holding the rem-th largest key: lane l owns bins 255-8l .. 248-8l
+      const int rem = sh_remaining;
+      int h[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { h[j] = hcur[255 - (lane * 8 + j)]; tot += h[j]; }
+      int incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+      const int excl = incl - tot;
+      if (excl < rem && incl >= rem) {
+        int cum = excl, bin = 255 - lane * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { if (cum + h[j] >= rem) { bin = 255 - (lane * 8 + j); break; } cum += h[j]; }
+        sh_prefix = prefix | ((uint32_t)bin << shift);
+        sh_remaining = rem - cum;
+      }
+    }
+    mask |= 0xFFu << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = sh_prefix;       // key of the k-th largest score
+  const int r_take = sh_remaining;      // how many of the scores equal to it are taken (lowest indices)
+  int mine = 0;                         // keys above (low half) and equal to (high half) the threshold
+#pragma unroll
+  for (int j = 0; j < KPT; ++j) mine += (int)(j < nmine && key[j] > thr) + ((int)(j < nmine && key[j] == thr) << 16);
+  int total;
+  const int before = block_excl_scan_256(mine, wsum, total);
+  int eq_run = before >> 16, pos = (before & 0xFFFF) + min(r_take, eq_run);   // of the equal keys before this thread, the first r_take are taken
+#pragma unroll
+  for (int j = 0; j < KPT; ++j) {
+    const bool v = j < nmine, eq = v && key[j] == thr;
+    if ((v && key[j] > thr) || (eq && eq_run < r_take)) {
+      const int i = i0 + j, val = i < n_csa ? i : pe.newc_blk[i - n_csa];
+      sel[pos] = val; if (usr) usr[pos] = val;
+      ++pos;
+    }
+    eq_run += eq;
+  }
+  if (t == 0) *selcnt = k;
+}
+
+// The kernel serves: bf16, 128-wide indexer rows, at most four indexer heads, lists the selection scores itself.
+bool topk_fused_applies(const tsv_shape& s, const TvaPlan& p) {
+  return p.need_scores && p.idx_fused && s.dtype == TSV_BF16 && s.di == fsel::DI && s.HI <= 4;
+}
+
+// Rows per staging buffer and dynamic shared memory: as many rows (<= 128, a multiple of 16) as let four CTAs share an SM.
+static void fused_smem(const TvaPlan& p, int& rows, int& score_cap, size_t& bytes) {
+  score_cap = p.score_ld;
+  const size_t fixed = 4 * fsel::DI * 2 + (size_t)score_cap * 4;
+  const size_t budget = 52 * 1024;                     // of 57 KiB per CTA at four per SM: static shared memory and the per-CTA reserve come on top
+  rows = 128;
+  while (rows > 16 && fixed + (size_t)2 * rows * 256 > budget) rows -= 16;
+  bytes = fixed + (size_t)2 * rows * 256;
+}
+
+int launch_topk_fused(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st) {
+  int rows, score_cap;
+  size_t bytes;
+  fused_smem(p, rows, score_cap, bytes);
+  const dim3 grid(s.D + (p.tc ? 1 : 0), s.B);           // + the column that ranks the attention tiles
+  if (c.page_table) {
+    TSV_PREP(topk_fused_kernel<true>);
+    if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    topk_fused_kernel<true><<<grid, 256, bytes, st>>>(s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
+  } else {
+    TSV_PREP(topk_fused_kernel<false>);
+    if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    topk_fused_kernel<false><<<grid, 256, bytes, st>>>(s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
+  }
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
+}
+
+}  // namespace tsv
