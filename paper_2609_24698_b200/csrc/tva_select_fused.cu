@@ -44,11 +44,10 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   __shared__ TreeStage tstage;
   __shared__ PathEntries pe;
   __shared__ float extra[TSV_MAX_D];
-  __shared__ int hist[2][256];                         // radix histogram; the buffers alternate between passes
+  __shared__ uint32_t hist[3][128];                    // radix histogram, two 16-bit bins per word (a list has < 65536 candidates); the buffers rotate between passes
   __shared__ int wsum[9];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_remaining;
   __shared__ int64_t row0_sm;
+  __shared__ uint8_t cdone_sm[TSV_MAX_D], hdone_sm[TSV_MAX_D];
   bf16* iqs = reinterpret_cast<bf16*>(dsm);
   float* ssm = reinterpret_cast<float*>(dsm + 4 * DI * 2);
   unsigned char* stage = dsm + 4 * DI * 2 + (size_t)score_cap * 4;
@@ -61,8 +60,20 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
-  if (!PAGED && t == 64) row0_sm = c.csa_row0[b];     // (in flight together with the tree's loads)
+  // Everything the CTA may need that depends on (b, n) alone is requested together with the tree's loads (one memory
+  // latency for all): the slab offset, the done flags, and -- used only if the node ranks -- its indexer queries and
+  // head weights.
+  if (!PAGED && t == 64) row0_sm = c.csa_row0[b];
+  if (t >= 96 && t < 96 + D) cdone_sm[t - 96] = sc.csa_done[(size_t)b * D + t - 96];
+  if (t >= 128 && t < 128 + D) hdone_sm[t - 128] = sc.hca_done[(size_t)b * D + t - 128];
+  const int lane = t & 31, w = t >> 5, g = lane >> 2, tq = lane & 3;
+  const bf16* iq = reinterpret_cast<const bf16*>(nd.iq) + ((size_t)b * D + n) * HI * DI;
+  const float* iwp = nd.iw + ((size_t)b * D + n) * HI;
+  uint4 qv = make_uint4(0u, 0u, 0u, 0u);
+  if (t < HI * 16) qv = __ldg(reinterpret_cast<const uint4*>(iq) + t);
+  const float iw0 = 2 * tq < HI ? __ldg(iwp + 2 * tq) : 0.f, iw1 = 2 * tq + 1 < HI ? __ldg(iwp + 2 * tq + 1) : 0.f;
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  if (t < 64) reinterpret_cast<uint4*>(iqs)[t] = qv;   // (read after the next barrier)
   const bool live = !tm.status && n < tm.nn;
   const int n_csa = tm.n_csa;
   // A node ranks iff its committed entries plus the blocks closed at its strict ancestors exceed k; at most depth(n)
@@ -86,7 +97,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   if (may_rank) issue(0);
   if (t == 0) {
     if (tm.status && n == 0) atomicOr(status + b, tm.status);
-    if (live) path_entries(pe, tm, s, n, sc.csa_done + (size_t)b * D, sc.hca_done + (size_t)b * D);
+    if (live) path_entries(pe, tm, s, n, cdone_sm, hdone_sm);
   }
   __syncthreads();
   if (!live) {
@@ -105,14 +116,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     return;
   }
   // ---------------------------------------------------------------------------------------------- the node ranks
-  const int lane = t & 31, w = t >> 5;
-  if (may_rank && nrd > 1) issue(1); else asm volatile("cp.async.commit_group;" ::: "memory");
-  // queries (raw bf16) to shared memory, head weights of this lane's two C columns to registers
-  const bf16* iq = reinterpret_cast<const bf16*>(nd.iq) + ((size_t)b * D + n) * HI * DI;
-  if (t < 64) reinterpret_cast<uint4*>(iqs)[t] = t < HI * 16 ? __ldg(reinterpret_cast<const uint4*>(iq) + t) : make_uint4(0u, 0u, 0u, 0u);
-  const int g = lane >> 2, tq = lane & 3;
-  const float* iwp = nd.iw + ((size_t)b * D + n) * HI;
-  const float iw0 = 2 * tq < HI ? iwp[2 * tq] : 0.f, iw1 = 2 * tq + 1 < HI ? iwp[2 * tq + 1] : 0.f;
+  if (nrd > 1) issue(1); else asm volatile("cp.async.commit_group;" ::: "memory");
   // scores of the in-tree entries on this node's path: warp w takes entries w, w + 8, ...
   for (int i = w; i < pe.n_newc; i += 8) {
     const bf16* ik = reinterpret_cast<const bf16*>(sc.new_csa_ik) + ((size_t)b * D + pe.newc[i]) * DI;
@@ -125,9 +129,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     }
     if (lane == 0) extra[i] = tot;
   }
-  hist[0][t] = 0;
-  if (t == 0) { sh_prefix = 0; sh_remaining = k; }
-  __syncthreads();
+  if (t < 128) hist[0][t] = 0;
   // B fragments of the eight k-steps: column g = head g (zero beyond HI), k = 16 ks + 2 tq (+ 8)
   uint32_t bq[8][2];
 #pragma unroll
@@ -135,20 +137,25 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     bq[ks][0] = g < 4 ? *reinterpret_cast<const uint32_t*>(iqs + g * DI + ks * 16 + 2 * tq) : 0u;
     bq[ks][1] = g < 4 ? *reinterpret_cast<const uint32_t*>(iqs + g * DI + ks * 16 + 2 * tq + 8) : 0u;
   }
+  // Rounds of `rows` rows in two buffers: the copies of the next round run under the products of the current one.
   for (int rd = 0; rd < nrd; ++rd) {                   // uniform trip count: barriers and shuffles below
     asm volatile("cp.async.wait_group 1;" ::: "memory");   // round rd has landed (this thread's copies)
     __syncthreads();
     const int base = rd * rows, nrow = min(rows, n_csa - base);
     const uint32_t buf = stage_s + (uint32_t)(rd & 1) * (uint32_t)(rows * 256);
     for (int r0 = 16 * w; r0 < nrow; r0 += 128) {       // a warp scores 16 rows per step
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      float acc[4] = {0.f, 0.f, 0.f, 0.f}, acd[4] = {0.f, 0.f, 0.f, 0.f};     // two chains: even and odd k-steps
       const int row = r0 + (lane & 15);
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        uint32_t a[4];
+      for (int ks = 0; ks < 8; ks += 2) {
+        uint32_t a[4], a2[4];
         ldmatrix_x4(buf + row * 256 + (((ks * 2 + (lane >> 4)) ^ (row & 7)) << 4), a);
+        ldmatrix_x4(buf + row * 256 + (((ks * 2 + 2 + (lane >> 4)) ^ (row & 7)) << 4), a2);
         mma_bf16_16816(acc, a, bq[ks][0], bq[ks][1]);
+        mma_bf16_16816(acd, a2, bq[ks + 1][0], bq[ks + 1][1]);
       }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) acc[x] += acd[x];
       // C: rows g and g + 8 of the step, columns (heads) 2 tq and 2 tq + 1
       float lo = fmaf(iw1, fmaxf(acc[1], 0.f), iw0 * fmaxf(acc[0], 0.f)), hi = fmaf(iw1, fmaxf(acc[3], 0.f), iw0 * fmaxf(acc[2], 0.f));
       lo += __shfl_xor_sync(0xffffffffu, lo, 1);
@@ -162,70 +169,91 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     if (rd + 2 < nrd) issue(rd + 2); else asm volatile("cp.async.commit_group;" ::: "memory");
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
-  // order-preserving keys of this thread's candidates [KPT t, KPT t + KPT)
+  if (nrd == 0) __syncthreads();                       // (the in-tree entries' scores, the cleared histogram)
+  // order-preserving keys: candidate t + 256 j is key j of thread t (all warps take part in every pass)
   uint32_t key[KPT];
-  const int i0 = KPT * t;
+  const int nj = (n_cand + 255) >> 8;
 #pragma unroll
   for (int j = 0; j < KPT; ++j) {
-    const int i = i0 + j;
-    key[j] = i < n_cand ? order_key(i < n_csa ? ssm[i] : extra[i - n_csa]) : 0u;
+    const int i = t + 256 * j;
+    key[j] = (j < nj && i < n_cand) ? order_key(i < n_csa ? ssm[i] : extra[i - n_csa]) : 0u;
   }
-  const int nmine = min(KPT, max(0, n_cand - i0));
-  uint32_t mask = 0;
+  // Four radix passes of 8 bits.  ONE barrier per pass: after it the histogram is complete and EVERY warp finds the bin of
+  // the rem-th largest key for itself (lane l owns bins 255 - 8 l .. 248 - 8 l); the histogram buffers rotate, the one for
+  // the next pass is cleared at the start of a pass (its last readers passed the previous pass's barrier before).
+  uint32_t mask = 0, prefix = 0;
+  int rem = k;
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    const uint32_t prefix = sh_prefix;
-    int* hcur = hist[pass & 1];
-    hist[(pass & 1) ^ 1][t] = 0;                       // for the next pass (last read before the previous pass's closing barrier)
+    uint32_t* hcur = hist[pass % 3];
+    if (t < 128) hist[(pass + 1) % 3][t] = 0;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-      const bool in = j < nmine && (key[j] & mask) == prefix;
-      const uint32_t bin = in ? (key[j] >> shift) & 255u : 256u;
-      // the scores of one list share their high digits: when the whole warp hits one bin, one lane adds for all
-      int uniform;
-      __match_all_sync(0xffffffffu, bin, &uniform);
-      if (uniform) { if (in && lane == 0) atomicAdd(&hcur[bin], 32); }
-      else if (in) atomicAdd(&hcur[bin], 1);
-    }
-    __syncthreads();
-    if (t < 32) {                                      // warp 0 finds the bin holding the rem-th largest key: lane l owns bins 255-8l .. 248-8l
-      const int rem = sh_remaining;
-      int h[8], tot = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { h[j] = hcur[255 - (lane * 8 + j)]; tot += h[j]; }
-      int incl = tot;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
-      const int excl = incl - tot;
-      if (excl < rem && incl >= rem) {
-        int cum = excl, bin = 255 - lane * 8;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { if (cum + h[j] >= rem) { bin = 255 - (lane * 8 + j); break; } cum += h[j]; }
-        sh_prefix = prefix | ((uint32_t)bin << shift);
-        sh_remaining = rem - cum;
+      if (j < nj) {
+        const bool in = t + 256 * j < n_cand && (key[j] & mask) == prefix;
+        const uint32_t bin = in ? (key[j] >> shift) & 255u : 256u;
+        // the scores of one list share their high digits: when the whole warp hits one bin, one lane adds for all
+        int uniform;
+        __match_all_sync(0xffffffffu, bin, &uniform);
+        if (uniform) { if (in && lane == 0) atomicAdd(&hcur[bin >> 1], 32u << (16 * (bin & 1))); }
+        else if (in) atomicAdd(&hcur[bin >> 1], 1u << (16 * (bin & 1)));
       }
     }
-    mask |= 0xFFu << shift;
     __syncthreads();
-  }
-  const uint32_t thr = sh_prefix;       // key of the k-th largest score
-  const int r_take = sh_remaining;      // how many of the scores equal to it are taken (lowest indices)
-  int mine = 0;                         // keys above (low half) and equal to (high half) the threshold
+    int h[8], tot = 0;
 #pragma unroll
-  for (int j = 0; j < KPT; ++j) mine += (int)(j < nmine && key[j] > thr) + ((int)(j < nmine && key[j] == thr) << 16);
-  int total;
-  const int before = block_excl_scan_256(mine, wsum, total);
-  int eq_run = before >> 16, pos = (before & 0xFFFF) + min(r_take, eq_run);   // of the equal keys before this thread, the first r_take are taken
+    for (int j = 0; j < 8; ++j) { const int bj = 255 - (lane * 8 + j); h[j] = (hcur[bj >> 1] >> (16 * (bj & 1))) & 0xFFFF; tot += h[j]; }
+    int incl = tot;
 #pragma unroll
-  for (int j = 0; j < KPT; ++j) {
-    const bool v = j < nmine, eq = v && key[j] == thr;
-    if ((v && key[j] > thr) || (eq && eq_run < r_take)) {
-      const int i = i0 + j, val = i < n_csa ? i : pe.newc_blk[i - n_csa];
-      sel[pos] = val; if (usr) usr[pos] = val;
-      ++pos;
+    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+    const int excl = incl - tot;
+    const bool owner = excl < rem && incl >= rem;      // exactly one lane
+    int cum = excl, bin = 255 - lane * 8;
+    if (owner) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { if (cum + h[j] >= rem) { bin = 255 - (lane * 8 + j); break; } cum += h[j]; }
     }
-    eq_run += eq;
+    const int src = __ffs(__ballot_sync(0xffffffffu, owner)) - 1;
+    prefix |= (uint32_t)__shfl_sync(0xffffffffu, bin, src) << shift;
+    rem -= __shfl_sync(0xffffffffu, cum, src);
+    mask |= 0xFFu << shift;
+  }
+  const uint32_t thr = prefix;          // key of the k-th largest score
+  const int r_take = rem;               // how many of the scores equal to it are taken (lowest indices)
+  // Ordered compaction: warp w owns the candidates [w * share, (w + 1) * share) (whole rows of 32; their keys are derived
+  // again from the scores), counts its keys above and equal to the threshold with ballots, the warps exchange their
+  // counts once, then each writes its selected indices row by row.
+  const int share = ((n_cand + 7) / 8 + 31) & ~31, beg = w * share;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t ckey[(KPT * 256 / 8 + 31) / 32 + 1];        // rows of the warp's share: at most 10
+  constexpr int CR = (KPT * 256 / 8 + 31) / 32 + 1;
+  int cgt = 0, ceq = 0;
+#pragma unroll
+  for (int r = 0; r < CR; ++r) {
+    const int i = beg + 32 * r + lane;
+    const bool v = 32 * r < share && i < n_cand;
+    ckey[r] = v ? order_key(i < n_csa ? ssm[i] : extra[i - n_csa]) : 0u;
+    cgt += __popc(__ballot_sync(0xffffffffu, v && ckey[r] > thr));
+    ceq += __popc(__ballot_sync(0xffffffffu, v && ckey[r] == thr));
+  }
+  if (lane == 0) wsum[w] = cgt | (ceq << 16);
+  __syncthreads();
+  int eq_base = 0, out_base = 0;
+  for (int x = 0; x < w; ++x) { const int v = wsum[x]; out_base += v & 0xFFFF; eq_base += v >> 16; }
+  out_base += min(r_take, eq_base);                    // of the equal keys before this share, the first r_take are taken
+#pragma unroll
+  for (int r = 0; r < CR; ++r) {
+    const int i = beg + 32 * r + lane;
+    const bool v = 32 * r < share && i < n_cand, eq = v && ckey[r] == thr;
+    const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
+    const bool take = (v && ckey[r] > thr) || (eq && eq_base + __popc(eqm & lt) < r_take);
+    const uint32_t tkm = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      const int pos = out_base + __popc(tkm & lt), val = i < n_csa ? i : pe.newc_blk[i - n_csa];
+      sel[pos] = val; if (usr) usr[pos] = val;
+    }
+    eq_base += __popc(eqm); out_base += __popc(tkm);
   }
   if (t == 0) *selcnt = k;
 }
@@ -235,7 +263,8 @@ bool topk_fused_applies(const tsv_shape& s, const TvaPlan& p) {
   return p.need_scores && p.idx_fused && s.dtype == TSV_BF16 && s.di == fsel::DI && s.HI <= 4;
 }
 
-// Rows per staging buffer and dynamic shared memory: as many rows (<= 128, a multiple of 16) as let four CTAs share an SM.
+// Rows per staging buffer (two buffers) and dynamic shared memory: as many rows (<= 128, a multiple of 16) as let four
+// CTAs share an SM.
 static void fused_smem(const TvaPlan& p, int& rows, int& score_cap, size_t& bytes) {
   score_cap = p.score_ld;
   const size_t fixed = 4 * fsel::DI * 2 + (size_t)score_cap * 4;
