@@ -47,6 +47,10 @@ struct TvaPlan {
   int32_t tc, tc_nt, tc_maxk, tc_chmax;
   int32_t tc_tma, tc_misc_rows;      // contiguous-run tiles go through TMA; rows of the per-sequence packed buffer
   size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt, off_pos;
+  // selection as a byte per candidate (1 = selected), one row of mask_ld bytes per node, written for the nodes that rank:
+  // the tile plan combines the rows of a tile's nodes into its per-key node masks
+  size_t off_selmask;
+  int32_t mask_ld;
 };
 bool make_tva_plan(const tsv_shape& s, TvaPlan& p);
 

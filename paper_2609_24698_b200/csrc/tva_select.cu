@@ -454,6 +454,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   }
   const uint32_t thr = sh_prefix;       // key of the k-th largest score
   const int r = sh_remaining;           // how many of the scores equal to it are taken (lowest indices)
+  uint8_t* selmask = pl.tc ? reinterpret_cast<uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n) * pl.mask_ld : nullptr;   // the selection as a byte per candidate (for the tile plan)
   if (!in_regs) {
     // Long lists: warp w owns a contiguous share of the candidates (whole 128-candidate steps: a lane holds four
     // consecutive candidates of a step) and walks it twice, eight steps per round: first counting the
@@ -502,12 +503,14 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
 #pragma unroll
         for (int j = 0; j < 4; ++j) { pos += __popc(tkm[j] & lt); ntk += __popc(tkm[j]); }
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < 4; ++j) {
+          if (selmask && (full || ib + j < end)) selmask[ib + j] = (uint8_t)take[j];
           if (take[j]) {
             const int i = ib + j, v = i < n_csa ? i : pe.newc_blk[i - n_csa];
             sel[pos] = v; if (usr) usr[pos] = v;
             ++pos;
           }
+        }
         eq_base += neq; out_base += ntk;
       }
     });
@@ -529,6 +532,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
     const int eq_rank = eq_base + block_excl_scan_256(eq, wsum, tot_eq);
     const int take = gt || (eq && eq_rank < r);
     const int pos = out_base + block_excl_scan_256(take, wsum, tot_take);
+    if (selmask && i < n_cand) selmask[i] = (uint8_t)take;
     if (take) {
       const int v = i < n_csa ? i : pe.newc_blk[i - n_csa];
       sel[pos] = v; if (usr) usr[pos] = v;

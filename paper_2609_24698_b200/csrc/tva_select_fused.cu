@@ -224,6 +224,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   // Ordered compaction: warp w owns the candidates [w * share, (w + 1) * share) (whole rows of 32; their keys are derived
   // again from the scores), counts its keys above and equal to the threshold with ballots, the warps exchange their
   // counts once, then each writes its selected indices row by row.
+  uint8_t* selmask = pl.tc ? reinterpret_cast<uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n) * pl.mask_ld : nullptr;   // (for the tile plan)
   const int share = ((n_cand + 7) / 8 + 31) & ~31, beg = w * share;
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t ckey[(KPT * 256 / 8 + 31) / 32 + 1];        // rows of the warp's share: at most 10
@@ -249,6 +250,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
     const bool take = (v && ckey[r] > thr) || (eq && eq_base + __popc(eqm & lt) < r_take);
     const uint32_t tkm = __ballot_sync(0xffffffffu, take);
+    if (v && selmask) selmask[i] = (uint8_t)take;
     if (take) {
       const int pos = out_base + __popc(tkm & lt), val = i < n_csa ? i : pe.newc_blk[i - n_csa];
       sel[pos] = val; if (usr) usr[pos] = val;

@@ -189,6 +189,7 @@ __global__ void __launch_bounds__(lsel::THREADS) topk_long_kernel(const tsv_shap
   cluster_sync();                                                 // the counts of the CTAs before this one are there
   int eq_run = (before >> 16) + before_sm[1], pos = (before & 0xFFFF) + before_sm[0];
   pos += min(r_take, eq_run);             // of the equal keys before this thread, the first r_take are taken
+  uint32_t mbytes[KEYS / 4] = {0u, 0u, 0u, 0u};             // the selection as a byte per candidate, for the tile plan
 #pragma unroll
   for (int j = 0; j < KEYS; ++j) {
     const bool v = (valid >> j) & 1u, eq = v && key[j] == thr;
@@ -196,9 +197,12 @@ __global__ void __launch_bounds__(lsel::THREADS) topk_long_kernel(const tsv_shap
       const int i = i0 + j, val = i < n_csa ? i : pe.newc_blk[i - n_csa];
       sel[pos] = val; if (usr) usr[pos] = val;
       ++pos;
+      mbytes[j >> 2] |= 1u << (8 * (j & 3));
     }
     eq_run += eq;
   }
+  if (owner && pl.tc)                                          // (i0 is a multiple of 16 and so is the row length)
+    *reinterpret_cast<uint4*>(ws + pl.off_selmask + ((size_t)b * D + n) * pl.mask_ld + i0) = make_uint4(mbytes[0], mbytes[1], mbytes[2], mbytes[3]);
   if (gt == 0) *selcnt = k;
 }
 

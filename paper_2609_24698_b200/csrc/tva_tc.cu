@@ -41,7 +41,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   uint64_t* kptr = reinterpret_cast<uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
-  const int32_t* sel = reinterpret_cast<const int32_t*>(ws + pl.off_sel) + (size_t)b * D * s.topk;
   // the done flags and the cache row offsets are fetched together with the tree scalars (one memory latency for all)
   __shared__ uint8_t cdone[TSV_MAX_D], hdone[TSV_MAX_D];
   __shared__ int64_t row0_sm[2];
@@ -131,8 +130,9 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   const int n_csa = tm.n_csa;
   const size_t rowb = (size_t)s.d * 2;
   // Ranked nodes: node bits per committed CSA entry (cmask) and, per node, which blocks closed inside the tree are in
-  // its selection (bit = block index - n_csa).  One pass over the selections of all the tile's nodes: the loads of a
-  // batch are issued together (the tile CTA of a ranked sequence is on the critical path of the whole stage).
+  // its selection (bit = block index - n_csa).  The selection kernel left, for every node that ranks, a byte per
+  // candidate (1 = selected): the rows of the tile's nodes are combined sixteen entries at a time (coalesced 16-byte
+  // loads; the tile CTA of a ranked sequence is on the critical path of the whole stage).
   //
   // Where gathered tiles may occur the array is padded by one word after every `per` entries (per: the power of two that
   // spreads the entries over the CTA's threads): the compaction below gives a thread `per` consecutive entries, and
@@ -142,34 +142,41 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   if (GENERAL) while ((256 << psh) < n_csa) ++psh;
   auto phys = [&](int i) { return GENERAL ? i + ((i >> psh) << 2) : i; };
   if (!dense) {
+    uint32_t allbits = 0, rankbits = 0;                // nodes that take every committed entry / nodes that rank
+    for (int nl = 0; nl < nvalid; ++nl) { if (n_cand[nl] <= s.topk) allbits |= 1u << nl; else rankbits |= 1u << nl; }
+    const uint8_t* mrow = reinterpret_cast<const uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n0) * pl.mask_ld;
+    if (threadIdx.x < 8) {
+      // in-tree entries: candidate n_csa + o of a node is the block closed at the o-th of its strict ancestors that closed one
+      uint32_t bits = 0;
+      const int nl = threadIdx.x;
+      if (nl < nvalid && ((rankbits >> nl) & 1u)) {
+        int o = 0;
+        for (int a = 0; a < n0 + nl; ++a) {
+          if (!((tm.anc[n0 + nl] >> a) & 1u) || !cdone[a]) continue;
+          const int dblk = (tm.L + tm.depth[a]) / s.m_csa - n_csa;
+          if (mrow[(size_t)nl * pl.mask_ld + n_csa + o] && dblk >= 0 && dblk < 32) bits |= 1u << dblk;
+          ++o;
+        }
+      }
+      newc_bits[nl] = bits;
+    }
     uint32_t* cm32 = reinterpret_cast<uint32_t*>(cmask);
-    for (int i = threadIdx.x; i < (phys(n_csa) + 3) / 4; i += blockDim.x) cm32[i] = 0;
-    if (threadIdx.x < 8) newc_bits[threadIdx.x] = 0;
-    __syncthreads();
-    uint32_t allbits = 0;                              // nodes that take every committed entry
-    for (int nl = 0; nl < nvalid; ++nl) if (n_cand[nl] <= s.topk) allbits |= 1u << nl;
-    const int total = nvalid * s.topk;
-    for (int x0 = 0; x0 < total; x0 += 8 * blockDim.x) {
-      int idx[8], nls[8];
+    const uint32_t all4 = 0x01010101u * allbits;
+#pragma unroll 2
+    for (int i = 16 * threadIdx.x; i < n_csa; i += 16 * blockDim.x) {
+      uint32_t acc[4] = {all4, all4, all4, all4};
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int x = x0 + u * blockDim.x + threadIdx.x;
-        const int nl = x < total ? x / s.topk : 0, jj = x - nl * s.topk;
-        nls[u] = nl;
-        idx[u] = (x < total && n_cand[nl] > s.topk) ? __ldcg(sel + (size_t)(n0 + nl) * s.topk + jj) : -1;   // unused slots hold -1
+      for (int nl = 0; nl < 8; ++nl) {
+        if ((rankbits >> nl) & 1u) {
+          const uint4 v = __ldcg(reinterpret_cast<const uint4*>(mrow + (size_t)nl * pl.mask_ld + i));
+          acc[0] |= (v.x & 0x01010101u) << nl; acc[1] |= (v.y & 0x01010101u) << nl;
+          acc[2] |= (v.z & 0x01010101u) << nl; acc[3] |= (v.w & 0x01010101u) << nl;
+        }
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (idx[u] < 0) continue;
-        if (idx[u] < n_csa) atomicOr(cm32 + (phys(idx[u]) >> 2), (1u << nls[u]) << (8 * (idx[u] & 3)));
-        else if (idx[u] - n_csa < 32) atomicOr(&newc_bits[nls[u]], 1u << (idx[u] - n_csa));
-      }
+      for (int q = 0; q < 4; ++q) cm32[phys(i + 4 * q) >> 2] = acc[q];      // (bytes past n_csa are never read)
     }
     __syncthreads();
-    if (allbits) {
-      for (int i = threadIdx.x; i < n_csa; i += blockDim.x) cmask[phys(i)] |= (uint8_t)allbits;
-      __syncthreads();
-    }
   }
   // is the entry closed at node a (a strict ancestor of node n0 + nl) among that node's selected CSA entries?
   auto newc_selected = [&](int nl, int a) {
