@@ -31,13 +31,14 @@ import numpy as np  # noqa: E402
 # attention stage with the bytes of ONE of its launches (one layer), and, where captured, the sum over all kernels of one
 # verify cycle.  The captures are summarised under profiles/; workloads without a capture report null.
 NCU_DRAM = {
-    "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 70_355_456, "cycle_bytes": None},   # 65.62 MB read + 4.73 MB written
-    # cfg5: tc_attn_kernel 62.28 MB read + 19.15 MB written; all kernels of one cycle 191.7 MB (cold cache per kernel)
-    "cfg5": {"kernel": "tc_attn_kernel", "launch_bytes": 81_427_712, "cycle_bytes": 191_703_808},
+    "cfg4": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 66_239_168, "cycle_bytes": None},   # 65.48 MB read + 0.76 MB written
+    # cfg5: tc_attn_pair_kernel 61.11 MB read + 1.70 MB written; all kernels of one cycle 138.1 MB (cold cache per kernel)
+    "cfg5": {"kernel": "tc_attn_pair_kernel", "launch_bytes": 62_808_320, "cycle_bytes": 138_081_792},
 }
-ATTN_KERNEL = {"cfg1": "attn_simt_kernel (fp32 CUDA-core path)", "cfg2": "tc_attn_pair_kernel", "cfg2_chain": "tc_attn_pair_kernel",
-               "cfg3": "tc_attn_pair_kernel + tc_attn_kernel (pointer gather) + tc_combine_kernel", "cfg4": "tc_attn_pair_kernel",
-               "cfg5": "tc_attn_kernel (pointer gather) + tc_combine_kernel"}
+ATTN_KERNEL = {"cfg1": "attn_simt_kernel (fp32 CUDA-core path)", "cfg2": "tc_attn_pair_kernel + tc_combine_pair_kernel",
+               "cfg2_chain": "tc_attn_pair_kernel + tc_combine_pair_kernel",
+               "cfg3": "tc_attn_pair_kernel (contiguous-run and gathered tiles) + tc_combine_pair_kernel", "cfg4": "tc_attn_pair_kernel",
+               "cfg5": "tc_attn_pair_kernel (gathered tiles) + tc_combine_pair_kernel"}
 
 
 def peaks():

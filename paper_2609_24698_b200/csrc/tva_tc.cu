@@ -811,7 +811,9 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   const int64_t br = kBoxRows;
   p.tc_misc_rows = (int32_t)((kHcaMiscMax + 3 * s.D + br - 1) / br * br);
   // (+ one box: in a paged pool the window run starts on a 32-aligned position and may be a box longer than the window)
-  const int64_t runs = (p.cand_cap + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
+  // (a tile takes the whole committed CSA run only while that is at most twice the selection size)
+  const int64_t run_csa = p.cand_cap < 2 * (int64_t)s.topk ? p.cand_cap : 2 * (int64_t)s.topk;
+  const int64_t runs = (run_csa + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
   if (runs > mk) mk = runs;
   // gathered tiles: the union of the nodes' selections, HCA entries, window and packed rows as four runs padded to boxes
   const int64_t gath = (uni + br - 1) / br * br + (s.max_L / s.m_hca + br - 1) / br * br + (s.window + br - 1) / br * br + br + p.tc_misc_rows;
