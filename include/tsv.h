@@ -120,8 +120,10 @@ typedef struct tsv_cache {
   float *csa_acc_ik;          /* [B][di] weighted sum of indexer-key vectors                */
   float *hca_mx, *hca_s;      /* [B] open HCA block                                         */
   float *hca_acc_kv;          /* [B][d]                                                     */
-  int64_t csa_rows;           /* HOST value: rows allocated in csa_kv / csa_ik (all slabs)  */
-  int64_t hca_rows;           /* HOST value: rows allocated in hca_kv                       */
+  int64_t csa_rows;           /* HOST value: rows allocated in csa_kv / csa_ik (all slabs); the tensor-core attention
+                               * path builds its tensor maps from it: with 0 ("unknown") every shape runs on the
+                               * CUDA-core path                                               */
+  int64_t hca_rows;           /* HOST value: rows allocated in hca_kv (0: a layer without HCA entries) */
   /* Paged pool (Section "Temporary Branch States and Compressed-State Handling": a page-based pool seen as one logical
    * layer and several physical layers that share page-level pointers).  With page_table non-NULL the CSA and HCA entries
    * of a sequence do not sit in one slab each: logical page lp holds the entries of tokens [lp, lp + 1) * page_tokens, and

@@ -56,14 +56,14 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   p.off_po = off;     if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * s.d * sizeof(float));
   p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
   p.tc = tva_tc_eligible(s);
-  p.tc_nt = p.tc_maxk = p.tc_chmax = p.tc_tma = p.tc_misc_rows = 0;
-  p.off_kptr = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = p.off_order = p.off_tcnt = p.off_pos = off;
+  p.tc_nt = p.tc_maxk = p.tc_chmax = p.tc_misc_rows = 0;
+  p.off_krow = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = p.off_order = p.off_tcnt = p.off_pos = off;
   p.off_selmask = off;
   p.mask_ld = (p.cand_cap + 15) & ~15;
   if (p.tc) {
     tva_tc_plan_sizes(s, p);
     const size_t tiles = (size_t)s.B * p.tc_nt;
-    p.off_kptr = off;  off = up256(off + tiles * p.tc_maxk * sizeof(uint64_t));
+    p.off_krow = off;  off = up256(off + tiles * p.tc_maxk * sizeof(uint32_t));   // row codes of gathered tiles
     p.off_kmask = off; off = up256(off + tiles * p.tc_maxk);
     p.off_nkeys = off; off = up256(off + tiles * sizeof(int32_t));
     p.off_tpo = off;   if (p.tc_chmax > 1) off = up256(off + 2 * tiles * p.tc_chmax * 128 * s.d * sizeof(float));
@@ -117,10 +117,12 @@ static int check_scratch(const tsv_scratch* s) {
 
 // tree_verify_attn after validation.  All host work that can fail (tensor maps, kernel attributes) comes before the
 // first launch, so a negative return means that nothing was enqueued by this call, unless a launch itself fails.
-static int tva_stages(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, void* out,
+static int tva_stages(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc, void* out,
                       int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st, int stages) {
   int r;
   TvaTcPrep prep;
+  TvaPlan p = p_in;
+  if (p.tc && !tva_tc_pair_usable(c)) p.tc = 0;       // no row counts for the tensor maps: the CUDA-core path (same workspace)
   if (p.tc && (stages & 2) && (r = prepare_tva_tc(s, p, c, nd, out, ws, prep))) return r;
   if ((stages & 1) && (r = launch_tva_select(s, p, c, nd, sc, topk_idx, ws, status, st))) return r;
   if (!(stages & 2)) return TSV_OK;

@@ -45,8 +45,8 @@ struct TvaPlan {
   size_t off_selcnt, off_sel, off_scores, off_po, off_pml, total;
   // tensor-core path (bf16, d = 512): row tiles per sequence, key-list capacity per tile, max chunks per tile
   int32_t tc, tc_nt, tc_maxk, tc_chmax;
-  int32_t tc_tma, tc_misc_rows;      // contiguous-run tiles go through TMA; rows of the per-sequence packed buffer
-  size_t off_kptr, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt, off_pos;
+  int32_t tc_misc_rows;              // rows of the per-sequence packed buffer
+  size_t off_krow, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt, off_pos;
   // selection as a byte per candidate (1 = selected), one row of mask_ld bytes per node, written for the nodes that rank:
   // the tile plan combines the rows of a tile's nodes into its per-key node masks
   size_t off_selmask;
@@ -80,12 +80,13 @@ constexpr int kIdxFusedMax = 2048;   // candidate capacity up to which topk_kern
 constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs are padded to a multiple of it
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
+// the tensor-core path needs the caller's row count of the CSA arrays (tensor maps) and the driver's map encoder; without
+// them a shape it would take runs on the CUDA-core path
 bool tva_tc_pair_usable(const tsv_cache& c);
 // Host-side preparation of the tensor-core attention path: everything that can fail on the host (tensor maps, kernel
 // attributes) is done here, before any kernel of the call is enqueued.
 struct TvaTcPrep {
   alignas(64) unsigned char maps[19 * 128];   // the paired kernel's tensor maps (a CUtensorMap is 128 bytes)
-  int32_t tma;                                // the contiguous-run path is usable for these caches
 };
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
 // general: gathered tiles or tiles of more than two chunks may occur (else the instantiation without that code runs)

@@ -10,14 +10,7 @@ namespace tc {
 constexpr int DH = 512;             // head dim handled by this path
 constexpr int BM = 128;             // rows per CTA
 constexpr int PR = 256;             // rows per plan tile: two row tiles (one CTA pair) share one key list
-constexpr int NC = 512;             // max keys per chunk (S columns in TMEM)
-constexpr int SLOT = 32768;
-constexpr int NS = 7;               // ring slots
-constexpr int LOOK = NS - 3;        // stages loaded ahead of the MMA issue
-constexpr int THREADS = 256;
-constexpr int kHcaMiscMaxTc = 32;
-constexpr int SMALL = 2048;         // barriers, masks, softmax exchange
-constexpr int SMEM_BYTES = SMALL + NS * SLOT + 1024;
+constexpr int NC = 512;             // keys per chunk of a list that is cut into several
 constexpr uint32_t WAIT_LIMIT = 1u << 14;   // polls before a wait gives up (then no later wait of the thread is attempted)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -34,10 +27,6 @@ __device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -102,24 +91,6 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-struct Small {                       // first SMALL bytes of dynamic shared memory
-  uint64_t slot_free[NS];
-  uint64_t acc_bar;
-  uint32_t tmem_base;
-  uint32_t pad;
-  uint8_t kmask[NC];
-  float xch[2][BM];                   // row max, later row sum, exchanged between the two column halves
-};
-static_assert(sizeof(Small) <= SMALL, "small region overflow");
-
-// chunking of a tile's key list: nch chunks of CL keys (CL a multiple of 128, <= NC)
-__device__ __host__ __forceinline__ void chunking(int nk, int& nch, int& CL) {
-  nch = (nk + NC - 1) / NC;
-  if (nch < 1) nch = 1;
-  CL = (((nk + nch - 1) / nch) + 127) / 128 * 128;
-  if (CL < 128) CL = 128;
 }
 
 constexpr int NCX = 768;             // max keys per chunk of the TMA kernel: P (bf16) takes 384 TMEM columns, an O quarter 128

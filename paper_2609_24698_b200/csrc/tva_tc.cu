@@ -1,25 +1,19 @@
-// tree_verify_attn on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 storage, d = 512: the tile plan, the
-// pointer-gather attention kernel and the merge of multi-chunk tiles.  (The main attention kernel, for key lists made of
-// contiguous runs, is in tva_tc_pair.cu.)
+// tree_verify_attn on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 storage, d = 512: the tile plan and the
+// merge of multi-chunk tiles.  (The attention kernel itself is in tva_tc_pair.cu.)
 //
 // Rows are grouped in plan tiles of 256 query rows = 256/H consecutive tree nodes x H heads; all of them attend over the
 // SAME staged key rows (key == value, MQA), so S = Q K^T and O = P K are dense contractions.  Which node sees which key is
 // a per-key bitmask applied to the S fragment after it is read back from tensor memory.
 //
-//   tc_plan_kernel   per (sequence, plan tile): the keys visible to at least one node of the tile.
-//                    mode 1 (every node selects all CSA candidates, or the CSA slab is at most 2 x topk rows): contiguous
-//                    runs {CSA slab, HCA slab, window ring, packed misc rows} as 32-row TMA boxes + node masks;
-//                    mode 0 (selection far from dense): row pointers of the union of the nodes' selections + masks.
+//   tc_plan_kernel   per (sequence, plan tile): the keys visible to at least one node of the tile, as four runs {CSA
+//                    entries, HCA entries, window ring, packed misc rows} padded to 32 rows, with a node mask per key.
+//                    Contiguous-run tiles (every node selects all CSA candidates, or the CSA slab is at most 2 x topk
+//                    rows): the runs as 32-row TMA boxes.  Gathered tiles (selection far from dense, or a paged pool
+//                    whose pages do not hold whole boxes): the first run holds only the entries some node of the tile
+//                    selected, and every key is named by array << 30 | row for four-row TMA gathers.
 //                    Each tile CTA leaves its record {tile, mode, keys} at the scheduling position the selection kernel
 //                    computed (most keys first); an extra CTA per sequence packs the small scattered rows.
-//   tc_attn_kernel   mode-0 tiles, one CTA per 128 rows and chunk of <= 512 keys:
-//       phase 1  S[128 x CL] = Q K^T      tcgen05.mma kind::f16, A = Q slice (smem, K-major), B = 256 key rows x 64 dims
-//       phase 2  exact softmax of the chunk on the fp32 S read with tcgen05.ld; P (bf16) written back over S (tcgen05.st)
-//       phase 3  O[128 x 256] = P K[:, half] twice; A = P from TMEM, B = 64 key rows x 256 dims (smem, MN-major)
-//     Operand tiles stream through a ring of seven 32 KiB slots filled with 16-byte cp.async copies written in the
-//     128-byte swizzle pattern (any row from any source array, zero fill for padding), four stages ahead of the MMA
-//     issue; slots are released by tcgen05.commit on per-slot mbarriers.  Every wait is bounded.
-//   tc_combine_kernel merges the chunks of mode-0 tiles that needed more than one (fixed order), per 128 rows.
+//   tc_combine_pair_kernel  merges the chunks of the paired kernel's multi-chunk tiles (fixed order).
 #include "tc_common.cuh"
 
 namespace tsv {
@@ -38,7 +32,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   const int tile = blockIdx.x, b = blockIdx.y, D = s.D, H = s.H;
   const int npt = tc::PR / H, n0 = tile * npt;
   const size_t tix = (size_t)b * pl.tc_nt + tile;
-  uint64_t* kptr = reinterpret_cast<uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
+  uint32_t* krow = reinterpret_cast<uint32_t*>(ws + pl.off_krow) + tix * pl.tc_maxk;    // gathered tiles: array << 30 | row per key
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
   // the done flags and the cache row offsets are fetched together with the tree scalars (one memory latency for all)
@@ -60,7 +54,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     // The extra CTA of the sequence (grid x = tiles + 1): rows that are small and scattered (few HCA entries, tree nodes,
     // entries closed inside the tree) are packed into one contiguous per-sequence buffer so that TMA boxes can fetch
     // them.  Kept off the tile CTAs: the copy is a chain of its own (addresses, loads, stores).
-    if (tm.status || !pl.tc_tma) return;
+    if (tm.status) return;
     const size_t rowb = (size_t)s.d * 2;
     const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
     int ncd = 0, nhd = 0;
@@ -124,11 +118,10 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   }
   __syncthreads();
   int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
-  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = pl.tc_tma ? 1 : 0; } return; }
+  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = 1; } return; }
   const int nvalid = min(npt, tm.nn - n0);
   const uint32_t validbits = (1u << nvalid) - 1u;
   const int n_csa = tm.n_csa;
-  const size_t rowb = (size_t)s.d * 2;
   // Ranked nodes: node bits per committed CSA entry (cmask) and, per node, which blocks closed inside the tree are in
   // its selection (bit = block index - n_csa).  The selection kernel left, for every node that ranks, a byte per
   // candidate (1 = selected): the rows of the tile's nodes are combined sixteen entries at a time (coalesced 16-byte
@@ -184,7 +177,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const int dblk = (tm.L + tm.depth[a]) / s.m_csa - n_csa;
     return dblk >= 0 && dblk < 32 && ((newc_bits[nl] >> dblk) & 1u);
   };
-  if (pl.tc_tma) {
+  {
     // the packed per-sequence rows (written by the sequence's extra CTA): few HCA entries, tree nodes, entries closed in the tree
     const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
     int ncd = 0, nhd = 0;
@@ -197,7 +190,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const bool runs_ok = !GENERAL || ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax));
     int n_uni = n_csa;                                 // keys of the first run
     __shared__ int uni_tot;
-    uint32_t* krow = reinterpret_cast<uint32_t*>(kptr);
     if (!runs_ok) {
       // Ordered compaction of the selected entries: a thread owns `per` consecutive entries, counts its selected ones
       // (four mask bytes per word), one block scan, then writes its rows and masks at consecutive positions.
@@ -289,75 +281,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       return;
     }
   }
-  if (threadIdx.x == 0) *mode = 0;
-  // committed CSA entries, in index order
-  // warp w owns a contiguous share of the entries: count its selected ones, exchange the counts once, then write the
-  // pointers in index order at positions found with ballots (no block-wide scan per 256 entries: runs are up to 32768 long)
-  int base = 0;
-  {
-    __shared__ int wcnt[8];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int share = ((n_csa + 7) / 8 + 31) & ~31;
-    const int beg = min(n_csa, w * share), end = min(n_csa, beg + share);
-    auto mask_of = [&](int i) -> uint32_t { return i < end ? (dense ? validbits : (uint32_t)cmask[phys(i)]) : 0u; };
-    int cnt = 0;
-    for (int i0 = beg; i0 < end; i0 += 32) cnt += mask_of(i0 + lane) != 0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    if (lane == 0) wcnt[w] = cnt;
-    __syncthreads();
-    int pos0 = 0, total = 0;
-    for (int x = 0; x < 8; ++x) { if (x < w) pos0 += wcnt[x]; total += wcnt[x]; }
-    const uint32_t lt = (1u << lane) - 1u;
-    for (int i0 = beg; i0 < end; i0 += 32) {
-      const int i = i0 + lane;
-      const uint32_t m = mask_of(i);
-      const uint32_t sel_m = __ballot_sync(0xffffffffu, m != 0);
-      if (m) {
-        const int pos = pos0 + __popc(sel_m & lt);
-        kptr[pos] = (uint64_t)((const char*)c.csa_kv + (size_t)csa_row(i) * rowb); kmask[pos] = (uint8_t)m;
-      }
-      pos0 += __popc(sel_m);
-    }
-    base = total;
-  }
-  // committed HCA entries
-  for (int i = threadIdx.x; i < tm.n_hca; i += blockDim.x) {
-    kptr[base + i] = (uint64_t)((const char*)c.hca_kv + (size_t)hca_row(i) * rowb); kmask[base + i] = (uint8_t)validbits;
-  }
-  base += tm.n_hca;
-  // committed window positions seen by at least one node of the tile
-  int lo = tm.L;
-  for (int nl = 0; nl < nvalid; ++nl) lo = min(lo, win_lo[nl]);
-  for (int i = threadIdx.x; i < tm.L - lo; i += blockDim.x) {
-    const int pos = lo + i;
-    uint32_t m = 0;
-    for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
-    kptr[base + i] = (uint64_t)((const char*)c.win_kv + (size_t)tok_row_of(c, s, b, pos) * rowb); kmask[base + i] = (uint8_t)m;
-  }
-  base += max(0, tm.L - lo);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    // tree nodes (ancestors-or-self) and the entries closed inside the tree at strict ancestors
-    for (int j = 0; j < tm.nn; ++j) {
-      uint32_t mt = 0, mc = 0, mh = 0;
-      for (int nl = 0; nl < nvalid; ++nl) {
-        const int n = n0 + nl;
-        if (!((tm.anc[n] >> j) & 1u)) continue;
-        mt |= 1u << nl;
-        if (j == n) continue;
-        if (hdone[j]) mh |= 1u << nl;
-        if (cdone[j]) {
-          if (newc_selected(nl, j)) mc |= 1u << nl;        // ranked nodes: is the entry in the node's selection?
-        }
-      }
-      const size_t nrow = (size_t)b * D + j;
-      if (mt) { kptr[base] = (uint64_t)((const char*)nd.kv + nrow * rowb); kmask[base++] = (uint8_t)mt; }
-      if (mc) { kptr[base] = (uint64_t)((const char*)sc.new_csa_kv + nrow * rowb); kmask[base++] = (uint8_t)mc; }
-      if (mh) { kptr[base] = (uint64_t)((const char*)sc.new_hca_kv + nrow * rowb); kmask[base++] = (uint8_t)mh; }
-    }
-    *nkeys = base;
-  }
 }
 
 // Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the scheduling
@@ -381,361 +304,7 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   }
 }
 
-// ------------------------------------------------------------------------------------------------ attention
-namespace tc {
-
-// 16 key-row pointers per thread: keys (tid>>3) + 32 j of the chunk, j = 0..15.  They serve the
-// K stages of phase 1 (key tile kt, rows 32 i: j = 8 kt + i) and the V stages of phase 3
-// (64-key block kb, rows 32 i: j = 2 kb + i).
-struct KeyPtrs { const char* p[16]; uint32_t valid; };
-
-template <int KT>
-__device__ __forceinline__ void load_k_stage(const KeyPtrs& kp, uint32_t slot, int dk, int ntk, int tid) {
-  const int r0 = tid >> 3, c = tid & 7;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if (i * 32 < ntk) {
-      const int r = r0 + 32 * i;
-      cp16(slot + r * 128 + ((c ^ (r & 7)) << 4), kp.p[8 * KT + i] + dk * 128 + c * 16, (kp.valid >> (8 * KT + i)) & 1u);
-    }
-  }
-}
-template <int KB>
-__device__ __forceinline__ void load_v_stage(const KeyPtrs& kp, uint32_t slot, int half, int tid) {
-  const int r0 = tid >> 3, c = tid & 7;
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    const int r = r0 + 32 * i;
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      cp16(slot + j * 8192 + r * 128 + ((c ^ (r & 7)) << 4), kp.p[2 * KB + i] + (half * 4 + j) * 128 + c * 16, (kp.valid >> (2 * KB + i)) & 1u);
-  }
-}
-
-}  // namespace tc
-
-__global__ void __launch_bounds__(tc::THREADS, 1) tc_attn_kernel(const tsv_shape s, const TvaPlan pl, const tsv_nodes nd, void* __restrict__ out_,
-                                                                 char* __restrict__ ws, int32_t* __restrict__ status) {
-  using namespace tc;
-  extern __shared__ unsigned char smem_raw[];
-  const int chunk = blockIdx.x, rt = blockIdx.y, tile = rt >> 1, b = blockIdx.z;     // rt: 128-row tile; tile: its plan tile
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int D = s.D, H = s.H;
-  const size_t tix = (size_t)b * pl.tc_nt + tile;
-  const size_t rix = (size_t)b * 2 * pl.tc_nt + rt;
-  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 0) return;      // a contiguous-run tile: the TMA kernel's
-  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
-  const int rows_seq = D * H;
-  if (rt * BM >= rows_seq) return;                              // second half of a plan tile that ends before it
-  const int row0 = rt * BM;                                     // first row of the CTA's tile within the sequence
-  bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
-  if (nk <= 0) {                                                // flagged sequence or padding-only tile: zeros
-    if (chunk == 0)
-      for (int i = tid; i < BM * DH / 8; i += THREADS)
-        if (row0 + i / (DH / 8) < rows_seq) reinterpret_cast<uint4*>(out)[i] = make_uint4(0, 0, 0, 0);
-    return;
-  }
-  int nch, CL;
-  chunking(nk, nch, CL);
-  if (chunk >= nch) return;
-  const int cbeg = chunk * CL, cend = min(nk, cbeg + CL);
-
-  // ---- shared memory carve-up (tiles need 1024-byte alignment for the 128-byte swizzle)
-  unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  Small& sm = *reinterpret_cast<Small*>(base);
-  const uint32_t ring = smem_u32(base + SMALL);
-  int fail = 0;
-
-  if (tid == 0) {
-    for (int i = 0; i < NS; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.slot_free[i])));
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.acc_bar)));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  // key masks of the chunk and this thread's 16 key-row pointers
-  const uint64_t* kptr_g = reinterpret_cast<const uint64_t*>(ws + pl.off_kptr) + tix * pl.tc_maxk;
-  const uint8_t* kmask_g = reinterpret_cast<const uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
-  for (int i = tid; i < NC; i += THREADS) sm.kmask[i] = (cbeg + i < cend) ? kmask_g[cbeg + i] : (uint8_t)0;
-  KeyPtrs kp;
-  kp.valid = 0;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const int key = cbeg + (tid >> 3) + 32 * j;
-    const bool v = key < cend;
-    kp.p[j] = v ? reinterpret_cast<const char*>(kptr_g[key]) : reinterpret_cast<const char*>(nd.q);
-    kp.valid |= (uint32_t)v << j;
-  }
-  fence_before();
-  __syncthreads();
-  fence_after();
-  const uint32_t tm = sm.tmem_base;
-
-  // ---- stage stream
-  const int nkt = (CL + 255) / 256;                 // key tiles of <= 256 keys
-  const int per_dk = 1 + nkt;                       // one Q stage + nkt K stages per 64-wide slice of d
-  const int G1 = 8 * per_dk;                        // stages of phase 1
-  const int nvs = CL / 64;                          // V stages per half of d
-  const int GT = G1 + 2 * nvs;
-  const char* qsrc = reinterpret_cast<const char*>(nd.q) + ((size_t)b * rows_seq + row0) * DH * 2;
-
-  auto load_stage = [&](int g) {
-    if (g < GT) {
-      const uint32_t slot = ring + (uint32_t)(g % NS) * SLOT;
-      if (g < G1) {
-        const int dk = g / per_dk, r = g % per_dk;
-        if (r == 0) {                               // Q slice: 128 rows x 64 dims
-          const int r0 = tid >> 3, c = tid & 7;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int row = r0 + 32 * i;
-            cp16(slot + row * 128 + ((c ^ (row & 7)) << 4), qsrc + (size_t)row * DH * 2 + dk * 128 + c * 16, row0 + row < rows_seq);
-          }
-        } else {
-          const int kt = r - 1, ntk = min(256, CL - kt * 256);
-          if (kt == 0) load_k_stage<0>(kp, slot, dk, ntk, tid); else load_k_stage<1>(kp, slot, dk, ntk, tid);
-        }
-      } else {
-        const int gv = g - G1, half = gv / nvs, kb = gv % nvs;
-        switch (kb) {
-          case 0: load_v_stage<0>(kp, slot, half, tid); break;
-          case 1: load_v_stage<1>(kp, slot, half, tid); break;
-          case 2: load_v_stage<2>(kp, slot, half, tid); break;
-          case 3: load_v_stage<3>(kp, slot, half, tid); break;
-          case 4: load_v_stage<4>(kp, slot, half, tid); break;
-          case 5: load_v_stage<5>(kp, slot, half, tid); break;
-          case 6: load_v_stage<6>(kp, slot, half, tid); break;
-          default: load_v_stage<7>(kp, slot, half, tid); break;
-        }
-      }
-    }
-    cp_commit();
-  };
-
-  const uint32_t idesc_k256 = make_idesc(256, 0), idesc_k128 = make_idesc(128, 0), idesc_v = make_idesc(256, 1);
-  const int q4 = warp & 3, hh = warp >> 2;          // TMEM lane quarter of this warp; column half it works on
-  const int row = q4 * 32 + lane;
-  const uint32_t tlane = tm + ((uint32_t)(q4 * 32) << 16);
-  const uint32_t mybit = 1u << ((rt & 1) * (BM / H) + row / H);
-  const float scale2 = s.sm_scale * 1.4426950408889634f;
-  float m_row = 0.f, l_row = 0.f;
-  uint32_t acc_parity = 0;
-
-  // epilogue of one half of d: O[128 x 256] in TMEM columns 256..511
-  auto epilogue = [&](int half) {
-    if (!fail && !mbar_wait(&sm.acc_bar, acc_parity)) fail = 1;
-    acc_parity ^= 1u;
-    fence_after();
-    const bool rowok = row0 + row < rows_seq;
-    if (nch == 1) {
-      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-      bf16* orow = out + (size_t)row * DH + half * 256 + hh * 128;
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tlane + 256 + hh * 128 + c0, r);
-        if (rowok) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            float f[8];
-#pragma unroll
-            for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(r[v * 8 + t]) * inv;
-            st16(orow + c0 + v * 8, f);
-          }
-        }
-      }
-    } else {
-      float* po = reinterpret_cast<float*>(ws + pl.off_tpo) + ((rix * pl.tc_chmax + chunk) * BM + row) * DH + half * 256 + hh * 128;
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tlane + 256 + hh * 128 + c0, r);
-#pragma unroll
-        for (int v = 0; v < 8; ++v)
-          *reinterpret_cast<float4*>(po + c0 + v * 4) = make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
-                                                                    __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-      }
-      if (half == 0 && hh == 0)
-        reinterpret_cast<float2*>(ws + pl.off_tpml)[(rix * pl.tc_chmax + chunk) * BM + row] = make_float2(m_row, l_row);
-    }
-    fence_before();
-    __syncthreads();                                 // O columns may be overwritten by the next half
-    fence_after();
-  };
-
-  // exact softmax of the chunk: S (fp32, columns 0..CL) -> P (bf16 pairs, columns 0..CL/2)
-  auto softmax = [&]() {
-    if (!fail && !mbar_wait(&sm.acc_bar, acc_parity)) fail = 1;
-    acc_parity ^= 1u;
-    fence_after();
-    const int nblk = CL / 128;
-    float mx = -INFINITY;
-    for (int e = 0; e < 2; ++e) {
-      const int jb = 2 * e + hh;
-      if (jb < nblk) {
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(tlane + jb * 128 + c0, r);
-#pragma unroll
-          for (int t = 0; t < 32; ++t)
-            if (sm.kmask[jb * 128 + c0 + t] & mybit) mx = fmaxf(mx, __uint_as_float(r[t]));
-        }
-      }
-    }
-    sm.xch[hh][row] = mx;
-    __syncthreads();
-    mx = fmaxf(sm.xch[0][row], sm.xch[1][row]);
-    m_row = mx * scale2;                              // scale2 > 0
-    const float moff = (mx == -INFINITY) ? 0.f : m_row;
-    float sum = 0.f;
-    for (int e = 0; e < 2; ++e) {
-      const int jb = 2 * e + hh;
-      uint32_t pk[64];
-      if (jb < nblk) {
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(tlane + jb * 128 + c0, r);
-#pragma unroll
-          for (int t = 0; t < 32; t += 2) {
-            const uint32_t mk0 = sm.kmask[jb * 128 + c0 + t] & mybit, mk1 = sm.kmask[jb * 128 + c0 + t + 1] & mybit;
-            const float p0 = mk0 ? ex2(fmaf(__uint_as_float(r[t]), scale2, -moff)) : 0.f;
-            const float p1 = mk1 ? ex2(fmaf(__uint_as_float(r[t + 1]), scale2, -moff)) : 0.f;
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);       // low half = even key
-            const float2 back = __bfloat1622float2(h2);
-            sum += back.x + back.y;
-            pk[(c0 + t) >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-        }
-      }
-      fence_before();
-      __syncthreads();                                // every warp has read S blocks 2e and 2e+1
-      fence_after();
-      if (jb < nblk) {
-#pragma unroll
-        for (int v = 0; v < 4; ++v) tmem_st16(tlane + jb * 64 + v * 16, pk + v * 16);
-      }
-    }
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-    sm.xch[hh][row] = sum;
-    fence_before();
-    __syncthreads();
-    fence_after();
-    l_row = sm.xch[0][row] + sm.xch[1][row];
-  };
-
-  // prologue: LOOK stages in flight
-  for (int g = 0; g < LOOK; ++g) load_stage(g);
-
-  for (int g = 0; g < GT; ++g) {
-    cp_wait<LOOK - 1>();                              // stage g has landed (this thread's copies)
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (g == G1) softmax();                           // S complete -> P in TMEM (also syncs the CTA)
-    else if (g == G1 + nvs) epilogue(0);
-    fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      fence_after();
-      const uint32_t slot = ring + (uint32_t)(g % NS) * SLOT;
-      if (g < G1) {
-        const int dk = g / per_dk, r = g % per_dk;
-        if (r > 0) {
-          const int kt = r - 1, ntk = min(256, CL - kt * 256);
-          const uint32_t qslot = ring + (uint32_t)((dk * per_dk) % NS) * SLOT;
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_ss(tm + kt * 256, make_desc(qslot + ks * 32, 16, 1024), make_desc(slot + ks * 32, 16, 1024),
-                   ntk == 256 ? idesc_k256 : idesc_k128, (dk | ks) != 0);
-          mma_commit(&sm.slot_free[g % NS]);
-          if (r == per_dk - 1) mma_commit(&sm.slot_free[(dk * per_dk) % NS]);        // Q slice no longer needed
-          if (g == G1 - 1) mma_commit(&sm.acc_bar);
-        }
-      } else {
-        const int gv = g - G1, kb = gv % nvs;
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          mma_ts(tm + 256, tm + kb * 32 + ks * 8, make_desc(slot + ks * 2048, 8192, 1024), idesc_v, (kb | ks) != 0);
-        mma_commit(&sm.slot_free[g % NS]);
-        if (kb == nvs - 1) mma_commit(&sm.acc_bar);
-      }
-    }
-    // refill the slot of stage g-3 (its release was committed at least two iterations ago) with stage g+LOOK
-    const int rs = g - 3;
-    if (rs >= 0 && rs + NS < GT) {
-      if (!fail && !mbar_wait(&sm.slot_free[rs % NS], (uint32_t)(rs / NS) & 1u)) fail = 1;
-    }
-    load_stage(g + LOOK);
-  }
-  epilogue(1);
-  cp_wait<0>();
-  if (fail && lane == 0) atomicOr(status + b, TSV_ST_INTERNAL);
-  fence_before();
-  __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tm) : "memory");
-}
-
-// ------------------------------------------------------------------------------------------------ combine
-__global__ void __launch_bounds__(256) tc_combine_kernel(const tsv_shape s, const TvaPlan pl, void* __restrict__ out_, const char* __restrict__ ws) {
-  using namespace tc;
-  const int rt = blockIdx.x, tile = rt >> 1, b = blockIdx.y;
-  const size_t tix = (size_t)b * pl.tc_nt + tile, rix = (size_t)b * 2 * pl.tc_nt + rt;
-  const int nk = reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix];
-  int nch, CL;
-  if (reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix] != 0) return;     // a tile of the paired kernel
-  chunking(nk, nch, CL);
-  if (nk <= 0 || nch <= 1) return;
-  const int rows_seq = s.D * s.H, row0 = rt * BM;
-  bf16* out = reinterpret_cast<bf16*>(out_) + ((size_t)b * rows_seq + row0) * DH;
-  const float* po = reinterpret_cast<const float*>(ws + pl.off_tpo) + rix * pl.tc_chmax * BM * DH;
-  const float2* pml = reinterpret_cast<const float2*>(ws + pl.off_tpml) + rix * pl.tc_chmax * BM;
-  // grid z splits the tile's 128 rows into groups of 8: a warp merges one row, a lane owns columns 4 (l + 32 k) .. + 3.
-  // The chunks are accumulated in order (the result does not depend on the launch shape), four chunks' loads in flight.
-  const int lane = threadIdx.x & 31, row = blockIdx.z * 8 + (threadIdx.x >> 5);
-  if (row >= BM || row0 + row >= rows_seq) return;
-  float m = -INFINITY;
-  for (int ch = lane; ch < nch; ch += 32) { const float2 ml = pml[ch * BM + row]; if (ml.y > 0.f) m = fmaxf(m, ml.x); }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  float l = 0.f;
-  float4 acc[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c0 = 0; c0 < nch; c0 += 4) {
-    float2 ml[4];
-    float4 v[4][4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int ch = c0 + u < nch ? c0 + u : nch - 1;
-      ml[u] = pml[ch * BM + row];
-      const float4* p4 = reinterpret_cast<const float4*>(po + ((size_t)ch * BM + row) * DH);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) v[u][k] = p4[lane + 32 * k];
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (c0 + u >= nch || !(ml[u].y > 0.f)) continue;
-      const float w = exp2f(ml[u].x - m);
-      l = fmaf(ml[u].y, w, l);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        acc[k].x = fmaf(v[u][k].x, w, acc[k].x); acc[k].y = fmaf(v[u][k].y, w, acc[k].y);
-        acc[k].z = fmaf(v[u][k].z, w, acc[k].z); acc[k].w = fmaf(v[u][k].w, w, acc[k].w);
-      }
-    }
-  }
-  const float inv = l > 0.f ? 1.f / l : 0.f;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k].x * inv, acc[k].y * inv), hi = __floats2bfloat162_rn(acc[k].z * inv, acc[k].w * inv);
-    uint2 o2;
-    o2.x = *reinterpret_cast<const uint32_t*>(&lo); o2.y = *reinterpret_cast<const uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(out + (size_t)row * DH + 4 * (lane + 32 * k)) = o2;
-  }
-}
-
+// ------------------------------------------------------------------------------------------------ merge
 // Merge of the paired kernel's multi-chunk tiles (launched with its general instantiation): every chunk left its NORMALISED partial output (bf16) with
 // the row's (reference max, sum); the row's output is the average of the partial outputs weighted by sum * 2^(max - row max).
 // grid (128-row tiles, sequences, groups of 8 rows): a warp merges one row, a lane owns 16 consecutive columns; the chunks
@@ -823,9 +392,6 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
 }
 
 static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) + 4 * 256 + 16 : 0; }   // node bits per entry, cleared by words (+ the padding words)
-// The pointer-gather kernel (and its merge kernel) serves every tile when the caches do not allow TMA (the caller gave no
-// row counts of the cache arrays); otherwise all tiles go to the paired kernel.
-static bool gather_kernel_needed(bool tma) { return !tma; }
 // Can the plan kernel produce a gathered tile for these capacities?  (A committed CSA run longer than twice the
 // selection size, or a paged pool whose pages do not hold whole 32-row boxes of a layer.)
 static bool gathered_tiles_possible(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c) {
@@ -840,54 +406,33 @@ static bool gathered_tiles_possible(const tsv_shape& s, const TvaPlan& p, const 
 
 // Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
-  prep.tma = tva_tc_pair_usable(c) ? 1 : 0;
   const size_t plan_sm = plan_smem_bytes(p);
   if (plan_sm > 32 * 1024 && (cudaFuncSetAttribute(tc_plan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess ||
                               cudaFuncSetAttribute(tc_plan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)) {
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
-  if (gather_kernel_needed(prep.tma) &&
-      cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess) {
-    cudaGetLastError();
-    return TSV_ERR_CUDA;
-  }
   TSV_PREP(tc_plan_kernel<true>);
   TSV_PREP(tc_plan_kernel<false>);
-  TSV_PREP(tc_attn_kernel);
-  TSV_PREP(tc_combine_kernel);
   TSV_PREP(tc_combine_pair_kernel);
-  if (prep.tma) return prepare_tva_tc_pair(s, p, c, nd, out, ws, prep);
-  return TSV_OK;
+  return prepare_tva_tc_pair(s, p, c, nd, out, ws, prep);
 }
 
-int launch_tva_tc(const tsv_shape& s, const TvaPlan& p_in, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
+int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
-  TvaPlan p = p_in;
-  p.tc_tma = prep.tma;
-  const bool gathered = !p.tc_tma || gathered_tiles_possible(s, p, c);
-  const dim3 pgrid(p.tc_nt + (p.tc_tma ? 1 : 0), s.B);                                                            // x: tiles (+ the packing CTA)
+  const bool gathered = gathered_tiles_possible(s, p, c);
+  const dim3 pgrid(p.tc_nt + 1, s.B);                                                                              // x: tiles + the packing CTA
   if (gathered) tc_plan_kernel<true><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
   else tc_plan_kernel<false><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
   count_launch();
-  if (p.tc_tma) {
-    // general: some tile may have more than two chunks of the longest kind, or be gathered; then every multi-chunk tile
-    // leaves bf16 partial outputs for the merge kernel
-    const bool general = (p.tc_maxk + tc::NCX - 1) / tc::NCX > 2 || gathered;
-    const int r = launch_tva_tc_pair(s, p, prep, general, out, ws, status, st);
-    if (r != TSV_OK) return r;
-    if (general && p.tc_chmax > 1) {
-      tc_combine_pair_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);
-      count_launch();
-    }
-  }
-  if (gather_kernel_needed(p.tc_tma)) {
-    tc_attn_kernel<<<dim3(p.tc_chmax, 2 * p.tc_nt, s.B), tc::THREADS, tc::SMEM_BYTES, st>>>(s, p, nd, out, ws, status);
+  // general: some tile may have more than two chunks of the longest kind, or be gathered; then every multi-chunk tile
+  // leaves bf16 partial outputs for the merge kernel
+  const bool general = (p.tc_maxk + tc::NCX - 1) / tc::NCX > 2 || gathered;
+  const int r = launch_tva_tc_pair(s, p, prep, general, out, ws, status, st);
+  if (r != TSV_OK) return r;
+  if (general && p.tc_chmax > 1) {
+    tc_combine_pair_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);   // z: groups of 8 rows
     count_launch();
-    if (p.tc_chmax > 1) {
-      tc_combine_kernel<<<dim3(2 * p.tc_nt, s.B, tc::BM / 8), 256, 0, st>>>(s, p, out, ws);   // z: groups of 8 rows
-      count_launch();
-    }
   }
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }

@@ -237,8 +237,7 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
     // Gathered tiles: the keys' row codes stay in global memory (the tile plan left them there, four-aligned groups
     // never mix arrays); lane l fetches the codes of rows 4 l .. 4 l + 3 of a stage itself.  Keys past the end of the list
     // read row 0 of the first array (they are masked).
-    // (the list shares the tile's slot of 8 bytes per key with the row pointers of the pointer-gather kernel)
-    const uint4* code_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(ws + pl.off_kptr + tix * (size_t)pl.tc_maxk * 8) + cbeg);
+    const uint4* code_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(ws + pl.off_krow) + tix * (size_t)pl.tc_maxk + cbeg);
     auto codes_at = [&](int key) { return cbeg + key < cend ? __ldg(code_g + (key >> 2)) : make_uint4(0u, 0u, 0u, 0u); };
     uint4 kcode = make_uint4(0u, 0u, 0u, 0u);                                // this lane's codes of the current piece's K stages
     int kcode_pc = -1;
@@ -718,7 +717,7 @@ static bool make_map(CUtensorMap* m, const void* basep, int64_t rows, int box_ro
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool tva_tc_pair_usable(const tsv_cache& c) { return c.csa_rows > 0 && c.hca_rows > 0 && encode_fn() != nullptr; }
+bool tva_tc_pair_usable(const tsv_cache& c) { return c.csa_rows > 0 && encode_fn() != nullptr; }
 
 static_assert(sizeof(pair::MapSet) <= sizeof(TvaTcPrep::maps), "tensor-map block of TvaTcPrep too small");
 
@@ -726,8 +725,10 @@ static_assert(sizeof(pair::MapSet) <= sizeof(TvaTcPrep::maps), "tensor-map block
 // the tensor maps and the kernel's shared-memory attribute.
 int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
   pair::MapSet& ms = *reinterpret_cast<pair::MapSet*>(prep.maps);
-  const void* bases[4] = {c.csa_kv, c.hca_kv, c.win_kv, ws + p.off_misc};
-  const int64_t rows[4] = {c.csa_rows, c.hca_rows, c.page_table ? c.tok_rows : (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
+  // (a layer without HCA entries has no HCA array to map: its map is never used and stands in as a copy of the CSA one)
+  const bool has_hca = c.hca_rows > 0 && c.hca_kv;
+  const void* bases[4] = {c.csa_kv, has_hca ? c.hca_kv : c.csa_kv, c.win_kv, ws + p.off_misc};
+  const int64_t rows[4] = {c.csa_rows, has_hca ? c.hca_rows : c.csa_rows, c.page_table ? c.tok_rows : (int64_t)s.B * s.window, (int64_t)s.B * p.tc_misc_rows};
   bool ok = make_map(&ms.q, nd.q, (int64_t)s.B * s.D * s.H, 128) && make_map(&ms.out, out, (int64_t)s.B * s.D * s.H, 32);
   for (int a = 0; a < 4 && ok; ++a) {
     for (int k = 0; k < 3 && ok; ++k) ok = make_map(&ms.src[a][k], bases[a], rows[a], 32 << k);

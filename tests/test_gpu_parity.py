@@ -388,6 +388,25 @@ def test_candidate_lists_beyond_the_cluster_capacity():
     lockstep(cfg, cycles=1)
 
 
+def test_tensor_core_shape_without_row_counts_takes_the_cuda_core_path(monkeypatch):
+    """A cache handed over without the row counts of its arrays (csa_rows = 0) gives the library nothing to build tensor
+    maps from: a shape of the tensor-core path then runs on the CUDA-core path, through the same workspace."""
+    from paper_2609_24698_b200 import binding as tsv
+    orig = tsv.LayerCache.struct
+
+    def no_rows(self):
+        st = orig(self)
+        st.csa_rows = 0
+        st.hca_rows = 0
+        return st
+    cfg = synth.Config("tc_no_rows", 76, synth.Shape("bf16", 3, 8, 64, 512, 4, 64, 4, 128, 128, 128), L_min=150, L_max=700, seed=12)
+    _, forced, _ = lockstep(cfg, cycles=1, flags=tsv.FLAG_FORCE_SIMT, return_engine=True)
+    monkeypatch.setattr(tsv.LayerCache, "struct", no_rows)
+    _, eng, _ = lockstep(cfg, cycles=1, return_engine=True)
+    for a, b in zip(eng.out, forced.out):                # bit for bit what the CUDA-core path gives when asked for by flag
+        assert torch.equal(a, b)
+
+
 def test_ranked_short_candidate_lists_bf16():
     """Benchmark head shape with a small top-k: every node ranks its candidates, the lists are short enough to be scored
     inside the selection kernel (256-byte indexer rows), and the committed runs lie on both sides of 2 x topk, so ranked
