@@ -32,7 +32,7 @@ __device__ __forceinline__ uint32_t order_key(float f) {       // larger float -
 // Ranks the 256-row attention tiles of all sequences by the number of keys they will stage, most first, so that the
 // paired attention kernel starts the long tiles first and the short ones fill the tail (run by ONE CTA of the selection
 // launch).  The counts follow from lengths, node counts and done flags alone (for tiles on the contiguous-run path they
-// are exact; for pointer-gather tiles an estimate: only the order depends on them), so the ranking is ready before the
+// are exact; for gathered tiles an estimate: only the order depends on them), so the ranking is ready before the
 // plan kernel runs and each plan CTA can leave its record at its final position.
 // nk_est: shared memory for 2048 ints.
 __device__ __forceinline__ void rank_tiles_in(int32_t* nk_est, const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,

@@ -410,7 +410,7 @@ def test_tensor_core_shape_without_row_counts_takes_the_cuda_core_path(monkeypat
 def test_ranked_short_candidate_lists_bf16():
     """Benchmark head shape with a small top-k: every node ranks its candidates, the lists are short enough to be scored
     inside the selection kernel (256-byte indexer rows), and the committed runs lie on both sides of 2 x topk, so ranked
-    tiles take the contiguous-run path with per-node masks as well as the pointer-gather path."""
+    tiles take the contiguous-run path with per-node masks as well as the gathered path."""
     cfg = synth.Config("ranked_short", 71, synth.Shape("bf16", 6, 8, 64, 512, 4, 128, 4, 128, 128, 128),
                        L_min=300, L_max=1400, seed=9)
     lockstep(cfg, cycles=2)
@@ -448,21 +448,21 @@ def _plant_peaks(cfg, gap_nats=14.0):
 def test_tc_planted_peaks_reach_rescale_and_merge_paths():
     """Benchmark head shape.  Sequence lengths put the planted window keys into: the second piece of a single-chunk
     tile (1200), the third piece (2040), a later chunk of a multi-chunk tile on the contiguous-run path (3500:
-    n_csa <= 2 topk), and a later chunk of the pointer-gather kernel (5000: n_csa > 2 topk)."""
+    n_csa <= 2 topk), and a gathered tile (5000: n_csa > 2 topk)."""
     cfg = synth.Config("tc_peaks", 81, synth.Shape("bf16", 5, 8, topk=512, **BENCH_HEADS), L_min=1, L_max=1, seed=3)
     lockstep(cfg, cycles=1, lengths=[1200, 2040, 1660, 3500, 5000], plant=_plant_peaks(cfg), per_row=True)
 
 
 def test_tc_planted_peaks_ranked_tiles():
     """Same planted keys with a small top-k, so that every node ranks: masked-run tiles (n_csa <= 2 topk) and
-    pointer-gather tiles, single- and multi-chunk."""
+    gathered tiles, single- and multi-chunk."""
     cfg = synth.Config("tc_peaks_ranked", 82, synth.Shape("bf16", 4, 8, topk=256, **BENCH_HEADS), L_min=1, L_max=1, seed=4)
     lockstep(cfg, cycles=1, lengths=[1500, 2040, 2600, 4400], plant=_plant_peaks(cfg, gap_nats=16.0), per_row=True)
 
 
 def test_tc_peaked_scale100():
     """sm_scale = 100 on the d = 512 path: logits are O(+-5) everywhere, so one wrongly masked or dropped key moves an
-    output row by far more than the tolerance.  Lengths cover single-chunk, multi-chunk and pointer-gather tiles."""
+    output row by far more than the tolerance.  Lengths cover single-chunk, multi-chunk and gathered tiles."""
     cfg = synth.Config("tc_scale100", 83, synth.Shape("bf16", 6, 8, topk=512, sm_scale=100.0, **BENCH_HEADS), L_min=1, L_max=1, seed=5)
     lockstep(cfg, cycles=2, lengths=[300, 900, 1400, 2047, 3300, 4700], per_row=True)
 
