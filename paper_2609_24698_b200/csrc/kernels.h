@@ -76,7 +76,7 @@ int launch_topk_long(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, c
 int launch_tva_simt(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                     void* out, char* ws, int32_t* status, cudaStream_t st);
 
-constexpr int kIdxFusedMax = 2048;   // candidate capacity up to which topk_kernel computes the indexer scores itself
+constexpr int kIdxFusedMax = 2272;   // candidate capacity up to which topk_kernel computes the indexer scores itself
 constexpr int kBoxRows = 32;       // rows of one TMA box; contiguous key runs are padded to a multiple of it
 constexpr int kHcaMiscMax = 32;    // up to this many HCA entries travel in the packed per-sequence buffer
 bool tva_tc_eligible(const tsv_shape& s);
