@@ -1,11 +1,12 @@
 // branch_state_build: chain-private online compression along every root-to-node path.
 //
 // Grid (sequence, element slab).  The scalar part of every fold (max gate, sum of weights, the two
-// blend coefficients, done flags) is a chain over at most 32 nodes: thread 0 of each CTA loads all
-// gates and parents up front (independent loads, one memory latency) and walks the chain in
-// registers.  Each thread then owns ONE vector element: it loads that element of every node's
-// compression vector up front, folds along the tree with the inherited values kept in shared
-// memory (indexed by parent), and stores states and closed entries.  No load depends on a store.
+// blend coefficients, done flags) follows the tree: in every CTA one warp per compressed layer (CSA,
+// HCA) holds a node per lane, loads gates and parents up front (independent loads, one memory
+// latency) and folds level by level, the parent's result arriving by shuffle.  Each thread then owns
+// ONE vector element: it loads that element of every node's compression vector up front, folds along
+// the tree with the inherited values kept in shared memory (indexed by parent), and stores states and
+// closed entries.  No load depends on a store.
 #include "kernels.h"
 
 namespace tsv {
@@ -16,8 +17,9 @@ struct FoldCoef {
   int32_t empty;     // the inherited block holds no token (inherited numbers are ignored)
 };
 
-__device__ __forceinline__ void scalar_fold(FoldCoef& fc, float& mx_out, float& s_out, int p, int blk, float mxp, float sp, float g) {
-  const bool empty = (p % blk) == 0;
+// empty / done: position p opens / closes a block of blk tokens (they depend on the position alone: a caller that folds
+// along a chain works them out ahead of it)
+__device__ __forceinline__ void scalar_fold(FoldCoef& fc, float& mx_out, float& s_out, bool empty, bool done, float mxp, float sp, float g) {
   float mx2, a, b, s2;
   if (empty) { mx2 = g; a = 0.f; b = 1.f; s2 = 1.f; }
   else {
@@ -27,7 +29,7 @@ __device__ __forceinline__ void scalar_fold(FoldCoef& fc, float& mx_out, float& 
     s2 = fmaf(sp, a, b);
   }
   fc.a = a; fc.b = b; fc.s = s2; fc.empty = empty;
-  fc.done = ((p + 1) % blk) == 0;
+  fc.done = done;
   mx_out = fc.done ? 0.f : mx2;
   s_out = fc.done ? 0.f : s2;
 }
@@ -42,7 +44,6 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
   __shared__ FoldCoef fcs[TSV_MAX_D], fhs[TSV_MAX_D];
-  __shared__ float cmx[TSV_MAX_D], cs[TSV_MAX_D], hmx[TSV_MAX_D], hs[TSV_MAX_D];   // thread 0's chain state per node
   const int b = blockIdx.x, D = s.D;
   const int d = s.d, di = s.di;
   const int e = blockIdx.y * kBsbThreads + threadIdx.x;   // element index: [0,d) CSA kv | [d,d+di) CSA indexer key | [d+di,2d+di) HCA kv
@@ -56,45 +57,49 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
   // (they learn the length first, one load, and leave before fetching any vector)
   if (DEFER && which == 2 && blockIdx.y * kBsbThreads >= (unsigned)(d + di) && hca_deferred(s, c.L[b])) return;
   // issue this thread's loads before the scalar chain is known (padding slots load too: the memory is there)
-  float cv[DMAX];
+  T cvr[DMAX];                                         // kept as loaded: a conversion here would wait for the data before the tree's loads leave
 #pragma unroll
-  for (int n = 0; n < DMAX; ++n) cv[n] = (live && n < D) ? to_f(cin[((size_t)b * D + n) * dim + el]) : 0.f;
+  for (int n = 0; n < DMAX; ++n) cvr[n] = (live && n < D) ? cin[((size_t)b * D + n) * dim + el] : T(0.f);
   const float pv = live ? pers[(size_t)b * dim + el] : 0.f;
-  float gcl = 0.f, ghl = 0.f;                        // lane n of warp 0 fetches node n's gates; thread 0 collects them by shuffle
-  if (threadIdx.x < D) { gcl = nd.g_csa[(size_t)b * D + threadIdx.x]; ghl = nd.g_hca[(size_t)b * D + threadIdx.x]; }
-  float pcm = 0.f, pcs = 0.f, phm = 0.f, phs = 0.f;
-  if (threadIdx.x == 0) { pcm = c.csa_mx[b]; pcs = c.csa_s[b]; phm = c.hca_mx[b]; phs = c.hca_s[b]; }
+  // The scalar chains: warp 0 folds the CSA block states, warp 1 the HCA ones, lane n owning node n.  A node's fold needs
+  // its parent's result, so the warp walks the tree level by level (nodes of one depth fold together, the parent's
+  // running max and sum arrive by shuffle): as many steps as the tree is deep, not as it has nodes.
+  const int lane = threadIdx.x & 31, chain = threadIdx.x >> 5;      // chain 0: CSA, 1: HCA (warps 2, 3 take no part)
+  float gate = 0.f, pmx = 0.f, psum = 0.f;
+  if (chain < 2 && lane < D) gate = (chain == 0 ? nd.g_csa : nd.g_hca)[(size_t)b * D + lane];
+  if (chain < 2 && lane == 0) { pmx = (chain == 0 ? c.csa_mx : c.hca_mx)[b]; psum = (chain == 0 ? c.csa_s : c.hca_s)[b]; }
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
-  float gc[DMAX], gh[DMAX];
-  if (threadIdx.x < 32) {
-#pragma unroll
-    for (int n = 0; n < DMAX; ++n) { gc[n] = __shfl_sync(0xffffffffu, gcl, n); gh[n] = __shfl_sync(0xffffffffu, ghl, n); }
-  }
 
   const bool hdef = DEFER && hca_deferred(s, tm.L) && !tm.status;     // (tm.L is 0 for a flagged length: such a sequence commits nothing)
-  if (threadIdx.x == 0) {
+  if (chain < 2) {
     const bool writer = blockIdx.y == 0;
-    if (tm.status && writer) atomicOr(status + b, tm.status);
-    const int nn = tm.status ? 0 : tm.nn;
+    if (tm.status && writer && threadIdx.x == 0) atomicOr(status + b, tm.status);
+    const int nn = tm.status ? 0 : tm.nn, n = lane;
+    const bool valid = n < nn;
+    const int depth = valid ? tm.depth[n] : -1, par = valid && n ? tm.parent[n] : 0;
+    int maxd = depth;
 #pragma unroll
-    for (int n = 0; n < DMAX; ++n) {
-      if (n < D) {
-        float m1 = 0.f, s1 = 0.f, m2 = 0.f, s2 = 0.f;
-        if (n < nn) {
-          const int p = tm.L + tm.depth[n], par = tm.parent[n];
-          float mp = pcm, sp = pcs, mq = phm, sq = phs;
-          if (n) { mp = cmx[par]; sp = cs[par]; mq = hmx[par]; sq = hs[par]; }
-          scalar_fold(fcs[n], m1, s1, p, s.m_csa, mp, sp, gc[n]);
-          if (hdef) fhs[n].done = 0; else scalar_fold(fhs[n], m2, s2, p, s.m_hca, mq, sq, gh[n]);
-        } else {
-          fcs[n].done = fhs[n].done = 0;
-        }
-        cmx[n] = m1; cs[n] = s1; hmx[n] = m2; hs[n] = s2;
-        if (writer) {
-          sc.csa_mx[(size_t)b * D + n] = m1; sc.csa_s[(size_t)b * D + n] = s1;
-          if (!hdef) { sc.hca_mx[(size_t)b * D + n] = m2; sc.hca_s[(size_t)b * D + n] = s2; }
-          sc.csa_done[(size_t)b * D + n] = (uint8_t)fcs[n].done;
-          sc.hca_done[(size_t)b * D + n] = (uint8_t)fhs[n].done;
+    for (int o = 16; o > 0; o >>= 1) maxd = max(maxd, __shfl_xor_sync(0xffffffffu, maxd, o));
+    FoldCoef fc;
+    fc.a = fc.b = fc.s = 0.f; fc.done = 0; fc.empty = 0;
+    float mx = 0.f, sm = 0.f;                          // this node's running max and sum after its fold
+    const bool skip = chain == 1 && hdef;              // deferred schedule: no HCA branch states
+    const int blk = chain == 0 ? s.m_csa : s.m_hca, p = tm.L + max(depth, 0);
+    const bool opens = (p % blk) == 0, closes = ((p + 1) % blk) == 0;
+    if (!skip) {
+      for (int level = 0; level <= maxd; ++level) {    // uniform trip count
+        const float mp = __shfl_sync(0xffffffffu, mx, par), sp = __shfl_sync(0xffffffffu, sm, par);
+        if (depth == level)
+          scalar_fold(fc, mx, sm, opens, closes, n ? mp : pmx, n ? sp : psum, gate);
+      }
+    }
+    if (n < D) {
+      (chain == 0 ? fcs : fhs)[n] = fc;
+      if (writer) {
+        if (chain == 0) { sc.csa_mx[(size_t)b * D + n] = mx; sc.csa_s[(size_t)b * D + n] = sm; sc.csa_done[(size_t)b * D + n] = (uint8_t)fc.done; }
+        else {
+          if (!hdef) { sc.hca_mx[(size_t)b * D + n] = mx; sc.hca_s[(size_t)b * D + n] = sm; }
+          sc.hca_done[(size_t)b * D + n] = (uint8_t)fc.done;
         }
       }
     }
@@ -112,10 +117,11 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
       float acc = 0.f, ent = 0.f;
       if (n < nn) {
         const FoldCoef f = fc[n];
-        if (f.empty) acc = cv[n];
+        const float cvn = to_f(cvr[n]);
+        if (f.empty) acc = cvn;
         else {
           const float ap = n ? hist[tm.parent[n] * kBsbThreads + threadIdx.x] : pv;
-          acc = fmaf(f.a, ap, f.b * cv[n]);
+          acc = fmaf(f.a, ap, f.b * cvn);
         }
         if (f.done) { ent = acc / f.s; acc = 0.f; }
       }
