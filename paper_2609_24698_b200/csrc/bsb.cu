@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(kBsbThreads) bsb_kernel(const tsv_shape s, con
   __shared__ TreeStage tstage;
   __shared__ FoldCoef fcs[TSV_MAX_D], fhs[TSV_MAX_D];
   const int b = blockIdx.x, D = s.D;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the selection may start the part of it that does not read this kernel's results
   const int d = s.d, di = s.di;
   const int e = blockIdx.y * kBsbThreads + threadIdx.x;   // element index: [0,d) CSA kv | [d,d+di) CSA indexer key | [d+di,2d+di) HCA kv
   const bool live = e < 2 * d + di;

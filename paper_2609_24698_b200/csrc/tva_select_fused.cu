@@ -52,7 +52,9 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   float* ssm = reinterpret_cast<float*>(dsm + 4 * DI * 2);
   unsigned char* stage = dsm + 4 * DI * 2 + (size_t)score_cap * 4;
   const int t = threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile plan may start its selection-independent part
   if (blockIdx.x == (unsigned)s.D) {                  // extra CTA column (tensor-core attention path): CTA (D, 0) ranks the attention tiles
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // (the ranking reads the state build's done flags)
     if (blockIdx.y == 0) rank_tiles_in(reinterpret_cast<int32_t*>(stage), s, pl, c, nd, sc, ws);
     return;
   }
@@ -61,11 +63,10 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
   // Everything the CTA may need that depends on (b, n) alone is requested together with the tree's loads (one memory
-  // latency for all): the slab offset, the done flags, and -- used only if the node ranks -- its indexer queries and
-  // head weights.
+  // latency for all): the slab offset and -- used only if the node ranks -- its indexer queries and head weights.  The
+  // kernel is launched as a programmatic dependent of the state build: up to the wait below it reads nothing that kernel
+  // writes (the done flags follow the wait).
   if (!PAGED && t == 64) row0_sm = c.csa_row0[b];
-  if (t >= 96 && t < 96 + D) cdone_sm[t - 96] = sc.csa_done[(size_t)b * D + t - 96];
-  if (t >= 128 && t < 128 + D) hdone_sm[t - 128] = sc.hca_done[(size_t)b * D + t - 128];
   const int lane = t & 31, w = t >> 5, g = lane >> 2, tq = lane & 3;
   const bf16* iq = reinterpret_cast<const bf16*>(nd.iq) + ((size_t)b * D + n) * HI * DI;
   const float* iwp = nd.iw + ((size_t)b * D + n) * HI;
@@ -95,6 +96,10 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
   if (may_rank) issue(0);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (t >= 96 && t < 96 + D) cdone_sm[t - 96] = sc.csa_done[(size_t)b * D + t - 96];
+  if (t >= 128 && t < 128 + D) hdone_sm[t - 128] = sc.hca_done[(size_t)b * D + t - 128];
+  __syncthreads();
   if (t == 0) {
     if (tm.status && n == 0) atomicOr(status + b, tm.status);
     if (live) path_entries(pe, tm, s, n, cdone_sm, hdone_sm);
@@ -282,14 +287,20 @@ int launch_topk_fused(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   size_t bytes;
   fused_smem(p, rows, score_cap, bytes);
   const dim3 grid(s.D + (p.tc ? 1 : 0), s.B);           // + the column that ranks the attention tiles
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = bytes; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;          // may start under the state build's tail (it waits inside)
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   if (c.page_table) {
     TSV_PREP(topk_fused_kernel<true>);
     if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-    topk_fused_kernel<true><<<grid, 256, bytes, st>>>(s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
+    cudaLaunchKernelEx(&cfg, topk_fused_kernel<true>, s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
   } else {
     TSV_PREP(topk_fused_kernel<false>);
     if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-    topk_fused_kernel<false><<<grid, 256, bytes, st>>>(s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
+    cudaLaunchKernelEx(&cfg, topk_fused_kernel<false>, s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
   }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;

@@ -24,7 +24,7 @@ namespace tsv {
 // latency chain of the contiguous-run plan.
 template <bool GENERAL>
 __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
-                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
+                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask, int& pos) {
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
   __shared__ int n_cand[8], win_lo[8];
@@ -35,14 +35,19 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   uint32_t* krow = reinterpret_cast<uint32_t*>(ws + pl.off_krow) + tix * pl.tc_maxk;    // gathered tiles: array << 30 | row per key
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
-  // the done flags and the cache row offsets are fetched together with the tree scalars (one memory latency for all)
+  // the cache row offsets are fetched together with the tree scalars (one memory latency for all)
   __shared__ uint8_t cdone[TSV_MAX_D], hdone[TSV_MAX_D];
   __shared__ int64_t row0_sm[2];
-  if (threadIdx.x >= 64 && threadIdx.x < 64 + D) cdone[threadIdx.x - 64] = sc.csa_done[(size_t)b * D + threadIdx.x - 64];
-  if (threadIdx.x >= 96 && threadIdx.x < 96 + D) hdone[threadIdx.x - 96] = sc.hca_done[(size_t)b * D + threadIdx.x - 96];
   if (threadIdx.x == 40) row0_sm[0] = c.page_table ? 0 : c.csa_row0[b];
   if (threadIdx.x == 41) row0_sm[1] = c.page_table ? 0 : c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  // The kernel is launched as a programmatic dependent of the selection kernel (itself one of the state build): up to here
+  // it has read only what the caller's inputs and the committed caches hold, under those kernels' tails.  What follows
+  // reads their results: the state build's done flags and entries, the selection's scheduling positions and mask rows.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + D) cdone[threadIdx.x - 64] = sc.csa_done[(size_t)b * D + threadIdx.x - 64];
+  if (threadIdx.x >= 96 && threadIdx.x < 96 + D) hdone[threadIdx.x - 96] = sc.hca_done[(size_t)b * D + threadIdx.x - 96];
+  __syncthreads();
   // rows of the sequence's CSA and HCA entries: slabs, or through the page table of a paged pool
   RowAddr csa_row, hca_row;
   csa_row.pt = hca_row.pt = c.page_table ? c.page_table + (size_t)b * c.max_pages : nullptr;
@@ -117,6 +122,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     if (lane == 0) dense = over == 0;
   }
   __syncthreads();
+  if (threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // fetched now, used at the end (when the attention stage runs alone: the previous call's)
   int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
   if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = 1; } return; }
   const int nvalid = min(npt, tm.nn - n0);
@@ -292,11 +298,10 @@ __global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const T
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
   const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
   const size_t tix = (size_t)blockIdx.y * pl.tc_nt + blockIdx.x;
-  int pos = (int)tix;                                 // fetched now, used at the end
-  if (tile_cta && threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // (when the attention stage runs alone: the previous call's)
+  int pos = (int)tix;
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
-  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm);
+  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm, pos);
   if (tile_cta && threadIdx.x == 0) {                 // thread 0 wrote the tile's key count and mode itself
     if (pos < 0 || pos >= s.B * pl.tc_nt) pos = (int)tix;
     reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
@@ -422,8 +427,16 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, c
                   void* out, char* ws, int32_t* status, cudaStream_t st) {
   const bool gathered = gathered_tiles_possible(s, p, c);
   const dim3 pgrid(p.tc_nt + 1, s.B);                                                                              // x: tiles + the packing CTA
-  if (gathered) tc_plan_kernel<true><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
-  else tc_plan_kernel<false><<<pgrid, 256, plan_smem_bytes(p), st>>>(s, p, c, nd, sc, ws);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = pgrid; cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = plan_smem_bytes(p); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;        // may start under the selection kernel's tail (it waits inside)
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (gathered) cudaLaunchKernelEx(&cfg, tc_plan_kernel<true>, s, p, c, nd, sc, ws);
+    else cudaLaunchKernelEx(&cfg, tc_plan_kernel<false>, s, p, c, nd, sc, ws);
+  }
   count_launch();
   // general: some tile may have more than two chunks of the longest kind, or be gathered; then every multi-chunk tile
   // leaves bf16 partial outputs for the merge kernel
