@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   __shared__ int wsum[9];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile plan may start its selection-independent part
   if (blockIdx.x == (unsigned)s.D) {
     // extra CTA column (only with the tensor-core attention path): CTA (D, 0) ranks the attention tiles
     if (blockIdx.y == 0) rank_tiles(s, pl, c, nd, sc, ws);
