@@ -381,6 +381,24 @@ def test_long_candidate_lists_exact_ties_across_the_cluster(dtype, di):
     lockstep(cfg, cycles=2, plant=_plant_tied_indexer_keys(), exact_topk=True)
 
 
+@pytest.mark.parametrize("HI,topk,L_min,L_max", [(1, 40, 300, 1500), (2, 100, 900, 2400), (3, 7, 0, 60), (4, 3, 0, 24)])
+def test_selection_inside_one_cta_head_counts_and_tiny_lists(HI, topk, L_min, L_max):
+    """The one-CTA selection kernel for 128-wide bf16 indexer rows (scores by warp-level tensor-core products, keys in
+    registers) with every head count it takes, on the CUDA-core attention path (no extra CTA column); the tiny cases have
+    nodes that rank with no committed entry at all (only blocks closed inside the tree) and lists of a few candidates."""
+    cfg = synth.small_config(name=f"fused_sel_hi{HI}", dtype="bf16", B=4, D=6, H=4, d=16, m_csa=2, topk=topk, HI=HI, di=128,
+                             m_hca=32, window=16, L_min=L_min, L_max=L_max, layers=1, seed=93 + HI, cfg_id=77)
+    lockstep(cfg, cycles=3)
+
+
+def test_selection_inside_one_cta_exact_ties():
+    """Nearly all candidates share one score: the threshold's ties are decided by index in the one-CTA selection kernel
+    (keys strided over the threads, ordered write by warp shares)."""
+    cfg = synth.small_config(name="fused_ties", dtype="bf16", B=3, D=6, H=4, d=16, m_csa=2, topk=100, HI=2, di=128, m_hca=32,
+                             window=16, L_min=700, L_max=2600, layers=1, seed=97, cfg_id=78)
+    lockstep(cfg, cycles=2, plant=_plant_tied_indexer_keys(every=40), exact_topk=True)
+
+
 def test_candidate_lists_beyond_the_cluster_capacity():
     """More than 65536 candidates per node: the single-CTA selection that re-reads the score array pass after pass."""
     cfg = synth.small_config(name="huge_lists", dtype="bf16", B=1, D=4, H=4, d=16, m_csa=2, topk=40, HI=2, di=128, m_hca=64,
