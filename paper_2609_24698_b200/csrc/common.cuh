@@ -205,4 +205,32 @@ __device__ __forceinline__ int block_excl_scan_256(int v, int* wsum /* shared[9]
   return wsum[w] + x - v;
 }
 
+// The same for CTAs of up to 1024 threads (a multiple of 32): wsum is shared[33].
+__device__ __forceinline__ int block_excl_scan(int v, int* wsum, int& total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) wsum[w] = x;
+  __syncthreads();
+  if (w == 0) {                                        // the warps' totals: an exclusive scan by warp 0
+    const int tw = lane < nw ? wsum[lane] : 0;
+    int y = tw;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int z = __shfl_up_sync(0xffffffffu, y, o);
+      if (lane >= o) y += z;
+    }
+    wsum[lane] = y - tw;
+    if (lane == 31) wsum[32] = y;
+  }
+  __syncthreads();
+  total = wsum[32];
+  return wsum[w] + x - v;
+}
+
 }  // namespace tsv

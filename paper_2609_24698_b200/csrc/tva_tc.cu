@@ -138,7 +138,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   // without the padding the threads of a warp would all read the same bank.
   __shared__ uint32_t newc_bits[8];
   int psh = 3;                                         // log2(per)
-  if (GENERAL) while ((256 << psh) < n_csa) ++psh;
+  if (GENERAL) while (((int)blockDim.x << psh) < n_csa) ++psh;
   auto phys = [&](int i) { return GENERAL ? i + ((i >> psh) << 2) : i; };
   if (!dense) {
     uint32_t allbits = 0, rankbits = 0;                // nodes that take every committed entry / nodes that rank
@@ -199,7 +199,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     if (!runs_ok) {
       // Ordered compaction of the selected entries: a thread owns `per` consecutive entries, counts its selected ones
       // (four mask bytes per word), one block scan, then writes its rows and masks at consecutive positions.
-      __shared__ int wsum_c[9];
+      __shared__ int wsum_c[33];
       const uint32_t* cm32 = reinterpret_cast<const uint32_t*>(cmask);
       const int per = 1 << psh, beg = min(n_csa, (int)threadIdx.x << psh), end = min(n_csa, beg + per);
       const uint32_t* mine = cm32 + (phys(beg) >> 2);  // this thread's words (its share starts on a word: per is a multiple of 8)
@@ -211,7 +211,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         cnt += (w & 0xFFu ? 1 : 0) + (w & 0xFF00u ? 1 : 0) + (w & 0xFF0000u ? 1 : 0) + (w & 0xFF000000u ? 1 : 0);
       }
       int total;
-      int pos = block_excl_scan_256(cnt, wsum_c, total);
+      int pos = block_excl_scan(cnt, wsum_c, total);
       if (threadIdx.x == 0) uni_tot = total;
       for (int i = beg; i < end; i += 4) {
         uint32_t w = dense ? 0x01010101u * dmask : mine[(i - beg) >> 2];
@@ -292,8 +292,10 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
 // Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the scheduling
 // position the selection kernel computed for it (most keys first): the paired attention kernel takes the tiles in that
 // order and learns all it needs about its tile from one load.
-template <bool GENERAL>
-__global__ void __launch_bounds__(256) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+// NT threads per CTA: 256, or 1024 for gathered tiles over long candidate lists (the union of a tile's selections over tens
+// of thousands of entries is the work of ONE CTA, alone on its SM).
+template <bool GENERAL, int NT>
+__global__ void __launch_bounds__(NT) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                       const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
   const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
@@ -396,7 +398,7 @@ void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p) {
   p.tc_chmax = (p.tc_maxk + tc::NC - 1) / tc::NC;
 }
 
-static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) + 4 * 256 + 16 : 0; }   // node bits per entry, cleared by words (+ the padding words)
+static size_t plan_smem_bytes(const TvaPlan& p) { return p.need_scores ? (((size_t)p.cand_cap + 3) & ~(size_t)3) + 4 * 1024 + 16 : 0; }   // node bits per entry, cleared by words (+ the padding words)
 // Can the plan kernel produce a gathered tile for these capacities?  (A committed CSA run longer than twice the
 // selection size, or a paged pool whose pages do not hold whole 32-row boxes of a layer.)
 static bool gathered_tiles_possible(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c) {
@@ -412,13 +414,15 @@ static bool gathered_tiles_possible(const tsv_shape& s, const TvaPlan& p, const 
 // Host-side work of the tensor-core path that can fail, before anything of the call is enqueued.
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep) {
   const size_t plan_sm = plan_smem_bytes(p);
-  if (plan_sm > 32 * 1024 && (cudaFuncSetAttribute(tc_plan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess ||
-                              cudaFuncSetAttribute(tc_plan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)) {
+  if (plan_sm > 32 * 1024 && (cudaFuncSetAttribute(tc_plan_kernel<true, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess ||
+                              cudaFuncSetAttribute(tc_plan_kernel<true, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess ||
+                              cudaFuncSetAttribute(tc_plan_kernel<false, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_sm) != cudaSuccess)) {
     cudaGetLastError();
     return TSV_ERR_CUDA;
   }
-  TSV_PREP(tc_plan_kernel<true>);
-  TSV_PREP(tc_plan_kernel<false>);
+  TSV_PREP((tc_plan_kernel<true, 1024>));
+  TSV_PREP((tc_plan_kernel<true, 256>));
+  TSV_PREP((tc_plan_kernel<false, 256>));
   TSV_PREP(tc_combine_pair_kernel);
   return prepare_tva_tc_pair(s, p, c, nd, out, ws, prep);
 }
@@ -429,13 +433,15 @@ int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, c
   const dim3 pgrid(p.tc_nt + 1, s.B);                                                                              // x: tiles + the packing CTA
   {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = pgrid; cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = plan_smem_bytes(p); cfg.stream = st;
+    const bool wide = gathered && p.cand_cap > 8192;    // long candidate lists: the CTA's passes over all entries want many threads
+    cfg.gridDim = pgrid; cfg.blockDim = dim3(wide ? 1024 : 256, 1, 1); cfg.dynamicSmemBytes = plan_smem_bytes(p); cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;        // may start under the selection kernel's tail (it waits inside)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (gathered) cudaLaunchKernelEx(&cfg, tc_plan_kernel<true>, s, p, c, nd, sc, ws);
-    else cudaLaunchKernelEx(&cfg, tc_plan_kernel<false>, s, p, c, nd, sc, ws);
+    if (wide) cudaLaunchKernelEx(&cfg, tc_plan_kernel<true, 1024>, s, p, c, nd, sc, ws);
+    else if (gathered) cudaLaunchKernelEx(&cfg, tc_plan_kernel<true, 256>, s, p, c, nd, sc, ws);
+    else cudaLaunchKernelEx(&cfg, tc_plan_kernel<false, 256>, s, p, c, nd, sc, ws);
   }
   count_launch();
   // general: some tile may have more than two chunks of the longest kind, or be gathered; then every multi-chunk tile
