@@ -242,10 +242,13 @@ def run_ours(args, cfg):
                 elif name == "attention":
                     tsv.bench_tree_verify_attn_stages(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None,
                                                       eng.workspace, eng.status, tsv.STAGE_ATTENTION)
+                elif name == "attention_kernels":    # the stage without its tile plan (the plan of the call before is used again)
+                    tsv.bench_tree_verify_attn_stages(eng.cshape, eng.caches[l], inp0.layers[l], eng.scratch[l], eng.out[l], None,
+                                                      eng.workspace, eng.status, tsv.STAGE_ATTENTION_KERNELS)
         return f
 
     t_parts = {}
-    for name in ("branch_state_build", "select", "attention"):
+    for name in ("branch_state_build", "select", "attention", "attention_kernels"):
         sg = torch.cuda.Stream(); sg.wait_stream(stream)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=sg):
@@ -267,6 +270,7 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     t_parts["accept_and_refresh"] = a0.elapsed_time(a1)
     attn_ms = float(t_parts["attention"])
+    kern_ms = float(t_parts["attention_kernels"])
 
     # ---- algorithmic work and roofline of the dominant kernel (attention)
     parents = wl.inputs[0].layers[0].parent.cpu().numpy()
@@ -289,7 +293,11 @@ def run_ours(args, cfg):
                 **(tensor if bound == "tensor" else hbm),
                 "traffic": cap["launch_bytes"] if cap else None,
                 "traffic_note": (f"ncu DRAM read+write of one {cap['kernel']} launch on this workload" if cap else "no ncu capture for this workload"),
-                "peak_source": pk["source"], "launch_ms": attn_ms, "flop_per_byte": intensity, "ridge_flop_per_byte": ridge,
+                "peak_source": pk["source"], "launch_ms": attn_ms,
+                # the same work over the duration of the attention kernels alone (without the tile plan's kernel)
+                "kernels_only": {"launch_ms": kern_ms, "frac_hbm": attn_gbs * attn_ms / kern_ms / pk["hbm_gbs"],
+                                 "frac_tensor": attn_tf * attn_ms / kern_ms / pk["bf16_tflops_sustained"]},
+                "flop_per_byte": intensity, "ridge_flop_per_byte": ridge,
                 "lengths": "algorithmic bytes and FLOPs from the initial prefix lengths (the caches grow by the accepted tokens while timed)",
                 "hbm": hbm, "tensor": tensor}
     cycle_s = sec / K

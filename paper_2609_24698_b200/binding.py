@@ -25,7 +25,7 @@ _lib = C.CDLL(LIB_PATH)
 
 TSV_FP32, TSV_BF16 = 0, 1
 FLAG_FORCE_SIMT, FLAG_HCA_DEFERRED = 1, 2
-STAGE_SELECT, STAGE_ATTENTION = 1, 2      # stages of tree_verify_attn for bench_tree_verify_attn_stages
+STAGE_SELECT, STAGE_ATTENTION, STAGE_ATTENTION_KERNELS = 1, 2, 4    # stages of tree_verify_attn for bench_tree_verify_attn_stages (4: without the tile plan)
 ST_NODES, ST_PARENT, ST_LENGTH, ST_CSA_CAP, ST_HCA_CAP, ST_INTERNAL = 1, 2, 4, 8, 16, 32
 ERR_NULL, ERR_ALIGN, ERR_SHAPE, ERR_WORKSPACE, ERR_CUDA, ERR_LIMIT = -1, -2, -3, -4, -5, -6
 

@@ -123,10 +123,10 @@ static int tva_stages(const tsv_shape& s, const TvaPlan& p_in, const tsv_cache& 
   TvaTcPrep prep;
   TvaPlan p = p_in;
   if (p.tc && !tva_tc_pair_usable(c)) p.tc = 0;       // no row counts for the tensor maps: the CUDA-core path (same workspace)
-  if (p.tc && (stages & 2) && (r = prepare_tva_tc(s, p, c, nd, out, ws, prep))) return r;
+  if (p.tc && (stages & 6) && (r = prepare_tva_tc(s, p, c, nd, out, ws, prep))) return r;
   if ((stages & 1) && (r = launch_tva_select(s, p, c, nd, sc, topk_idx, ws, status, st))) return r;
-  if (!(stages & 2)) return TSV_OK;
-  if (p.tc) return launch_tva_tc(s, p, prep, c, nd, sc, out, ws, status, st);
+  if (!(stages & 6)) return TSV_OK;
+  if (p.tc) return launch_tva_tc(s, p, prep, c, nd, sc, out, ws, status, st, (stages & 2) != 0);
   return launch_tva_simt(s, p, c, nd, sc, out, ws, status, st);
 }
 
@@ -184,7 +184,9 @@ int tree_verify_attn(const tsv_shape* shape, const tsv_cache* cache, const tsv_n
 }
 
 // Not part of the public interface (not declared in tsv.h): tree_verify_attn restricted to some of its stages, for
-// per-stage timing by the benchmark.  stages: bit 0 = CSA selection, bit 1 = attention (tile plan + attention kernels).
+// per-stage timing by the benchmark.  stages: bit 0 = CSA selection, bit 1 = attention (tile plan + attention kernels),
+// bit 2 = the attention kernels WITHOUT the tile plan (tensor-core path: the plan a previous call left is used again; the
+// finished-chunk counters of two-chunk tiles are not reset, so only timings of such a call mean anything).
 // The attention stage alone reuses the selection a previous full call on the same inputs left in `workspace`.
 int tsv_bench_tree_verify_attn_stages(const tsv_shape* shape, const tsv_cache* cache, const tsv_nodes* nodes, const tsv_scratch* scratch,
                                       void* out, int32_t* topk_idx, void* workspace, size_t workspace_bytes, int32_t* status, void* stream,
@@ -198,7 +200,7 @@ int tsv_bench_tree_verify_attn_stages(const tsv_shape* shape, const tsv_cache* c
   TvaPlan p;
   make_tva_plan(s, p);
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < p.total) return TSV_ERR_WORKSPACE;
-  return tva_stages(s, p, *cache, *nodes, *scratch, out, topk_idx, (char*)workspace, status, (cudaStream_t)stream, stages & 3);
+  return tva_stages(s, p, *cache, *nodes, *scratch, out, topk_idx, (char*)workspace, status, (cudaStream_t)stream, stages & 7);
 }
 
 int accept_and_refresh(const tsv_shape* shape, int32_t n_layers, const tsv_cache* const* caches, const tsv_nodes* const* nodes,

