@@ -146,7 +146,8 @@ typedef struct tsv_cache {
    * pages can hold, and the pages must cover positions up to L + D - 1.  page_tokens must be a multiple of m_csa and of
    * m_hca.  The tensor-core path fetches rows by 32-row TMA boxes where a page holds whole boxes of the layer (CSA: epp a
    * multiple of 32, e.g. 128-token pages with m_csa = 4: one box per page; window: page_tokens a multiple of 32); otherwise,
-   * and for HCA rows beyond the first 32 entries unless hpp is a multiple of 32, it gathers rows by pointer. */
+   * and for HCA rows beyond the first 32 entries unless hpp is a multiple of 32, it gathers the rows four at a time by
+   * index. */
   const int32_t *page_table;  /* [B][max_pages] device, or NULL: flat slabs and window ring   */
   int32_t page_tokens;        /* HOST value                                                 */
   int32_t max_pages;          /* HOST value: columns of page_table                          */
