@@ -57,7 +57,7 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
   p.off_pml = off;    if (p.nsplit > 1) off = up256(off + (size_t)s.B * s.D * s.H * p.nsplit * 2 * sizeof(float));
   p.tc = tva_tc_eligible(s);
   p.tc_nt = p.tc_maxk = p.tc_chmax = p.tc_misc_rows = 0;
-  p.off_krow = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = p.off_order = p.off_tcnt = p.off_pos = off;
+  p.off_krow = p.off_kmask = p.off_nkeys = p.off_tpo = p.off_tpml = p.off_box = p.off_mode = p.off_misc = p.off_order = p.off_tcnt = off;
   p.off_selmask = off;
   p.mask_ld = (p.cand_cap + 15) & ~15;
   if (p.tc) {
@@ -73,7 +73,6 @@ bool make_tva_plan(const tsv_shape& s, TvaPlan& p) {
     p.off_misc = off;  off = up256(off + (size_t)s.B * p.tc_misc_rows * s.d * 2);
     p.off_order = off; off = up256(off + tiles * 4 * sizeof(int32_t));
     p.off_tcnt = off;  off = up256(off + 2 * tiles * sizeof(int32_t));     // finished chunks per 128-row tile (paired kernel)
-    p.off_pos = off;   off = up256(off + tiles * sizeof(int32_t));         // scheduling position of each tile (selection kernel)
     p.off_selmask = off; if (p.need_scores) off = up256(off + (size_t)s.B * s.D * p.mask_ld);
   }
   p.total = off;

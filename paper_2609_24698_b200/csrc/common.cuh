@@ -166,6 +166,11 @@ __device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, cons
   __syncthreads();
 }
 
+// Does the node at depth `depth` of a sequence of committed length L close a block of m tokens?  (What the state build
+// writes into its done flags for a valid node: a function of the position alone, so kernels that run under the state
+// build's tail work it out instead of reading the flag.)
+__device__ __forceinline__ bool node_closes(int L, int depth, int m) { return ((L + depth + 1) % m) == 0; }
+
 // C128-deferred schedule: no node of this sequence can close an HCA block (a node at depth delta closes one iff
 // (L + delta + 1) % m_hca == 0, and delta <= D - 1), so its HCA branch states are not built and the accepted path is
 // folded into the persistent state at commit time.

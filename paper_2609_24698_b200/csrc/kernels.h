@@ -46,7 +46,7 @@ struct TvaPlan {
   // tensor-core path (bf16, d = 512): row tiles per sequence, key-list capacity per tile, max chunks per tile
   int32_t tc, tc_nt, tc_maxk, tc_chmax;
   int32_t tc_misc_rows;              // rows of the per-sequence packed buffer
-  size_t off_krow, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt, off_pos;
+  size_t off_krow, off_kmask, off_nkeys, off_tpo, off_tpml, off_box, off_mode, off_misc, off_order, off_tcnt;
   // selection as a byte per candidate (1 = selected), one row of mask_ld bytes per node, written for the nodes that rank:
   // the tile plan combines the rows of a tile's nodes into its per-key node masks
   size_t off_selmask;

@@ -179,11 +179,6 @@ __global__ void __launch_bounds__(256) topk_kernel(const tsv_shape s, const TvaP
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile plan may start its selection-independent part
-  if (blockIdx.x == (unsigned)s.D) {
-    // extra CTA column (only with the tensor-core attention path): CTA (D, 0) ranks the attention tiles
-    if (blockIdx.y == 0) rank_tiles(s, pl, c, nd, sc, ws);
-    return;
-  }
   const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk;
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
@@ -572,7 +567,7 @@ int launch_tva_select(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   }
   if (topk_long_applies(s, p)) return launch_topk_long(s, p, c, nd, sc, topk_idx, ws, status, st);
   if (topk_fused_applies(s, p)) return launch_topk_fused(s, p, c, nd, sc, topk_idx, ws, status, st);
-  dim3 g2(s.D + (p.tc ? 1 : 0), s.B);                                  // + the column that ranks the attention tiles
+  dim3 g2(s.D, s.B);
   const bool paged = c.page_table != nullptr;
   size_t sm2 = p.idx_fused ? (size_t)s.HI * s.di * sizeof(float) : 0;         // the node's indexer queries ...
   if (p.idx_fused && (size_t)s.di * (bf ? 2 : 4) == 256 && s.HI <= 4) sm2 += (size_t)2 * kStageRows * kStagePitch + (size_t)kIdxFusedMax * sizeof(float);   // ... the staged rows (two buffers), the scores

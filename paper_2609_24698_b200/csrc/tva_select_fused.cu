@@ -53,19 +53,25 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   unsigned char* stage = dsm + 4 * DI * 2 + (size_t)score_cap * 4;
   const int t = threadIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile plan may start its selection-independent part
-  if (blockIdx.x == (unsigned)s.D) {                  // extra CTA column (tensor-core attention path): CTA (D, 0) ranks the attention tiles
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // (the ranking reads the state build's done flags)
-    if (blockIdx.y == 0) rank_tiles_in(reinterpret_cast<int32_t*>(stage), s, pl, c, nd, sc, ws);
-    return;
-  }
   const int n = blockIdx.x, b = blockIdx.y, D = s.D, k = s.topk, HI = s.HI;
+  const bool anchor = blockIdx.x == 0 && blockIdx.y == 0;
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
+  // The tensor-core attention path reads mask rows of ranking nodes only, never the index lists: when the caller does not
+  // ask for the lists either, the CTA of a node that cannot rank (the sequence's committed entries plus one per node
+  // of the tree stay within k) has nothing to do.  One load decides it; node 0 of every sequence still goes on, to
+  // validate the sequence's inputs.  (A CTA takes up the registers of a ranking one while it lives, and the plan kernel
+  // starts when the last CTA of this kernel has: the sooner it leaves the better.)
+  if (pl.tc && !topk_user && n != 0) {
+    const int L0 = c.L[b];
+    if (L0 >= 0 && L0 / s.m_csa + D <= k) return;
+  }
   // Everything the CTA may need that depends on (b, n) alone is requested together with the tree's loads (one memory
   // latency for all): the slab offset and -- used only if the node ranks -- its indexer queries and head weights.  The
-  // kernel is launched as a programmatic dependent of the state build: up to the wait below it reads nothing that kernel
-  // writes (the done flags follow the wait).
+  // kernel is launched as a programmatic dependent of the state build and reads nothing that kernel writes until a node
+  // that ranks scores the entries closed inside the tree (the done flags are worked out from the positions).  A CTA that
+  // does not rank leaves without waiting, except CTA (0, 0): through it this kernel's completion implies that one's.
   if (!PAGED && t == 64) row0_sm = c.csa_row0[b];
   const int lane = t & 31, w = t >> 5, g = lane >> 2, tq = lane & 3;
   const bf16* iq = reinterpret_cast<const bf16*>(nd.iq) + ((size_t)b * D + n) * HI * DI;
@@ -96,9 +102,11 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
   if (may_rank) issue(0);
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (t >= 96 && t < 96 + D) cdone_sm[t - 96] = sc.csa_done[(size_t)b * D + t - 96];
-  if (t >= 128 && t < 128 + D) hdone_sm[t - 128] = sc.hca_done[(size_t)b * D + t - 128];
+  if (t < D) {                                         // the done flags of the sequence's nodes, from their positions
+    const bool valid = !tm.status && t < tm.nn;
+    cdone_sm[t] = valid && node_closes(tm.L, tm.depth[t], s.m_csa);
+    hdone_sm[t] = valid && node_closes(tm.L, tm.depth[t], s.m_hca);
+  }
   __syncthreads();
   if (t == 0) {
     if (tm.status && n == 0) atomicOr(status + b, tm.status);
@@ -108,6 +116,7 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   if (!live) {
     for (int i = t; i < k; i += 256) { sel[i] = -1; if (usr) usr[i] = -1; }
     if (t == 0) *selcnt = 0;
+    if (anchor) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
   const int n_cand = n_csa + pe.n_newc;
@@ -118,22 +127,11 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     }
     if (t == 0) *selcnt = n_cand;
     if (may_rank) asm volatile("cp.async.wait_group 0;" ::: "memory");     // (requested in vain: the bound was not reached)
+    if (anchor) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
   // ---------------------------------------------------------------------------------------------- the node ranks
   if (nrd > 1) issue(1); else asm volatile("cp.async.commit_group;" ::: "memory");
-  // scores of the in-tree entries on this node's path: warp w takes entries w, w + 8, ...
-  for (int i = w; i < pe.n_newc; i += 8) {
-    const bf16* ik = reinterpret_cast<const bf16*>(sc.new_csa_ik) + ((size_t)b * D + pe.newc[i]) * DI;
-    float tot = 0.f;
-    for (int h = 0; h < HI; ++h) {
-      float p = 0.f;
-      for (int x = lane; x < DI; x += 32) p = fmaf(to_f(iq[h * DI + x]), to_f(ik[x]), p);
-      p = warp_sum(p);
-      tot = fmaf(iwp[h], fmaxf(p, 0.f), tot);
-    }
-    if (lane == 0) extra[i] = tot;
-  }
   if (t < 128) hist[0][t] = 0;
   // B fragments of the eight k-steps: column g = head g (zero beyond HI), k = 16 ks + 2 tq (+ 8)
   uint32_t bq[8][2];
@@ -174,7 +172,21 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     if (rd + 2 < nrd) issue(rd + 2); else asm volatile("cp.async.commit_group;" ::: "memory");
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
-  if (nrd == 0) __syncthreads();                       // (the in-tree entries' scores, the cleared histogram)
+  // Scores of the in-tree entries on this node's path: the state build's results, the first thing of that kernel this
+  // CTA reads (all of the committed entries' scoring above may run under its tail).  Warp w takes entries w, w + 8, ...
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  for (int i = w; i < pe.n_newc; i += 8) {
+    const bf16* ik = reinterpret_cast<const bf16*>(sc.new_csa_ik) + ((size_t)b * D + pe.newc[i]) * DI;
+    float tot = 0.f;
+    for (int h = 0; h < HI; ++h) {
+      float p = 0.f;
+      for (int x = lane; x < DI; x += 32) p = fmaf(to_f(iqs[h * DI + x]), to_f(ik[x]), p);
+      p = warp_sum(p);
+      tot = fmaf(iwp[h], fmaxf(p, 0.f), tot);
+    }
+    if (lane == 0) extra[i] = tot;
+  }
+  __syncthreads();                                     // (the in-tree entries' scores, the cleared histogram)
   // order-preserving keys: candidate t + 256 j is key j of thread t (all warps take part in every pass)
   uint32_t key[KPT];
   const int nj = (n_cand + 255) >> 8;
@@ -286,7 +298,7 @@ int launch_topk_fused(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   int rows, score_cap;
   size_t bytes;
   fused_smem(p, rows, score_cap, bytes);
-  const dim3 grid(s.D + (p.tc ? 1 : 0), s.B);           // + the column that ranks the attention tiles
+  const dim3 grid(s.D, s.B);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = bytes; cfg.stream = st;
   cudaLaunchAttribute attr[1];

@@ -44,10 +44,6 @@ __global__ void __launch_bounds__(lsel::THREADS) topk_long_kernel(const tsv_shap
   const int n = blockIdx.x / CS, b = blockIdx.y, D = s.D, k = s.topk;
   // every exit below is taken by all CTAs of a cluster alike (it depends on the node's facts only); after the last
   // cluster barrier no CTA touches a peer's memory, so they leave independently
-  if (n == D) {                          // extra cluster (only with the tensor-core attention path): one CTA ranks the attention tiles
-    if (rank == 0 && b == 0) rank_tiles(s, pl, c, nd, sc, ws);
-    return;
-  }
   int32_t* sel = reinterpret_cast<int32_t*>(ws + pl.off_sel) + ((size_t)b * D + n) * k;
   int32_t* selcnt = reinterpret_cast<int32_t*>(ws + pl.off_selcnt) + (size_t)b * D + n;
   int32_t* usr = topk_user ? topk_user + ((size_t)b * D + n) * k : nullptr;
@@ -215,7 +211,7 @@ bool topk_long_applies(const tsv_shape&, const TvaPlan& p) {
 int launch_topk_long(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, const tsv_nodes& nd, const tsv_scratch& sc,
                      int32_t* topk_idx, char* ws, int32_t* status, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((s.D + (p.tc ? 1 : 0)) * lsel::CS), (unsigned)s.B, 1);   // + the cluster that ranks the attention tiles
+  cfg.gridDim = dim3((unsigned)(s.D * lsel::CS), (unsigned)s.B, 1);
   cfg.blockDim = dim3(lsel::THREADS, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = st;

@@ -11,8 +11,8 @@
 //                    rows): the runs as 32-row TMA boxes.  Gathered tiles (selection far from dense, or a paged pool
 //                    whose pages do not hold whole boxes): the first run holds only the entries some node of the tile
 //                    selected, and every key is named by array << 30 | row for four-row TMA gathers.
-//                    Each tile CTA leaves its record {tile, mode, keys} at the scheduling position the selection kernel
-//                    computed (most keys first); an extra CTA per sequence packs the small scattered rows.
+//                    Each tile CTA leaves its record {tile, mode, keys} at the tile's scheduling position (its rank by
+//                    estimated key count, most first); an extra CTA per sequence packs the small scattered rows.
 //   tc_combine_pair_kernel  merges the chunks of the paired kernel's multi-chunk tiles (fixed order).
 #include "tc_common.cuh"
 
@@ -24,7 +24,7 @@ namespace tsv {
 // latency chain of the contiguous-run plan.
 template <bool GENERAL>
 __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
-                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask, int& pos) {
+                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
   __shared__ int n_cand[8], win_lo[8];
@@ -41,12 +41,16 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   if (threadIdx.x == 40) row0_sm[0] = c.page_table ? 0 : c.csa_row0[b];
   if (threadIdx.x == 41) row0_sm[1] = c.page_table ? 0 : c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
-  // The kernel is launched as a programmatic dependent of the selection kernel (itself one of the state build): up to here
-  // it has read only what the caller's inputs and the committed caches hold, under those kernels' tails.  What follows
-  // reads their results: the state build's done flags and entries, the selection's scheduling positions and mask rows.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (threadIdx.x >= 64 && threadIdx.x < 64 + D) cdone[threadIdx.x - 64] = sc.csa_done[(size_t)b * D + threadIdx.x - 64];
-  if (threadIdx.x >= 96 && threadIdx.x < 96 + D) hdone[threadIdx.x - 96] = sc.hca_done[(size_t)b * D + threadIdx.x - 96];
+  // The kernel is launched as a programmatic dependent of the selection kernel (itself one of the state build) and runs
+  // under those kernels' tails as far as it reads only the caller's inputs and the committed caches: the done flags are
+  // worked out from the positions, and a tile no node of which ranks is planned completely.  It waits for the two kernels
+  // (griddepcontrol.wait, below) before it reads what they write: the entries closed inside the tree (packing CTA), the
+  // ranking nodes' mask rows.
+  if (threadIdx.x < D) {
+    const bool valid = !tm.status && (int)threadIdx.x < tm.nn;
+    cdone[threadIdx.x] = valid && node_closes(tm.L, tm.depth[threadIdx.x], s.m_csa);
+    hdone[threadIdx.x] = valid && node_closes(tm.L, tm.depth[threadIdx.x], s.m_hca);
+  }
   __syncthreads();
   // rows of the sequence's CSA and HCA entries: slabs, or through the page table of a paged pool
   RowAddr csa_row, hca_row;
@@ -85,28 +89,33 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       }
       return reinterpret_cast<const uint4*>(src);
     };
-    if (cpr == 64) {                                   // d = 512 in bf16: two 16-byte pieces of a row per lane
-      for (int r0 = w; r0 < rows_out; r0 += 8 * nw) {
-        uint4 v[8][2];
+    auto copy_rows = [&](int lo, int hi) {             // rows [lo, hi) of the packed buffer
+      if (cpr == 64) {                                 // d = 512 in bf16: two 16-byte pieces of a row per lane
+        for (int r0 = lo + w; r0 < hi; r0 += 8 * nw) {
+          uint4 v[8][2];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int r = r0 + k * nw;
-          const uint4* src = r < rows_out ? row_src(r) : nullptr;
-          v[k][0] = src ? __ldg(src + lane) : make_uint4(0, 0, 0, 0);
-          v[k][1] = src ? __ldg(src + 32 + lane) : make_uint4(0, 0, 0, 0);
+          for (int k = 0; k < 8; ++k) {
+            const int r = r0 + k * nw;
+            const uint4* src = r < hi ? row_src(r) : nullptr;
+            v[k][0] = src ? __ldg(src + lane) : make_uint4(0, 0, 0, 0);
+            v[k][1] = src ? __ldg(src + 32 + lane) : make_uint4(0, 0, 0, 0);
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int r = r0 + k * nw;
+            if (r < hi) { dst[(size_t)r * 64 + lane] = v[k][0]; dst[(size_t)r * 64 + 32 + lane] = v[k][1]; }
+          }
         }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int r = r0 + k * nw;
-          if (r < rows_out) { dst[(size_t)r * 64 + lane] = v[k][0]; dst[(size_t)r * 64 + 32 + lane] = v[k][1]; }
+      } else {
+        for (int r = lo + w; r < hi; r += nw) {
+          const uint4* src = row_src(r);
+          for (int cc = lane; cc < cpr; cc += 32) dst[(size_t)r * cpr + cc] = src ? src[cc] : make_uint4(0, 0, 0, 0);
         }
       }
-    } else {
-      for (int r = w; r < rows_out; r += nw) {
-        const uint4* src = row_src(r);
-        for (int cc = lane; cc < cpr; cc += 32) dst[(size_t)r * cpr + cc] = src ? src[cc] : make_uint4(0, 0, 0, 0);
-      }
-    }
+    };
+    copy_rows(0, nh_in + tm.nn);                       // committed HCA entries and the tree nodes' rows: the caller's data
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    copy_rows(nh_in + tm.nn, rows_out);                // the entries closed inside the tree (the state build's), the zero padding
     return;
   }
   if (threadIdx.x < 32) {                              // lane nl: candidates and window start of node n0 + nl
@@ -122,7 +131,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     if (lane == 0) dense = over == 0;
   }
   __syncthreads();
-  if (threadIdx.x == 0) pos = reinterpret_cast<const int32_t*>(ws + pl.off_pos)[tix];   // fetched now, used at the end (when the attention stage runs alone: the previous call's)
   int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
   if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = 1; } return; }
   const int nvalid = min(npt, tm.nn - n0);
@@ -140,10 +148,15 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   int psh = 3;                                         // log2(per)
   if (GENERAL) while (((int)blockDim.x << psh) < n_csa) ++psh;
   auto phys = [&](int i) { return GENERAL ? i + ((i >> psh) << 2) : i; };
-  if (!dense) {
-    uint32_t allbits = 0, rankbits = 0;                // nodes that take every committed entry / nodes that rank
-    for (int nl = 0; nl < nvalid; ++nl) { if (n_cand[nl] <= s.topk) allbits |= 1u << nl; else rankbits |= 1u << nl; }
-    const uint8_t* mrow = reinterpret_cast<const uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n0) * pl.mask_ld;
+  // Contiguous-run tiles with ranking nodes (`late`): everything that does not depend on the selection -- boxes, the masks of
+  // the HCA, window and packed runs -- is written before the wait; after it only the masks of the committed CSA run (the
+  // combined mask rows, stored straight into the key masks) and of the entries closed inside the tree.
+  const bool runs_ok = !GENERAL || ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax));
+  const bool late = !dense && runs_ok;
+  uint32_t allbits = 0, rankbits = 0;                  // nodes that take every committed entry / nodes that rank
+  for (int nl = 0; nl < nvalid; ++nl) { if (n_cand[nl] <= s.topk) allbits |= 1u << nl; else rankbits |= 1u << nl; }
+  const uint8_t* mrow = reinterpret_cast<const uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n0) * pl.mask_ld;
+  auto fetch_newc_bits = [&]() {                       // (threads 0..7; the caller synchronises)
     if (threadIdx.x < 8) {
       // in-tree entries: candidate n_csa + o of a node is the block closed at the o-th of its strict ancestors that closed one
       uint32_t bits = 0;
@@ -159,19 +172,28 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
       }
       newc_bits[nl] = bits;
     }
-    uint32_t* cm32 = reinterpret_cast<uint32_t*>(cmask);
+  };
+  // sixteen committed entries from entry i: the node bits of each as four words of four mask bytes
+  auto combine16 = [&](int i, uint32_t acc[4]) {
     const uint32_t all4 = 0x01010101u * allbits;
+    acc[0] = acc[1] = acc[2] = acc[3] = all4;
+#pragma unroll
+    for (int nl = 0; nl < 8; ++nl) {
+      if ((rankbits >> nl) & 1u) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(mrow + (size_t)nl * pl.mask_ld + i));
+        acc[0] |= (v.x & 0x01010101u) << nl; acc[1] |= (v.y & 0x01010101u) << nl;
+        acc[2] |= (v.z & 0x01010101u) << nl; acc[3] |= (v.w & 0x01010101u) << nl;
+      }
+    }
+  };
+  if (!dense && !runs_ok) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the selection's mask rows
+    fetch_newc_bits();
+    uint32_t* cm32 = reinterpret_cast<uint32_t*>(cmask);
 #pragma unroll 2
     for (int i = 16 * threadIdx.x; i < n_csa; i += 16 * blockDim.x) {
-      uint32_t acc[4] = {all4, all4, all4, all4};
-#pragma unroll
-      for (int nl = 0; nl < 8; ++nl) {
-        if ((rankbits >> nl) & 1u) {
-          const uint4 v = __ldcg(reinterpret_cast<const uint4*>(mrow + (size_t)nl * pl.mask_ld + i));
-          acc[0] |= (v.x & 0x01010101u) << nl; acc[1] |= (v.y & 0x01010101u) << nl;
-          acc[2] |= (v.z & 0x01010101u) << nl; acc[3] |= (v.w & 0x01010101u) << nl;
-        }
-      }
+      uint32_t acc[4];
+      combine16(i, acc);
 #pragma unroll
       for (int q = 0; q < 4; ++q) cm32[phys(i + 4 * q) >> 2] = acc[q];      // (bytes past n_csa are never read)
     }
@@ -193,7 +215,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     // entries are staged and the unselected ones are masked per node.  Beyond that (or where a paged pool's pages do not
     // hold whole boxes) the tile is GATHERED: the same four runs, but the first holds only the committed entries some node
     // of the tile selected, and every key is named by its row (array << 30 | row) for four-row TMA gathers.
-    const bool runs_ok = !GENERAL || ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax));
     int n_uni = n_csa;                                 // keys of the first run
     __shared__ int uni_tot;
     if (!runs_ok) {
@@ -258,8 +279,9 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
         const int i = k - k0[g];
         uint32_t m = 0;
+        if (late && (g == 0 || (g == 3 && i >= nh_in + tm.nn && i < nh_in + tm.nn + ncd))) continue;   // after the wait, below
         if (i < cnt[g]) {
-          if (g == 0) m = dense ? validbits : cmask[phys(i)];       // (contiguous-run tiles only: see the loop's start)
+          if (g == 0) m = validbits;                                 // (dense contiguous-run tiles only: see the loop's start and the line above)
           else if (g == 1) m = validbits;
           else if (g == 2) {
             const int pos = c.page_table ? win_a + i : tm.L - 1 - ((tm.L - 1 - i) % s.window);
@@ -284,31 +306,92 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         if (!runs_ok) krow[k] = ((uint32_t)g << 30) | (uint32_t)(cnt[g] ? run_row(g, i < cnt[g] ? i : 0) : 0);
       }
       if (threadIdx.x == 0) { *nkeys = kb; *mode = runs_ok ? 1 : 2; }
+      if (late) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the selection's mask rows
+        fetch_newc_bits();
+        // the committed CSA run (its first key is key 0 of the tile): sixteen key masks per store; the run's padding is zero
+        uint4* km4 = reinterpret_cast<uint4*>(kmask);
+        for (int i = 16 * threadIdx.x; i < k0[1]; i += 16 * blockDim.x) {
+          uint32_t acc[4] = {0u, 0u, 0u, 0u};
+          if (i < n_csa) combine16(i, acc);             // (a mask row holds a multiple of 16 bytes that covers n_csa)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int left = n_csa - (i + 4 * q);
+            if (left < 4) acc[q] = left <= 0 ? 0u : acc[q] & ((1u << (8 * left)) - 1u);
+          }
+          km4[i >> 4] = make_uint4(acc[0], acc[1], acc[2], acc[3]);
+        }
+        __syncthreads();
+        // the CSA entries closed inside the tree (ncd keys of the packed run)
+        if ((int)threadIdx.x < ncd) {
+          int ord = threadIdx.x, a = 0;
+          for (int j = 0; j < tm.nn; ++j) if (cdone[j]) { if (ord == 0) { a = j; break; } --ord; }
+          uint32_t m = 0;
+          for (int nl = 0; nl < nvalid; ++nl)
+            if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && newc_selected(nl, a)) m |= 1u << nl;
+          kmask[k0[3] + nh_in + tm.nn + threadIdx.x] = (uint8_t)m;
+        }
+      }
       return;
     }
   }
 }
 
-// Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the scheduling
-// position the selection kernel computed for it (most keys first): the paired attention kernel takes the tiles in that
-// order and learns all it needs about its tile from one load.
+// Estimated number of keys a tile of a sequence stages, from its committed length and node count alone (for tiles on the
+// contiguous-run path it is exact up to the entries closed inside the tree; only the order of the tiles depends on it).
+__device__ __forceinline__ int tile_keys_estimate(const tsv_shape& s, int L, int nn, int tile, int npt) {
+  if (L < 0 || (int64_t)L + s.D > s.max_L || nn < 1 || nn > s.D || tile * npt >= nn) return 0;
+  auto r32 = [](int x) { return (x + kBoxRows - 1) / kBoxRows * kBoxRows; };
+  const int n_csa = L / s.m_csa, n_hca = L / s.m_hca, nh_in = n_hca <= kHcaMiscMax ? n_hca : 0, win = min(L, s.window);
+  if (n_csa <= 2 * s.topk) return r32(n_csa) + (n_hca > kHcaMiscMax ? r32(n_hca) : 0) + r32(win) + r32(nh_in + nn);
+  return min(n_csa, npt * s.topk) + n_hca + win + 3 * nn;
+}
+
+// Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the tile's
+// scheduling position: its rank among all tiles by estimated key count, most first, which every CTA works out for itself
+// from the lengths and node counts of all sequences (the paired attention kernel takes the tiles in that order, long
+// ones first and short ones in the tail, and learns all it needs about its tile from one load).  A tile no node of which
+// ranks is planned from the caller's inputs alone: its CTA never waits for the kernels before this one.
 // NT threads per CTA: 256, or 1024 for gathered tiles over long candidate lists (the union of a tile's selections over tens
 // of thousands of entries is the work of ONE CTA, alone on its SM).
+constexpr int kRankTilesMax = 2048;                    // beyond that many tiles they keep their natural order
 template <bool GENERAL, int NT>
 __global__ void __launch_bounds__(NT) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
-                                                      const tsv_scratch sc, char* __restrict__ ws) {
+                                                                         const tsv_scratch sc, char* __restrict__ ws) {
   extern __shared__ uint8_t cmask_sm[];                // [cand_cap] node bits per committed CSA entry (ranked case only)
+  __shared__ int est_sm[kRankTilesMax];
+  __shared__ int ahead_sm;
   const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
+  const int ntile = s.B * pl.tc_nt, npt = tc::PR / s.H;
   const size_t tix = (size_t)blockIdx.y * pl.tc_nt + blockIdx.x;
-  int pos = (int)tix;
+  if (tile_cta && ntile <= kRankTilesMax) {            // requested with the tile's own first loads
+    for (int i = threadIdx.x; i < ntile; i += NT) {
+      const int b = i / pl.tc_nt;
+      est_sm[i] = tile_keys_estimate(s, c.L[b], nd.n_nodes[b], i - b * pl.tc_nt, npt);
+    }
+  }
+  if (threadIdx.x == 0) ahead_sm = 0;
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
-  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm, pos);
-  if (tile_cta && threadIdx.x == 0) {                 // thread 0 wrote the tile's key count and mode itself
-    if (pos < 0 || pos >= s.B * pl.tc_nt) pos = (int)tix;
-    reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
-        make_int4((int)tix, reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix], reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix], 0);
+  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm);
+  if (tile_cta) {                                      // (barriers since the estimates were written)
+    int pos = (int)tix;
+    if (ntile <= kRankTilesMax) {
+      const int mine = est_sm[tix];
+      int ahead = 0;
+      for (int j = threadIdx.x; j < ntile; j += NT) { const int e = est_sm[j]; ahead += (e > mine) || (e == mine && j < (int)tix); }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
+      if ((threadIdx.x & 31) == 0 && ahead) atomicAdd(&ahead_sm, ahead);
+      __syncthreads();
+      pos = ahead_sm;
+    }
+    if (threadIdx.x == 0)                              // thread 0 wrote the tile's key count and mode itself
+      reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
+          make_int4((int)tix, reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix], reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix], 0);
   }
+  // one CTA waits for the selection in any case, so that the completion of this kernel implies that one's
+  if (blockIdx.x == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------------------ merge
