@@ -276,8 +276,11 @@ def run_ours(args, cfg):
     parents = wl.inputs[0].layers[0].parent.cpu().numpy()
     work = W.algorithmic_work(sh, cfg.layers, wl.lengths, parents)
     pk = peaks()
-    attn_gbs = work["attn_bytes_per_layer"] / (attn_ms * 1e-3) / 1e9
-    attn_tf = work["attn_flops_per_layer"] / (attn_ms * 1e-3) / 1e12
+    # the dominant kernel is the attention kernel (with the merge kernel where a workload launches one): its duration is that
+    # of the attention stage replayed without the tile plan; the stage with its plan kernel is reported next to it (in a
+    # full cycle the plan runs under the tails of the state build and the selection, replayed alone it cannot)
+    attn_gbs = work["attn_bytes_per_layer"] / (kern_ms * 1e-3) / 1e9
+    attn_tf = work["attn_flops_per_layer"] / (kern_ms * 1e-3) / 1e12
     hbm = {"achieved": attn_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / pk["hbm_gbs"],
            "algorithmic_bytes_per_launch": work["attn_bytes_per_layer"]}
     tensor = {"achieved": attn_tf, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": attn_tf / pk["bf16_tflops_sustained"],
@@ -288,15 +291,14 @@ def run_ours(args, cfg):
     intensity = work["attn_flops_per_layer"] / work["attn_bytes_per_layer"]
     bound = "tensor" if (sh.dtype == "bf16" and intensity > ridge) else "hbm"
     cap = NCU_DRAM.get(cfg.name)
-    roofline = {"bound": bound, "kernel": f"tree_verify_attn attention stage (tile plan + {ATTN_KERNEL.get(cfg.name, 'attention kernels')}), "
-                                          "one layer, all sequences",
+    roofline = {"bound": bound, "kernel": f"tree_verify_attn: {ATTN_KERNEL.get(cfg.name, 'attention kernels')}, one layer, all sequences",
                 **(tensor if bound == "tensor" else hbm),
                 "traffic": cap["launch_bytes"] if cap else None,
                 "traffic_note": (f"ncu DRAM read+write of one {cap['kernel']} launch on this workload" if cap else "no ncu capture for this workload"),
-                "peak_source": pk["source"], "launch_ms": attn_ms,
-                # the same work over the duration of the attention kernels alone (without the tile plan's kernel)
-                "kernels_only": {"launch_ms": kern_ms, "frac_hbm": attn_gbs * attn_ms / kern_ms / pk["hbm_gbs"],
-                                 "frac_tensor": attn_tf * attn_ms / kern_ms / pk["bf16_tflops_sustained"]},
+                "peak_source": pk["source"], "launch_ms": kern_ms,
+                # the same work over the duration of the stage replayed with its tile plan kernel
+                "with_tile_plan": {"launch_ms": attn_ms, "frac_hbm": attn_gbs * kern_ms / attn_ms / pk["hbm_gbs"],
+                                   "frac_tensor": attn_tf * kern_ms / attn_ms / pk["bf16_tflops_sustained"]},
                 "flop_per_byte": intensity, "ridge_flop_per_byte": ridge,
                 "lengths": "algorithmic bytes and FLOPs from the initial prefix lengths (the caches grow by the accepted tokens while timed)",
                 "hbm": hbm, "tensor": tensor}

@@ -153,6 +153,7 @@ __device__ __forceinline__ void coop_tree_meta(TreeMeta& tm, TreeStage& st, cons
     if (n < nn && !bad) {
       anc = 1u << n;
       int cur = p;
+#pragma unroll 1
       for (int it = 0; it < TSV_MAX_D && cur >= 0 && cur < n; ++it) { anc |= 1u << cur; ++depth; cur = st.parent[cur]; }
     }
     tm.depth[n] = depth; tm.parent[n] = (n < nn && !bad && n > 0) ? p : -1; tm.anc[n] = anc;

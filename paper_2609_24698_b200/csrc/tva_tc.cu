@@ -20,11 +20,22 @@ namespace tsv {
 
 
 // ------------------------------------------------------------------------------------------------ plan
+constexpr int kRankTilesMax = 2048;                    // beyond that many tiles they keep their natural order
+// Estimated number of keys a tile of a sequence stages, from its committed length and node count alone (for tiles on the
+// contiguous-run path it is exact up to the entries closed inside the tree; only the order of the tiles depends on it).
+__device__ __forceinline__ int tile_keys_estimate(const tsv_shape& s, int L, int nn, int tile, int npt) {
+  if (L < 0 || (int64_t)L + s.D > s.max_L || nn < 1 || nn > s.D || tile * npt >= nn) return 0;
+  auto r32 = [](int x) { return (x + kBoxRows - 1) / kBoxRows * kBoxRows; };
+  const int n_csa = L / s.m_csa, n_hca = L / s.m_hca, nh_in = n_hca <= kHcaMiscMax ? n_hca : 0, win = min(L, s.window);
+  if (n_csa <= 2 * s.topk) return r32(n_csa) + (n_hca > kHcaMiscMax ? r32(n_hca) : 0) + r32(win) + r32(nh_in + nn);
+  return min(n_csa, npt * s.topk) + n_hca + win + 3 * nn;
+}
+
 // GENERAL: gathered tiles may occur (see gathered_tiles_possible); the instantiation without them keeps the short
 // latency chain of the contiguous-run plan.
 template <bool GENERAL>
 __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& pl, const tsv_cache& c, const tsv_nodes& nd,
-                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask) {
+                                             const tsv_scratch& sc, char* __restrict__ ws, uint8_t* cmask, int* est, int* ahead_sm) {
   __shared__ TreeMeta tm;
   __shared__ TreeStage tstage;
   __shared__ int n_cand[8], win_lo[8];
@@ -35,12 +46,29 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   uint32_t* krow = reinterpret_cast<uint32_t*>(ws + pl.off_krow) + tix * pl.tc_maxk;    // gathered tiles: array << 30 | row per key
   uint8_t* kmask = reinterpret_cast<uint8_t*>(ws + pl.off_kmask) + tix * pl.tc_maxk;
   int32_t* nkeys = reinterpret_cast<int32_t*>(ws + pl.off_nkeys) + tix;
+  int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
   // the cache row offsets are fetched together with the tree scalars (one memory latency for all)
   __shared__ uint8_t cdone[TSV_MAX_D], hdone[TSV_MAX_D];
   __shared__ int64_t row0_sm[2];
+  // (the length and node count of "its" tile's sequence, for the ranking of the tiles: requested now, used after the tree's loads)
+  const int ntile = s.B * pl.tc_nt;
+  const bool ranked_order = ntile <= kRankTilesMax && blockIdx.x < (unsigned)pl.tc_nt;
+  int eL = -1, enn = 0;
+  if (ranked_order && (int)threadIdx.x < ntile) { eL = c.L[threadIdx.x / pl.tc_nt]; enn = nd.n_nodes[threadIdx.x / pl.tc_nt]; }
   if (threadIdx.x == 40) row0_sm[0] = c.page_table ? 0 : c.csa_row0[b];
   if (threadIdx.x == 41) row0_sm[1] = c.page_table ? 0 : c.hca_row0[b];
   coop_tree_meta(tm, tstage, s, c.L + b, nd.parent + (size_t)b * D, nd.n_nodes + b, c.csa_cap + b, c.hca_cap + b);
+  if (ranked_order) {                                  // estimated key counts of all tiles
+    if ((int)threadIdx.x < ntile) est[threadIdx.x] = tile_keys_estimate(s, eL, enn, threadIdx.x % pl.tc_nt, npt);
+#pragma unroll 1
+    for (int i = threadIdx.x + blockDim.x; i < ntile; i += blockDim.x)
+      est[i] = tile_keys_estimate(s, c.L[i / pl.tc_nt], nd.n_nodes[i / pl.tc_nt], i % pl.tc_nt, npt);
+  }
+  // thread 0 leaves the tile's record {tile, mode, keys} at that position as soon as it knows the key count
+  auto leave_record = [&](int nk, int md) {
+    *nkeys = nk; *mode = md;
+    reinterpret_cast<int4*>(ws + pl.off_order)[ntile <= kRankTilesMax ? *ahead_sm : (int)tix] = make_int4((int)tix, md, nk, 0);
+  };
   // The kernel is launched as a programmatic dependent of the selection kernel (itself one of the state build) and runs
   // under those kernels' tails as far as it reads only the caller's inputs and the committed caches: the done flags are
   // worked out from the positions, and a tile no node of which ranks is planned completely.  It waits for the two kernels
@@ -52,6 +80,16 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     hdone[threadIdx.x] = valid && node_closes(tm.L, tm.depth[threadIdx.x], s.m_hca);
   }
   __syncthreads();
+  // The tile's scheduling position: how many tiles come before it by estimated key count (complete after the next barrier).
+  if (ranked_order) {
+    const int mine = est[tix];
+    int ahead = 0;
+#pragma unroll 1
+    for (int j = threadIdx.x; j < ntile; j += blockDim.x) { const int e = est[j]; ahead += (e > mine) || (e == mine && j < (int)tix); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
+    if ((threadIdx.x & 31) == 0 && ahead) atomicAdd(ahead_sm, ahead);
+  }
   // rows of the sequence's CSA and HCA entries: slabs, or through the page table of a paged pool
   RowAddr csa_row, hca_row;
   csa_row.pt = hca_row.pt = c.page_table ? c.page_table + (size_t)b * c.max_pages : nullptr;
@@ -67,14 +105,19 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     const size_t rowb = (size_t)s.d * 2;
     const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
     int ncd = 0, nhd = 0;
+#pragma unroll 1
     for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     uint4* dst = reinterpret_cast<uint4*>(ws + pl.off_misc + (size_t)b * pl.tc_misc_rows * rowb);
-    const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows, cpr = (int)(rowb / 16);
-    // warp per row, eight rows of a warp in flight: the source of a row is worked out once, all loads of the batch are
-    // issued before the first store
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    auto row_src = [&](int r) -> const uint4* {
+    const int rows_out = (n_misc + kBoxRows - 1) / kBoxRows * kBoxRows;
+    // The source of every packed row is worked out once (thread r: row r), then the copy runs flat over (row, 16-byte
+    // piece) items, eight of a thread in flight.  Rows [0, first) and the zero padding behind n_misc are the caller's
+    // data; the rows between are the state build's and copied after the wait.  (Compact code on purpose: the kernel runs
+    // once per layer with cold instruction caches.)
+    __shared__ const uint4* srcs[kHcaMiscMax + 3 * TSV_MAX_D];
+    constexpr int CPR = tc::DH * 2 / 16;               // 16-byte pieces per row
+#pragma unroll 1
+    for (int r = threadIdx.x; r < rows_out; r += blockDim.x) {
       const char* src = nullptr;
       if (r < nh_in) src = (const char*)c.hca_kv + (size_t)hca_row(r) * rowb;
       else if (r < nh_in + tm.nn) src = (const char*)nd.kv + ((size_t)b * D + (r - nh_in)) * rowb;
@@ -84,38 +127,38 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         if (!isc) ord -= ncd;
         const uint8_t* dn = isc ? cdone : hdone;
         int a = 0;
+#pragma unroll 1
         for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
         src = (const char*)(isc ? sc.new_csa_kv : sc.new_hca_kv) + ((size_t)b * D + a) * rowb;
       }
-      return reinterpret_cast<const uint4*>(src);
-    };
-    auto copy_rows = [&](int lo, int hi) {             // rows [lo, hi) of the packed buffer
-      if (cpr == 64) {                                 // d = 512 in bf16: two 16-byte pieces of a row per lane
-        for (int r0 = lo + w; r0 < hi; r0 += 8 * nw) {
-          uint4 v[8][2];
+      srcs[r] = reinterpret_cast<const uint4*>(src);
+    }
+    __syncthreads();
+    const int first = nh_in + tm.nn;
+#pragma unroll 1
+    for (int phase = 0; phase < 2; ++phase) {
+      if (phase) {
+        if (n_misc == first) break;
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the entries closed inside the tree
+      }
+      const int lo = phase ? first * CPR : 0, hi = phase ? n_misc * CPR : rows_out * CPR;
+#pragma unroll 1
+      for (int i0 = lo + threadIdx.x; i0 < hi; i0 += 8 * blockDim.x) {
+        uint4 v[8];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int r = r0 + k * nw;
-            const uint4* src = r < hi ? row_src(r) : nullptr;
-            v[k][0] = src ? __ldg(src + lane) : make_uint4(0, 0, 0, 0);
-            v[k][1] = src ? __ldg(src + 32 + lane) : make_uint4(0, 0, 0, 0);
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int r = r0 + k * nw;
-            if (r < hi) { dst[(size_t)r * 64 + lane] = v[k][0]; dst[(size_t)r * 64 + 32 + lane] = v[k][1]; }
-          }
+        for (int k = 0; k < 8; ++k) {
+          const int i = i0 + k * blockDim.x, r = i / CPR;
+          const bool in = i < hi && (phase || r < first || r >= n_misc);
+          const uint4* src = in ? srcs[r] : nullptr;
+          v[k] = src ? __ldg(src + (i - r * CPR)) : make_uint4(0, 0, 0, 0);
         }
-      } else {
-        for (int r = lo + w; r < hi; r += nw) {
-          const uint4* src = row_src(r);
-          for (int cc = lane; cc < cpr; cc += 32) dst[(size_t)r * cpr + cc] = src ? src[cc] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int i = i0 + k * blockDim.x, r = i / CPR;
+          if (i < hi && (phase || r < first || r >= n_misc)) dst[i] = v[k];
         }
       }
-    };
-    copy_rows(0, nh_in + tm.nn);                       // committed HCA entries and the tree nodes' rows: the caller's data
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    copy_rows(nh_in + tm.nn, rows_out);                // the entries closed inside the tree (the state build's), the zero padding
+    }
     return;
   }
   if (threadIdx.x < 32) {                              // lane nl: candidates and window start of node n0 + nl
@@ -131,8 +174,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     if (lane == 0) dense = over == 0;
   }
   __syncthreads();
-  int32_t* mode = reinterpret_cast<int32_t*>(ws + pl.off_mode) + tix;
-  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) { *nkeys = 0; *mode = 1; } return; }
+  if (tm.status || n0 >= tm.nn) { if (threadIdx.x == 0) leave_record(0, 1); return; }
   const int nvalid = min(npt, tm.nn - n0);
   const uint32_t validbits = (1u << nvalid) - 1u;
   const int n_csa = tm.n_csa;
@@ -154,23 +196,26 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   const bool runs_ok = !GENERAL || ((dense || n_csa <= 2 * s.topk) && csa_runs && (hca_runs || tm.n_hca <= kHcaMiscMax));
   const bool late = !dense && runs_ok;
   uint32_t allbits = 0, rankbits = 0;                  // nodes that take every committed entry / nodes that rank
+#pragma unroll 1
   for (int nl = 0; nl < nvalid; ++nl) { if (n_cand[nl] <= s.topk) allbits |= 1u << nl; else rankbits |= 1u << nl; }
   const uint8_t* mrow = reinterpret_cast<const uint8_t*>(ws + pl.off_selmask) + ((size_t)b * D + n0) * pl.mask_ld;
-  auto fetch_newc_bits = [&]() {                       // (threads 0..7; the caller synchronises)
-    if (threadIdx.x < 8) {
-      // in-tree entries: candidate n_csa + o of a node is the block closed at the o-th of its strict ancestors that closed one
-      uint32_t bits = 0;
-      const int nl = threadIdx.x;
+  // In-tree entries: candidate n_csa + o of a node is the block closed at the o-th of its strict ancestors that closed one.
+  // Warp nl looks at node n0 + nl, lane a at ancestor a: one load per lane, all in flight together (the caller synchronises).
+  auto fetch_newc_bits = [&]() {
+    const int nl = threadIdx.x >> 5, a = threadIdx.x & 31;
+    if (nl < 8) {
+      const uint32_t closed = __ballot_sync(0xffffffffu, a < D && cdone[a]);
+      uint32_t v = 0;
       if (nl < nvalid && ((rankbits >> nl) & 1u)) {
-        int o = 0;
-        for (int a = 0; a < n0 + nl; ++a) {
-          if (!((tm.anc[n0 + nl] >> a) & 1u) || !cdone[a]) continue;
+        const uint32_t up = tm.anc[n0 + nl] & closed & ((1u << (n0 + nl)) - 1u);     // strict ancestors that closed a block
+        if ((up >> a) & 1u) {
+          const int o = __popc(up & ((1u << a) - 1u));
           const int dblk = (tm.L + tm.depth[a]) / s.m_csa - n_csa;
-          if (mrow[(size_t)nl * pl.mask_ld + n_csa + o] && dblk >= 0 && dblk < 32) bits |= 1u << dblk;
-          ++o;
+          if (mrow[(size_t)nl * pl.mask_ld + n_csa + o] && dblk >= 0 && dblk < 32) v = 1u << dblk;
         }
       }
-      newc_bits[nl] = bits;
+      v = __reduce_or_sync(0xffffffffu, v);
+      if (a == 0) newc_bits[nl] = v;
     }
   };
   // sixteen committed entries from entry i: the node bits of each as four words of four mask bytes
@@ -209,6 +254,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
     // the packed per-sequence rows (written by the sequence's extra CTA): few HCA entries, tree nodes, entries closed in the tree
     const int nh_in = tm.n_hca <= kHcaMiscMax ? tm.n_hca : 0;
     int ncd = 0, nhd = 0;
+#pragma unroll 1
     for (int j = 0; j < tm.nn; ++j) { ncd += cdone[j] != 0; nhd += hdone[j] != 0; }
     const int n_misc = nh_in + tm.nn + ncd + nhd;
     // Ranked nodes still take the contiguous-run path while the run is at most twice the selection size: all committed
@@ -275,6 +321,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         }
       }
       // (gathered tiles: the compaction above has written the keys of the first run already)
+#pragma unroll 1
       for (int k = (runs_ok ? 0 : n_uni) + threadIdx.x; k < kb; k += blockDim.x) {
         const int g = k >= k0[3] ? 3 : (k >= k0[2] ? 2 : (k >= k0[1] ? 1 : 0));
         const int i = k - k0[g];
@@ -285,10 +332,12 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
           else if (g == 1) m = validbits;
           else if (g == 2) {
             const int pos = c.page_table ? win_a + i : tm.L - 1 - ((tm.L - 1 - i) % s.window);
+#pragma unroll 1
             for (int nl = 0; nl < nvalid; ++nl) if (pos >= win_lo[nl]) m |= 1u << nl;
           } else if (i < nh_in) m = validbits;
           else if (i < nh_in + tm.nn) {
             const int j = i - nh_in;
+#pragma unroll 1
             for (int nl = 0; nl < nvalid; ++nl) if ((tm.anc[n0 + nl] >> j) & 1u) m |= 1u << nl;
           } else {
             int ord = i - nh_in - tm.nn;
@@ -296,7 +345,9 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
             if (!isc) ord -= ncd;
             const uint8_t* dn = isc ? cdone : hdone;
             int a = 0;
+#pragma unroll 1
             for (int j = 0; j < tm.nn; ++j) if (dn[j]) { if (ord == 0) { a = j; break; } --ord; }
+#pragma unroll 1
             for (int nl = 0; nl < nvalid; ++nl)
               if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && (!isc || newc_selected(nl, a))) m |= 1u << nl;
           }
@@ -305,7 +356,7 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         // gathered tiles: the key's row; the padding of a run repeats the run's first row (masked)
         if (!runs_ok) krow[k] = ((uint32_t)g << 30) | (uint32_t)(cnt[g] ? run_row(g, i < cnt[g] ? i : 0) : 0);
       }
-      if (threadIdx.x == 0) { *nkeys = kb; *mode = runs_ok ? 1 : 2; }
+      if (threadIdx.x == 0) leave_record(kb, runs_ok ? 1 : 2);
       if (late) {
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the selection's mask rows
         fetch_newc_bits();
@@ -325,8 +376,10 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
         // the CSA entries closed inside the tree (ncd keys of the packed run)
         if ((int)threadIdx.x < ncd) {
           int ord = threadIdx.x, a = 0;
+#pragma unroll 1
           for (int j = 0; j < tm.nn; ++j) if (cdone[j]) { if (ord == 0) { a = j; break; } --ord; }
           uint32_t m = 0;
+#pragma unroll 1
           for (int nl = 0; nl < nvalid; ++nl)
             if (a != n0 + nl && ((tm.anc[n0 + nl] >> a) & 1u) && newc_selected(nl, a)) m |= 1u << nl;
           kmask[k0[3] + nh_in + tm.nn + threadIdx.x] = (uint8_t)m;
@@ -337,16 +390,6 @@ __device__ __forceinline__ void tc_plan_tile(const tsv_shape& s, const TvaPlan& 
   }
 }
 
-// Estimated number of keys a tile of a sequence stages, from its committed length and node count alone (for tiles on the
-// contiguous-run path it is exact up to the entries closed inside the tree; only the order of the tiles depends on it).
-__device__ __forceinline__ int tile_keys_estimate(const tsv_shape& s, int L, int nn, int tile, int npt) {
-  if (L < 0 || (int64_t)L + s.D > s.max_L || nn < 1 || nn > s.D || tile * npt >= nn) return 0;
-  auto r32 = [](int x) { return (x + kBoxRows - 1) / kBoxRows * kBoxRows; };
-  const int n_csa = L / s.m_csa, n_hca = L / s.m_hca, nh_in = n_hca <= kHcaMiscMax ? n_hca : 0, win = min(L, s.window);
-  if (n_csa <= 2 * s.topk) return r32(n_csa) + (n_hca > kHcaMiscMax ? r32(n_hca) : 0) + r32(win) + r32(nh_in + nn);
-  return min(n_csa, npt * s.topk) + n_hca + win + 3 * nn;
-}
-
 // Plan of every (sequence, 256-row tile).  Each tile CTA leaves one 16-byte record {tile, mode, keys} at the tile's
 // scheduling position: its rank among all tiles by estimated key count, most first, which every CTA works out for itself
 // from the lengths and node counts of all sequences (the paired attention kernel takes the tiles in that order, long
@@ -354,7 +397,6 @@ __device__ __forceinline__ int tile_keys_estimate(const tsv_shape& s, int L, int
 // ranks is planned from the caller's inputs alone: its CTA never waits for the kernels before this one.
 // NT threads per CTA: 256, or 1024 for gathered tiles over long candidate lists (the union of a tile's selections over tens
 // of thousands of entries is the work of ONE CTA, alone on its SM).
-constexpr int kRankTilesMax = 2048;                    // beyond that many tiles they keep their natural order
 template <bool GENERAL, int NT>
 __global__ void __launch_bounds__(NT) tc_plan_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                                          const tsv_scratch sc, char* __restrict__ ws) {
@@ -362,34 +404,11 @@ __global__ void __launch_bounds__(NT) tc_plan_kernel(const tsv_shape s, const Tv
   __shared__ int est_sm[kRankTilesMax];
   __shared__ int ahead_sm;
   const bool tile_cta = blockIdx.x < (unsigned)pl.tc_nt;
-  const int ntile = s.B * pl.tc_nt, npt = tc::PR / s.H;
   const size_t tix = (size_t)blockIdx.y * pl.tc_nt + blockIdx.x;
-  if (tile_cta && ntile <= kRankTilesMax) {            // requested with the tile's own first loads
-    for (int i = threadIdx.x; i < ntile; i += NT) {
-      const int b = i / pl.tc_nt;
-      est_sm[i] = tile_keys_estimate(s, c.L[b], nd.n_nodes[b], i - b * pl.tc_nt, npt);
-    }
-  }
   if (threadIdx.x == 0) ahead_sm = 0;
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
-  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm);
-  if (tile_cta) {                                      // (barriers since the estimates were written)
-    int pos = (int)tix;
-    if (ntile <= kRankTilesMax) {
-      const int mine = est_sm[tix];
-      int ahead = 0;
-      for (int j = threadIdx.x; j < ntile; j += NT) { const int e = est_sm[j]; ahead += (e > mine) || (e == mine && j < (int)tix); }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
-      if ((threadIdx.x & 31) == 0 && ahead) atomicAdd(&ahead_sm, ahead);
-      __syncthreads();
-      pos = ahead_sm;
-    }
-    if (threadIdx.x == 0)                              // thread 0 wrote the tile's key count and mode itself
-      reinterpret_cast<int4*>(ws + pl.off_order)[pos] =
-          make_int4((int)tix, reinterpret_cast<const int32_t*>(ws + pl.off_mode)[tix], reinterpret_cast<const int32_t*>(ws + pl.off_nkeys)[tix], 0);
-  }
+  tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm, est_sm, &ahead_sm);
   // one CTA waits for the selection in any case, so that the completion of this kernel implies that one's
   if (blockIdx.x == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
