@@ -16,6 +16,7 @@ __device__ inline void path_entries(PathEntries& pe, const TreeMeta& tm, const t
                                     const uint8_t* csa_done_b, const uint8_t* hca_done_b) {
   pe.n_newc = pe.n_newh = 0;
   const uint32_t a = tm.anc[n] & ~(1u << n);
+#pragma unroll 1                                        // (compact code: the kernels run with cold instruction caches)
   for (int j = 0; j < n; ++j) {
     if (!((a >> j) & 1u)) continue;
     if (csa_done_b[j]) { pe.newc[pe.n_newc] = j; pe.newc_blk[pe.n_newc++] = (tm.L + tm.depth[j]) / s.m_csa; }

@@ -16,8 +16,10 @@ namespace tsv {
 namespace fsel {
 
 constexpr int DI = 128;                       // indexer width (bf16: 256-byte rows)
-constexpr int KPT = 9;                        // candidates per thread: 9 x 256 >= kIdxFusedMax + TSV_MAX_D
-static_assert(kIdxFusedMax + TSV_MAX_D <= KPT * 256, "candidate lists must fit the in-register keys");
+// candidates per thread (keys in registers): 3 for lists of up to 768 candidates, else 9 (9 x 256 >= kIdxFusedMax + TSV_MAX_D);
+// two instantiations, so that the short lists of the common shapes do not step through the predicated code of nine
+constexpr int KPT_SHORT = 3, KPT_LONG = 9;
+static_assert(kIdxFusedMax + TSV_MAX_D <= KPT_LONG * 256, "candidate lists must fit the in-register keys");
 
 __device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -34,7 +36,7 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
 
 // Dynamic shared memory: [4][128] bf16 queries (heads beyond HI zero) | scores [score_cap] fp32 | two buffers of `rows`
 // staged indexer rows of 256 bytes (16-byte pieces XOR-swizzled by the row, so that ldmatrix reads without conflicts).
-template <bool PAGED>
+template <bool PAGED, int KPT>
 __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                             const tsv_scratch sc, int32_t* __restrict__ topk_user, char* __restrict__ ws,
                                                             int32_t* __restrict__ status, const int rows, const int score_cap) {
@@ -305,15 +307,16 @@ int launch_topk_fused(const tsv_shape& s, const TvaPlan& p, const tsv_cache& c, 
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;          // may start under the state build's tail (it waits inside)
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  if (c.page_table) {
-    TSV_PREP(topk_fused_kernel<true>);
-    if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-    cudaLaunchKernelEx(&cfg, topk_fused_kernel<true>, s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
-  } else {
-    TSV_PREP(topk_fused_kernel<false>);
-    if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-    cudaLaunchKernelEx(&cfg, topk_fused_kernel<false>, s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);
-  }
+#define TSV_FUSED_LAUNCH(PG_, KPT_)                                                                                                     \
+  do {                                                                                                                                 \
+    TSV_PREP((topk_fused_kernel<PG_, KPT_>));                                                                                          \
+    if (bytes > 40 * 1024) cudaFuncSetAttribute(topk_fused_kernel<PG_, KPT_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
+    cudaLaunchKernelEx(&cfg, topk_fused_kernel<PG_, KPT_>, s, p, c, nd, sc, topk_idx, ws, status, rows, score_cap);                     \
+  } while (0)
+  const bool shortl = p.cand_cap <= fsel::KPT_SHORT * 256;
+  if (c.page_table) { if (shortl) TSV_FUSED_LAUNCH(true, fsel::KPT_SHORT); else TSV_FUSED_LAUNCH(true, fsel::KPT_LONG); }
+  else { if (shortl) TSV_FUSED_LAUNCH(false, fsel::KPT_SHORT); else TSV_FUSED_LAUNCH(false, fsel::KPT_LONG); }
+#undef TSV_FUSED_LAUNCH
   count_launch();
   return cudaGetLastError() == cudaSuccess ? TSV_OK : TSV_ERR_CUDA;
 }
