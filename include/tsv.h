@@ -20,12 +20,14 @@
  *   - Stream order: the calls of a layer run in the order given above on one stream.  Some kernels of
  *     tree_verify_attn are launched as PROGRAMMATIC DEPENDENTS of the kernel before them on the stream: the part
  *     of them that reads only the call's inputs (tsv_nodes, the committed tsv_cache) may run before that kernel
- *     has finished; they wait for it before they read anything the library's own kernels write.  For the
- *     caller this matters in one case only: a kernel of the caller's that is enqueued directly before
- *     tree_verify_attn, WRITES that call's inputs and itself signals its dependents early
- *     (griddepcontrol.launch_dependents / cudaTriggerProgrammaticLaunchCompletion) must have written those
- *     inputs before it signals.  Kernels that do not use that feature are complete before any of the
- *     library's kernels starts, as always.
+ *     has finished, and that part already writes the call's workspace, topk_idx and status; they wait for
+ *     it before they read anything the library's own kernels write.  For the caller this matters in one
+ *     case only: a kernel of the caller's that is enqueued directly before tree_verify_attn and itself
+ *     signals its dependents early (griddepcontrol.launch_dependents /
+ *     cudaTriggerProgrammaticLaunchCompletion) must, before it signals, have written whatever it writes
+ *     of that call's inputs and have read whatever it reads of that call's workspace, topk_idx and
+ *     status.  Kernels that do not use that feature are complete before any of the library's kernels
+ *     starts, as always.
  *   - "storage dtype" = tsv_shape.dtype (fp32 or bf16): all vectors and cache rows.  All
  *     partial-block accumulators, gates and weights are fp32.
  *   - Row-major, innermost dimension contiguous, no padding.  Vector pointers must be

@@ -25,7 +25,7 @@ __device__ __forceinline__ void add_peer(int* p, uint32_t rank, int v) {
 }  // namespace lsel
 
 template <typename T>
-__global__ void __launch_bounds__(lsel::THREADS) topk_long_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
+__global__ void __launch_bounds__(lsel::THREADS, 2) topk_long_kernel(const tsv_shape s, const TvaPlan pl, const tsv_cache c, const tsv_nodes nd,
                                                                   const tsv_scratch sc, int32_t* __restrict__ topk_user,
                                                                   char* __restrict__ ws, int32_t* __restrict__ status) {
   using namespace lsel;
