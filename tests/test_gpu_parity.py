@@ -24,7 +24,7 @@ def _np(t):
 
 def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None, check_recompress=False,
              parent_fn=None, return_engine=False, plant=None, graph=False, recompress_pairs=None, on_cycle=None,
-             per_row=False, incremental_caches=False, page_tokens=0, exact_topk=False):
+             per_row=False, incremental_caches=False, page_tokens=0, exact_topk=False, want_topk=True):
     """Advance oracle and device cycle by cycle from the same prefix; compare everything each cycle.
     out_pairs: None = compare attention outputs of every (layer, seq); else callable cycle -> iterable of pairs.
     plant: callable(states, lengths) editing the oracle's prefix states in place before they are uploaded.
@@ -38,6 +38,8 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
     page_tokens: the persistent caches live in a paged pool with pages of that many tokens (shuffled page tables).
     exact_topk: the device's selection must BE the oracle's (for inputs whose scores tie exactly, where the tie band of the
            usual check would accept a wrong tie-break).
+    want_topk: False = the call gets no buffer for the index lists (the way the benchmark calls it: selection kernels may
+           then skip work nobody reads); the outputs are compared with the oracle's own selection.
     per_row: also require every (node, head) output row to be within the tolerance of ITS OWN max magnitude (for inputs
            where a few rows are far larger than the rest, so that the tensor-wide bound would say little about the others)."""
     from paper_2609_24698_b200 import binding as tsv, harness as hz
@@ -52,7 +54,7 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
                      for l in range(cfg.layers)]                 # per tensor: list of pieces, joined when checked
     ccap, hcap = hz.capacities(sh, lengths, cycles * sh.D)
     max_L = int(lengths.max()) + (cycles + 1) * sh.D
-    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=True, page_tokens=page_tokens)
+    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, max_L, flags=flags, want_topk=want_topk, page_tokens=page_tokens)
     for l in range(cfg.layers):
         for b in range(sh.B):
             hz.fill_cache(eng.caches[l], sh, b, int(lengths[b]), state_arrays(states[l][b]))
@@ -126,10 +128,12 @@ def lockstep(cfg, cycles, flags=0, lengths=None, n_nodes_fn=None, out_pairs=None
         for (l, b) in pairs:
             nb, nn = per_seq(nodes[l], b), int(n_nodes[b])
             ref_out, ref_sel = O.tree_verify_attn(states[l][b], sh, nb, parent[b], nn, scs[(l, b)])
-            g_idx = eng.topk_idx[l][b].cpu().numpy()
-            same = all([check_topk(sh, states[l][b], nb, parent[b], n, scs[(l, b)], g_idx[n], ref_sel[n]) for n in range(nn)])
-            assert np.all(g_idx[nn:] == -1)
-            assert same or not exact_topk, f"cycle {cyc} layer {l} seq {b}: selection differs from the oracle's"
+            same = True
+            if want_topk:
+                g_idx = eng.topk_idx[l][b].cpu().numpy()
+                same = all([check_topk(sh, states[l][b], nb, parent[b], n, scs[(l, b)], g_idx[n], ref_sel[n]) for n in range(nn)])
+                assert np.all(g_idx[nn:] == -1)
+                assert same or not exact_topk, f"cycle {cyc} layer {l} seq {b}: selection differs from the oracle's"
             if not same:       # inside the tie band: evaluate the oracle with the device's selection
                 ref_out, _ = O.tree_verify_attn(states[l][b], sh, nb, parent[b], nn, scs[(l, b)], forced_sel=[g_idx[n] for n in range(nn)])
             e = rel_err(_np(eng.out[l][b]), ref_out)
@@ -476,6 +480,17 @@ def test_tc_planted_peaks_ranked_tiles():
     gathered tiles, single- and multi-chunk."""
     cfg = synth.Config("tc_peaks_ranked", 82, synth.Shape("bf16", 4, 8, topk=256, **BENCH_HEADS), L_min=1, L_max=1, seed=4)
     lockstep(cfg, cycles=1, lengths=[1500, 2040, 2600, 4400], plant=_plant_peaks(cfg, gap_nats=16.0), per_row=True)
+
+
+def test_tc_without_index_lists_ranked_and_unranked_sequences():
+    """The call as the benchmark makes it: no buffer for the index lists.  Selection CTAs of nodes that cannot rank then
+    leave after one load, tiles without ranking nodes are planned without waiting for the selection, tiles with ranking
+    nodes finish their key masks after it.  Lengths: far below the ranking threshold (top-k 256 of L / 4 entries), just
+    below it so that only deep nodes rank (entries closed inside the tree count as candidates) and the sequence crosses
+    it while the cycles run, above it, and above twice the top-k (gathered tiles); sm_scale 8 makes a wrongly masked key
+    visible."""
+    cfg = synth.Config("tc_no_lists", 84, synth.Shape("bf16", 7, 8, topk=256, sm_scale=8.0, **BENCH_HEADS), L_min=1, L_max=1, seed=6)
+    lockstep(cfg, cycles=4, lengths=[200, 900, 1003, 1015, 1023, 1500, 2300], want_topk=False, per_row=True)
 
 
 def test_tc_peaked_scale100():
