@@ -49,7 +49,6 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
   __shared__ uint32_t hist[3][128];                    // radix histogram, two 16-bit bins per word (a list has < 65536 candidates); the buffers rotate between passes
   __shared__ int wsum[9];
   __shared__ int64_t row0_sm;
-  __shared__ uint8_t cdone_sm[TSV_MAX_D], hdone_sm[TSV_MAX_D];
   bf16* iqs = reinterpret_cast<bf16*>(dsm);
   float* ssm = reinterpret_cast<float*>(dsm + 4 * DI * 2);
   unsigned char* stage = dsm + 4 * DI * 2 + (size_t)score_cap * 4;
@@ -104,15 +103,20 @@ __global__ void __launch_bounds__(256, 4) topk_fused_kernel(const tsv_shape s, c
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
   if (may_rank) issue(0);
-  if (t < D) {                                         // the done flags of the sequence's nodes, from their positions
+  if (t < 32) {
+    // Warp 0, lane j = node j: which nodes close a block (from their positions), and from that the entries on this node's
+    // path -- the strict ancestors that closed a CSA / HCA block, root first -- by ballots instead of a loop of one thread.
     const bool valid = !tm.status && t < tm.nn;
-    cdone_sm[t] = valid && node_closes(tm.L, tm.depth[t], s.m_csa);
-    hdone_sm[t] = valid && node_closes(tm.L, tm.depth[t], s.m_hca);
-  }
-  __syncthreads();
-  if (t == 0) {
-    if (tm.status && n == 0) atomicOr(status + b, tm.status);
-    if (live) path_entries(pe, tm, s, n, cdone_sm, hdone_sm);
+    const uint32_t strict = live ? tm.anc[n] & ~(1u << n) : 0u;
+    const uint32_t cm = __ballot_sync(0xffffffffu, valid && node_closes(tm.L, tm.depth[t], s.m_csa)) & strict;
+    const uint32_t hm = __ballot_sync(0xffffffffu, valid && node_closes(tm.L, tm.depth[t], s.m_hca)) & strict;
+    const uint32_t lower = (1u << t) - 1u;
+    if ((cm >> t) & 1u) { const int o = __popc(cm & lower); pe.newc[o] = t; pe.newc_blk[o] = (tm.L + tm.depth[t]) / s.m_csa; }
+    if ((hm >> t) & 1u) pe.newh[__popc(hm & lower)] = t;
+    if (t == 0) {
+      pe.n_newc = __popc(cm); pe.n_newh = __popc(hm);
+      if (tm.status && n == 0) atomicOr(status + b, tm.status);
+    }
   }
   __syncthreads();
   if (!live) {
