@@ -165,7 +165,8 @@ def workload_config(cfg, args):
             "l2_policy": "inputs larger than L2: every cycle reads a different input set (q alone is 268 MB per cycle)",
             "launch": "one CUDA graph replay per cycle", "hca_refresh_schedule": getattr(args, "schedule", "timely"),
             "cache_layout": (f"paged pool, {args.page_tokens}-token pages, one page table for the CSA and HCA layers"
-                             if getattr(args, "page_tokens", 0) else "flat slab per sequence")}
+                             if getattr(args, "page_tokens", 0) else "flat slab per sequence"),
+            "topk_idx": "not requested (tree_verify_attn's optional output; the selection is used by the attention only)"}
 
 
 # ------------------------------------------------------------------------------------------ our arm
