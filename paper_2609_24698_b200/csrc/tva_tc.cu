@@ -409,6 +409,7 @@ __global__ void __launch_bounds__(NT) tc_plan_kernel(const tsv_shape s, const Tv
   if (threadIdx.x < 2 && tile_cta)                      // finished-chunk counters of the tile's two 128-row halves
     reinterpret_cast<int32_t*>(ws + pl.off_tcnt)[tix * 2 + threadIdx.x] = 0;
   tc_plan_tile<GENERAL>(s, pl, c, nd, sc, ws, cmask_sm, est_sm, &ahead_sm);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // (at the END of the CTA's work: the attention kernel's CTAs take their places as this kernel's leave)
   // one CTA waits for the selection in any case, so that the completion of this kernel implies that one's
   if (blockIdx.x == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }

@@ -139,6 +139,9 @@ tc_attn_pair_kernel(const __grid_constant__ pair::MapSet maps, const tsv_shape s
   // the two CTAs of a pair are neighbours in x; pairs take the (sequence, tile) items in the order the plan kernel left
   // (most keys first)
   const int chunk = blockIdx.y;
+  // launched as a programmatic dependent of the tile plan: the CTAs take their places while that kernel's last CTAs
+  // finish, and read nothing before it has completed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int4 rec = reinterpret_cast<const int4*>(ws + pl.off_order)[blockIdx.x >> 1];   // {tile index, mode, keys, -}: one load
   const int item = rec.x;
   const int b = item / pl.tc_nt, tile = item % pl.tc_nt;
@@ -760,11 +763,13 @@ int launch_tva_tc_pair(const tsv_shape& s, const TvaPlan& p, const TvaTcPrep& pr
   cfg.blockDim = dim3(pair::TTHREADS, 1, 1);
   cfg.dynamicSmemBytes = pair::SMEM_X;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;          // may take its places under the plan kernel's tail (it waits inside)
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t le = general ? cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel<true>, ms, s, p, out, ws, status)
                                  : cudaLaunchKernelEx(&cfg, tc_attn_pair_kernel<false>, ms, s, p, out, ws, status);
   if (le != cudaSuccess) {
