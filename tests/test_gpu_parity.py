@@ -493,11 +493,12 @@ def test_tc_without_index_lists_ranked_and_unranked_sequences():
     lockstep(cfg, cycles=4, lengths=[200, 900, 1003, 1015, 1023, 1500, 2300], want_topk=False, per_row=True)
 
 
-def test_tc_more_tiles_than_the_plan_ranks():
-    """More than 2048 plan tiles (1030 sequences x 2 tiles): the plan kernel then leaves the tile records in their natural
-    order instead of ranking the tiles by key count.  Short prefixes; branch states, acceptance and caches are compared for
-    every sequence, the attention output for a sample (the first, the last, and ten in between)."""
-    B = 1030
+@pytest.mark.parametrize("B", [200, 1030])
+def test_tc_more_tiles_than_the_plan_ranks(B):
+    """Many plan tiles.  1030 sequences x 2 tiles = more than 2048: the plan kernel then leaves the tile records in their
+    natural order instead of ranking the tiles by key count.  200 sequences = 400 tiles: ranked, with more tiles than a plan
+    CTA has threads (every thread sums over several tiles).  Short prefixes; branch states, acceptance and caches are
+    compared for every sequence, the attention output for a sample (the first, the last, and some in between)."""
     cfg = synth.Config("tc_many_tiles", 85, synth.Shape("bf16", B, 8, topk=512, sm_scale=8.0, **BENCH_HEADS), L_min=40, L_max=200, seed=7)
     sample = [(0, b) for b in [0, B - 1] + list(range(97, B - 1, 103))]
     lockstep(cfg, cycles=1, out_pairs=lambda c: sample)
