@@ -636,16 +636,24 @@ def test_graph_replayed_cycles_match_oracle_and_eager():
     assert torch.equal(eng_g.accept_path, eng_e.accept_path) and torch.equal(eng_g.accept_len, eng_e.accept_len)
 
 # ------------------------------------------------------------------------------------------------ status / error paths
-def test_device_detected_errors_commit_nothing():
+@pytest.mark.parametrize("path", ["cuda_cores", "tensor_cores_without_index_lists"])
+def test_device_detected_errors_commit_nothing(path):
+    """Flagged sequences (parent array out of order, node count out of range, no room for a closing entry) next to a good
+    one: status bits, zero outputs, nothing committed.  Once on a small fp32 shape (CUDA-core attention) and once on the
+    benchmark head shape without a buffer for the index lists (selection CTAs that leave early, the tile plan's empty
+    records, the paired kernel's zero fill)."""
     from paper_2609_24698_b200 import binding as tsv, harness as hz
-    cfg = synth.small_config(dtype="fp32", B=4, D=6, H=2, d=16, m_csa=2, topk=3, HI=1, di=8, m_hca=3, window=8,
-                             L_min=4, L_max=9, layers=2, seed=40)
+    if path == "cuda_cores":
+        cfg = synth.small_config(dtype="fp32", B=4, D=6, H=2, d=16, m_csa=2, topk=3, HI=1, di=8, m_hca=3, window=8,
+                                 L_min=4, L_max=9, layers=2, seed=40)
+    else:
+        cfg = synth.Config("tc_flagged", 86, synth.Shape("bf16", 4, 8, topk=512, **BENCH_HEADS), L_min=300, L_max=900, seed=8)
     sh = cfg.shape
     lengths = synth.prefix_lengths(cfg)
     states = oracle_states(cfg, lengths)
     ccap, hcap = hz.capacities(sh, lengths, 64)
     ccap[3] = int(lengths[3]) // sh.m_csa            # sequence 3: no room for the entry a deep path could close
-    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, int(lengths.max()) + 64, want_topk=True)
+    eng = hz.VerifyEngine(sh, cfg.layers, ccap, hcap, int(lengths.max()) + 64, want_topk=(path == "cuda_cores"))
     for l in range(cfg.layers):
         for b in range(sh.B):
             hz.fill_cache(eng.caches[l], sh, b, int(lengths[b]), state_arrays(states[l][b]))
