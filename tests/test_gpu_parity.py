@@ -577,6 +577,13 @@ def test_paged_pool_tensor_core_path(page_tokens, m_csa, topk, lengths):
                        L_min=1, L_max=1, seed=page_tokens + topk)
     lockstep(cfg, cycles=3, lengths=lengths, page_tokens=page_tokens, check_recompress="final")
 
+
+def test_paged_pool_tensor_core_path_without_index_lists():
+    """The paged pool called the way the benchmark calls it (no buffer for the index lists): sequences that cannot rank,
+    one at the ranking threshold, ranked contiguous-run tiles and a gathered one."""
+    cfg = synth.Config("paged_tc_no_lists", 95, synth.Shape("bf16", 5, 8, topk=256, sm_scale=8.0, **BENCH_HEADS), layers=1, L_min=1, L_max=1, seed=9)
+    lockstep(cfg, cycles=3, lengths=[300, 1015, 1023, 1700, 2600], page_tokens=128, want_topk=False, per_row=True)
+
 # ------------------------------------------------------------------------------------------------ refresh schedules
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_c128_deferred_refresh_schedule_small(dtype):
