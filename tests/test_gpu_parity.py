@@ -313,6 +313,28 @@ def test_cfg4_full_size_stack_50_cycles():
     assert cfg.cycles == 50 and ranked[-1] >= 2, "the run is meant to end with sequences past top-k candidates"
 
 
+def test_cfg4_full_size_as_the_benchmark_launches_it():
+    """The benchmark workload in the benchmark's launch configuration: every cycle one replay of a CUDA graph captured
+    over a fixed input slot, no buffer for the index lists.  24 cycles, so that the run ends with sequences whose nodes
+    rank; branch states, acceptance and appended cache rows every cycle, attention outputs for all pairs on the first and
+    last cycle and for a seeded sample plus the longest sequence in between."""
+    cfg = synth.CONFIGS["cfg4"]
+    sh = cfg.shape
+    rng = np.random.default_rng(44)
+    longest = int(np.argmax(synth.prefix_lengths(cfg)))
+    everyone = [(l, b) for l in range(cfg.layers) for b in range(sh.B)]
+    cycles = 24
+    def pairs(cyc):
+        if cyc in (0, cycles - 1):
+            return everyone
+        return [(int(rng.integers(0, cfg.layers)), int(rng.integers(0, sh.B))) for _ in range(12)] + [(cyc % cfg.layers, longest)]
+    ranked = []
+    def watch(cyc, eng, states):
+        ranked.append(sum(S.L // sh.m_csa > sh.topk for S in states[0]))
+    lockstep(cfg, cycles=cycles, out_pairs=pairs, incremental_caches=True, on_cycle=watch, graph=True, want_topk=False)
+    assert ranked[-1] >= 1, "the run is meant to end with a sequence past top-k candidates"
+
+
 def test_cfg5_long_context_100_cycles():
     """131072-token prefixes, top-k 2048 of 32768 candidates, 100 verify-accept-refresh cycles: branch states,
     acceptance and caches every cycle; attention outputs and selections on cycles 0, 1, 2, then every 16th and the
